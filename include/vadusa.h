@@ -1,0 +1,239 @@
+/*
+ * vadusa.h — C ABI of libvadusa: the tree draft-and-verify step of VADUSA
+ * (MEDUSA-style speculative decoding with a tolerance rule for a VALL-E-style
+ * decoder-only speech-token language model) on NVIDIA B200 (sm_100a).
+ *
+ * Conventions
+ *  - Every call returns a vadusa_status; no C++ exception crosses this boundary.
+ *  - Pointers are DEVICE pointers unless the parameter name starts with h_ (host).
+ *    Any output pointer may be NULL, which means "do not write it".
+ *  - The caller owns every buffer it passes (weights, KV pool, workspace, block
+ *    table, inputs, outputs) and keeps it alive until vadusa_destroy.  The
+ *    library owns only the opaque vadusa_ctx (host memory, two CUDA events and
+ *    a few pinned host words).
+ *  - All device work is enqueued on the stream given in the configuration, in
+ *    call order; calls do not synchronise unless they say so.
+ *  - Errors found on the host make the call return at once with a message in
+ *    vadusa_last_error.  Errors found on the device (capacity exhausted, a
+ *    bounded wait that expired) set bits in a device error word; they surface
+ *    as the return value of the next call that synchronises
+ *    (vadusa_get_lengths, vadusa_generate, vadusa_check).
+ *  - There is no CPU path: if no sm_100 device is present vadusa_init fails
+ *    with VADUSA_ECUDA.
+ *
+ * Model (paper Sec. III-A.1; details the paper leaves to VALL-E are fixed here):
+ *  a pre-LayerNorm decoder-only transformer with learned absolute positions,
+ *  multi-head attention (every head has its own K/V), ReLU feed-forward, biases
+ *  on all projections except the vocabulary heads, LayerNorm with affine
+ *  parameters, one running position index over [phonemes ; prompt ; generated].
+ *  Phoneme tokens use their own embedding table; on this interface a phoneme id
+ *  p is written as the token id vocab + p.
+ *  Draft head i (i = 1..n_draft_heads) is z = h + SiLU(W_i h + b_i), then its own
+ *  vocabulary projection U_i z (Sec. II-A, III-A.1); h is the final-LayerNorm
+ *  output at the last committed token.
+ *
+ * Numeric types: dtype 0 keeps weights, K/V and activations in fp32 (plain
+ *  fp32 FMA arithmetic).  dtype 1 keeps matrices, embeddings, K/V and the
+ *  activations that feed a matrix product in bf16 (rounded to nearest even
+ *  where produced: LayerNorm outputs, q/k/v, softmax weights before P.V,
+ *  attention output, feed-forward hidden layer, final hidden state, draft
+ *  residual block output) and accumulates in fp32; the residual stream,
+ *  softmax statistics, logits and sampling keys are fp32.
+ */
+#ifndef VADUSA_H
+#define VADUSA_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define VADUSA_ABI_VERSION 1u
+#define VADUSA_MAX_TREE_NODES 64   /* one 64-bit ancestor word per node */
+#define VADUSA_MAX_DRAFT_TOPK 16
+#define VADUSA_MAX_DEPTH 15        /* a root path has at most 16 nodes */
+
+typedef enum {
+  VADUSA_OK = 0,
+  VADUSA_EINVAL = 1,     /* bad argument or configuration */
+  VADUSA_ENOMEM = 2,     /* caller's workspace / KV pool / weight blob too small */
+  VADUSA_ECUDA = 3,      /* a CUDA runtime or driver call failed */
+  VADUSA_ECAPACITY = 4,  /* a sequence ran out of KV blocks, positions or output room */
+  VADUSA_ESTATE = 5,     /* call order (e.g. verify before a tree was set) */
+  VADUSA_ETIMEOUT = 6    /* a bounded device-side wait expired */
+} vadusa_status;
+
+typedef struct vadusa_ctx vadusa_ctx;
+
+typedef struct {
+  uint32_t struct_size;        /* sizeof(vadusa_config) */
+  uint32_t abi_version;        /* VADUSA_ABI_VERSION */
+  int32_t n_layers, d_model, n_heads, d_ffn;
+  int32_t vocab;               /* speech-token ids, the last one (vocab-1) is EOS */
+  int32_t n_phonemes;
+  int32_t max_pos;             /* rows of the position table */
+  int32_t dtype;               /* 0 fp32, 1 bf16 */
+  int32_t n_draft_heads;       /* <= VADUSA_MAX_DEPTH */
+  int32_t draft_topk;          /* candidates kept per draft head, <= VADUSA_MAX_DRAFT_TOPK */
+  int32_t max_batch;
+  int32_t max_tree_nodes;      /* <= VADUSA_MAX_TREE_NODES */
+  int32_t kv_block;            /* tokens per KV block; must be 64 */
+  int32_t max_blocks_per_seq;  /* row length of the block table */
+  int64_t kv_num_blocks;       /* blocks per layer in the pool */
+  float ln_eps;
+  int32_t device;              /* CUDA device ordinal */
+  void *kv_pool;               /* [n_layers][kv_num_blocks][2 (K,V)][n_heads][kv_block][head_dim] of dtype */
+  int64_t kv_pool_bytes;
+  void *workspace;             /* >= vadusa_workspace_bytes(cfg) bytes, 256-byte aligned */
+  int64_t workspace_bytes;
+  void *stream;                /* cudaStream_t; NULL = the legacy default stream */
+} vadusa_config;
+
+/* The weight blob: all tensors back to back in device memory, in the order and at
+ * the offsets reported by vadusa_weight_info.  Matrices are row-major
+ * [out_features][in_features] in the model dtype; the vocabulary matrices ("lm",
+ * "draft<i>.u") have their rows padded with zeros to a multiple of 128; vectors
+ * (biases, LayerNorm gains and offsets) are fp32. */
+typedef struct { const void *blob; int64_t nbytes; } vadusa_weights;
+
+typedef struct {
+  char name[32];       /* "emb_audio", "emb_phon", "pos", "l<k>.ln1_g", "l<k>.wqkv", ..., "lnf_g", "lm", "draft<i>.w" ... */
+  int64_t offset;      /* byte offset in the blob, a multiple of 256 */
+  int64_t nbytes;
+  int32_t rows, cols;  /* logical shape (cols = 1 for vectors) */
+  int32_t rows_padded; /* rows as stored */
+  int32_t is_matrix;   /* 1: stored in the model dtype; 0: fp32 vector */
+} vadusa_tensor_info;
+
+/* Sampling of the base head and the acceptance rule (Algorithm 1, Sec. II-C).
+ * At every scored node the base head "samples tau times"; a child candidate is
+ * accepted if it is one of those samples.  The tau samples are drawn without
+ * replacement from the top-p nucleus of softmax(logits / temperature) by
+ * perturbing logits/temperature with Gumbel noise and taking the tau largest
+ * keys; the first of them is the ordinary single sample.  The noise is a pure
+ * function of (seed, sequence index, absolute position of the predicted token,
+ * token id): 23 bits of a three-stage splitmix64 hash give u = (x + 1/2) / 2^23,
+ * g = -log(-log(u)) in fp32, key = logit * (1/temperature) + g in fp32.  Ties
+ * go to the lower token id.  temperature 0 means greedy: keys are the logits
+ * and top_p is ignored.  top_p >= 1 switches the nucleus off. */
+typedef struct {
+  int32_t tau;           /* tolerance, >= 1 */
+  float temperature;     /* 0 = greedy */
+  float top_p;
+  int32_t eos_masked;    /* 1: the EOS logit counts as -inf everywhere (base and draft heads) */
+  int32_t accept_rule;   /* 0: Algorithm 1 as above; 1: membership in the plain top-tau of the
+                            unperturbed logits (the root is still sampled with noise) */
+  uint64_t seed;
+} vadusa_sampling;
+
+typedef struct {
+  int64_t iterations;        /* draft-and-verify iterations run */
+  int64_t tokens_generated;  /* over all sequences */
+  double elapsed_ms;         /* device time of the loop (CUDA events) */
+  int64_t kernel_launches;   /* kernels of this library enqueued by the call */
+} vadusa_stats;
+
+/* ---- sizing and layout (host only, no GPU needed) ------------------------------ */
+int64_t vadusa_workspace_bytes(const vadusa_config *cfg);       /* < 0 on a bad configuration */
+int64_t vadusa_weights_bytes(const vadusa_config *cfg);
+int64_t vadusa_kv_pool_bytes(const vadusa_config *cfg);
+int32_t vadusa_weight_count(const vadusa_config *cfg);
+vadusa_status vadusa_weight_info(const vadusa_config *cfg, int32_t index, vadusa_tensor_info *h_out);
+
+/* ---- life cycle ------------------------------------------------------------------ */
+/* Validates the configuration, records the pointers, clears the state area of the
+ * workspace.  Synchronises the stream once. */
+vadusa_status vadusa_init(const vadusa_weights *weights, const vadusa_config *cfg, vadusa_ctx **h_out);
+vadusa_status vadusa_destroy(vadusa_ctx *ctx);
+const char *vadusa_last_error(const vadusa_ctx *ctx);   /* NUL-terminated, owned by the context */
+
+/* The static candidate tree (Sec. II-A, II-D): node 0 is the root (the base head's
+ * own next token); node n >= 1 has parent h_parent[n] < n and holds candidate
+ * number h_rank[n] (0 = best) of draft head depth(n).  Nodes must come in
+ * (depth, rank path) order so that, among equally deep nodes, a smaller index is
+ * a more-left branch.  per_sequence = 0: one template [n_nodes] for all sequences.
+ * per_sequence = 1: arrays are [batch][n_nodes], one topology per sequence
+ * (call after vadusa_begin).  Host arrays; copied. */
+vadusa_status vadusa_set_tree(vadusa_ctx *ctx, int32_t n_nodes, const int32_t *h_parent,
+                              const int32_t *h_rank, int32_t per_sequence);
+
+/* Starts a batch.  block_table: device int32 [batch][max_blocks_per_seq], the KV
+ * blocks of every sequence in logical order; it must cover every position the
+ * sequence can reach plus max_tree_nodes (tree nodes are scored in place behind the
+ * context).  h_ctx_len: host int32 [batch], tokens already present in the cache
+ * (NULL = all zero). */
+vadusa_status vadusa_begin(vadusa_ctx *ctx, int32_t batch, const int32_t *block_table,
+                           const int32_t *h_ctx_len);
+
+/* Feeds the prefix [phonemes ; prompt speech tokens] of every sequence through the
+ * model (paper Fig. 1a), in chunks, each chunk scored as a chain-shaped tree whose
+ * nodes are all accepted.  h_tokens: host int32 [batch][stride], phoneme p written
+ * as vocab + p; h_len: host int32 [batch].  Leaves the hidden state and base-head
+ * logits of the last prefix token as the start of decoding. */
+vadusa_status vadusa_prefill(vadusa_ctx *ctx, const int32_t *h_tokens, const int32_t *h_len, int32_t stride);
+
+/* Microbenchmark / test entry: sets the carried state directly.  hstar: [batch][d_model]
+ * in the model dtype; logits_star: fp32 [batch][vocab]. */
+vadusa_status vadusa_load_state(vadusa_ctx *ctx, const void *hstar, const float *logits_star);
+
+/* ---- the hot path ------------------------------------------------------------------ */
+/* Draft (Sec. II-A): root = the base head's sample for the next position, from the
+ * carried logits; every draft head's top-k at the carried hidden state; tokens
+ * scattered into the tree.  tree_tokens: int32 [batch][n_nodes] out.
+ * draft_topk_out: int32 [batch][n_draft_heads][draft_topk] out. */
+vadusa_status vadusa_draft(vadusa_ctx *ctx, const vadusa_sampling *sampling, int32_t *tree_tokens,
+                           int32_t *draft_topk_out);
+
+/* Verify (Sec. II-A "tree attention", Alg. 1 line 1): one forward pass of the base
+ * model over all tree nodes; node n sits at position ctx_len + depth(n), attends to
+ * the whole cached context and to its ancestors and itself.  Its K/V rows are
+ * written behind the context (slot ctx_len + n).  tree_tokens_override: int32
+ * [batch][n_nodes] replaces the drafted tokens (test hook; NULL = use the draft).
+ * logits_out: fp32 [batch][n_nodes][vocab]; attn_tap: [n_layers][batch][n_nodes][d_model]
+ * in the model dtype (attention output before the output projection);
+ * hidden_out: [batch][n_nodes][d_model] final-LayerNorm output in the model dtype. */
+vadusa_status vadusa_verify_step(vadusa_ctx *ctx, const int32_t *tree_tokens_override,
+                                 float *logits_out, void *attn_tap, void *hidden_out);
+
+/* Accept and commit (Alg. 1 lines 2-15, Sec. II-C): per edge, is the child token among
+ * the tau draws at its parent; a node is accepted if its whole root path is; the
+ * deepest accepted node wins, the smallest index among equally deep ones; the K/V
+ * rows of its path move to slots ctx_len .. ctx_len + accept_len - 1, its hidden state
+ * and logits become the carried state, ctx_len grows by accept_len.
+ * forced_best_node: int32 [batch] overrides the winner (test hook; -1 entries keep the rule).
+ * accept_len int32 [batch]; path_nodes, path_tokens int32 [batch][VADUSA_MAX_DEPTH+1]
+ * (entries beyond accept_len are -1); kv_slots int64 [batch][VADUSA_MAX_DEPTH+1]:
+ * block * kv_block + offset of every committed token; edge_bits uint64 [batch]: bit n set
+ * iff edge parent(n)->n was tested and accepted (bit 0 always set); next_root int32 [batch]:
+ * the base head's sample for the position after the winner. */
+vadusa_status vadusa_accept_and_commit(vadusa_ctx *ctx, const vadusa_sampling *sampling,
+                                       const int32_t *forced_best_node, int32_t *accept_len,
+                                       int32_t *path_nodes, int32_t *path_tokens, int64_t *kv_slots,
+                                       uint64_t *edge_bits, int32_t *next_root);
+
+/* Runs draft -> verify -> accept+commit until every sequence has max_new_tokens tokens
+ * (or max_iters iterations, if > 0).  out_tokens: int32 [batch][max_new_tokens]
+ * (a sequence's surplus tokens of its last iteration are dropped); out_len: int32
+ * [batch].  Synchronises; returns device-side errors.  h_stats may be NULL. */
+vadusa_status vadusa_generate(vadusa_ctx *ctx, const vadusa_sampling *sampling, int32_t max_new_tokens,
+                              int32_t max_iters, int32_t *out_tokens, int32_t *out_len,
+                              vadusa_stats *h_stats);
+
+/* The same from host memory to host memory (what an application calls): begin,
+ * prefill from h_tokens, generate, copy the tokens back.  block_table is a device
+ * pointer as in vadusa_begin; all other buffers are host memory.  Synchronises. */
+vadusa_status vadusa_generate_host(vadusa_ctx *ctx, const vadusa_sampling *sampling, int32_t batch,
+                                   const int32_t *block_table, const int32_t *h_tokens,
+                                   const int32_t *h_len, int32_t stride, int32_t max_new_tokens,
+                                   int32_t *h_out_tokens, int32_t *h_out_len, vadusa_stats *h_stats);
+
+/* ---- state ---------------------------------------------------------------------- */
+vadusa_status vadusa_get_lengths(vadusa_ctx *ctx, int32_t *h_ctx_len);  /* synchronises */
+vadusa_status vadusa_check(vadusa_ctx *ctx);                            /* synchronises; device error word */
+int64_t vadusa_kernel_launches(const vadusa_ctx *ctx);                  /* total kernels enqueued so far */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VADUSA_H */
