@@ -1,0 +1,737 @@
+// libvadusa: host engine and C ABI.  Every step of the draft-and-verify path runs in
+// the kernels included below; this file only validates, lays out memory and launches.
+#include <cuda_runtime.h>
+#include <stdarg.h>
+
+#include <new>
+
+#include "accept.cuh"
+#include "attention_simt.cuh"
+#include "elementwise.cuh"
+#include "gemm_simt.cuh"
+#include "layout.h"
+#include "select.cuh"
+
+using namespace vadusa;
+
+struct LayerW {
+  const float *ln1_g, *ln1_b, *bqkv, *bo, *ln2_g, *ln2_b, *b1, *b2;
+  const void *wqkv, *wo, *w1, *w2;
+};
+
+struct vadusa_ctx {
+  vadusa_config cfg;
+  std::vector<LayerW> layers;
+  const void *emb_audio = nullptr, *emb_phon = nullptr, *pos = nullptr, *lm = nullptr, *dw = nullptr, *du = nullptr;
+  const float *lnf_g = nullptr, *lnf_b = nullptr, *db = nullptr;
+  long long dw_stride = 0, du_stride = 0;     // bytes between draft heads
+  WorkspaceLayout ws;
+  std::vector<TensorDesc> wl;
+  const char* blob = nullptr;
+  char* wsp = nullptr;
+  cudaStream_t stream = nullptr;
+  int batch = 0;
+  int n_nodes = 0;            // current tree size (0: none set)
+  int tree_per_seq = 0;
+  int max_rank_used = 0;
+  const int32_t* block_table = nullptr;
+  bool have_draft = false, have_verify = false;
+  int64_t launches = 0;
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr, ev_poll = nullptr;
+  int32_t* h_pinned = nullptr;     // [2]: done_count, err
+  char err[512] = {0};
+};
+
+namespace {
+
+vadusa_status fail(vadusa_ctx* c, vadusa_status s, const char* fmt, ...) {
+  if (c) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(c->err, sizeof(c->err), fmt, ap);
+    va_end(ap);
+  }
+  return s;
+}
+
+#define CU(call)                                                                                   \
+  do {                                                                                             \
+    cudaError_t e_ = (call);                                                                       \
+    if (e_ != cudaSuccess) return fail(ctx, VADUSA_ECUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
+  } while (0)
+
+#define LAUNCH_CHECK()                                                                             \
+  do {                                                                                             \
+    cudaError_t e_ = cudaGetLastError();                                                           \
+    if (e_ != cudaSuccess) return fail(ctx, VADUSA_ECUDA, "kernel launch: %s", cudaGetErrorString(e_)); \
+    ctx->launches++;                                                                               \
+  } while (0)
+
+template <typename P> P* wsptr(vadusa_ctx* c, int64_t off) { return reinterpret_cast<P*>(c->wsp + off); }
+
+const TensorDesc* find(const vadusa_ctx* c, const std::string& name) {
+  for (const auto& t : c->wl)
+    if (t.name == name) return &t;
+  return nullptr;
+}
+const void* wraw(const vadusa_ctx* c, const std::string& name) {
+  const TensorDesc* t = find(c, name);
+  return t ? c->blob + t->offset : nullptr;
+}
+
+void resolve_weights(vadusa_ctx* c) {
+  auto f = [&](const std::string& n) { return reinterpret_cast<const float*>(wraw(c, n)); };
+  c->layers.resize(c->cfg.n_layers);
+  for (int l = 0; l < c->cfg.n_layers; ++l) {
+    const std::string p = "l" + std::to_string(l) + ".";
+    LayerW& w = c->layers[l];
+    w.ln1_g = f(p + "ln1_g"); w.ln1_b = f(p + "ln1_b"); w.bqkv = f(p + "bqkv"); w.bo = f(p + "bo");
+    w.ln2_g = f(p + "ln2_g"); w.ln2_b = f(p + "ln2_b"); w.b1 = f(p + "b1"); w.b2 = f(p + "b2");
+    w.wqkv = wraw(c, p + "wqkv"); w.wo = wraw(c, p + "wo"); w.w1 = wraw(c, p + "w1"); w.w2 = wraw(c, p + "w2");
+  }
+  c->emb_audio = wraw(c, "emb_audio"); c->emb_phon = wraw(c, "emb_phon"); c->pos = wraw(c, "pos");
+  c->lnf_g = f("lnf_g"); c->lnf_b = f("lnf_b"); c->lm = wraw(c, "lm");
+  c->dw = wraw(c, "draft0.w"); c->db = f("draft0.b"); c->du = wraw(c, "draft0.u");
+  if (c->cfg.n_draft_heads > 1) {
+    c->dw_stride = find(c, "draft1.w")->offset - find(c, "draft0.w")->offset;
+    c->du_stride = find(c, "draft1.u")->offset - find(c, "draft0.u")->offset;
+  }
+}
+template <typename T> const T* as(const void* p) { return reinterpret_cast<const T*>(p); }
+
+uint32_t* err_word(vadusa_ctx* c) { return wsptr<uint32_t>(c, c->ws.scalars); }
+int32_t* done_word(vadusa_ctx* c) { return wsptr<int32_t>(c, c->ws.scalars) + 1; }
+
+KvGeom geom_of(const vadusa_ctx* c) {
+  KvGeom g;
+  g.n_heads = c->cfg.n_heads;
+  g.head_dim = c->cfg.d_model / c->cfg.n_heads;
+  g.max_blocks_per_seq = c->cfg.max_blocks_per_seq;
+  g.num_blocks = c->cfg.kv_num_blocks;
+  g.layer_stride = (long long)c->cfg.kv_num_blocks * 2 * c->cfg.d_model * kKvBlock;
+  return g;
+}
+
+TreeView tree_of(vadusa_ctx* c, bool chain) {
+  TreeView t;
+  if (chain) {
+    t.parent = wsptr<int32_t>(c, c->ws.chain_parent);
+    t.depth = wsptr<int32_t>(c, c->ws.chain_depth);
+    t.rank = wsptr<int32_t>(c, c->ws.chain_rank);
+    t.anc = wsptr<unsigned long long>(c, c->ws.chain_anc);
+    t.n_nodes = c->cfg.max_tree_nodes;
+    t.per_seq = 0;
+  } else {
+    t.parent = wsptr<int32_t>(c, c->ws.tree_parent);
+    t.depth = wsptr<int32_t>(c, c->ws.tree_depth);
+    t.rank = wsptr<int32_t>(c, c->ws.tree_rank);
+    t.anc = wsptr<unsigned long long>(c, c->ws.tree_anc);
+    t.n_nodes = c->n_nodes;
+    t.per_seq = c->tree_per_seq;
+  }
+  return t;
+}
+
+SeqState state_of(vadusa_ctx* c, int32_t* out_tokens, int out_cap, int target) {
+  SeqState s;
+  s.ctx_len = wsptr<int32_t>(c, c->ws.ctx_len);
+  s.nvalid = wsptr<int32_t>(c, c->ws.nvalid);
+  s.gen_count = wsptr<int32_t>(c, c->ws.gen_count);
+  s.commit_base = wsptr<int32_t>(c, c->ws.commit_base);
+  s.commit_len = wsptr<int32_t>(c, c->ws.commit_len);
+  s.commit_path = wsptr<int32_t>(c, c->ws.commit_path);
+  s.best = wsptr<int32_t>(c, c->ws.best);
+  s.out_tokens = out_tokens;
+  s.done_count = done_word(c);
+  s.out_cap = out_cap;
+  s.target = target;
+  return s;
+}
+
+vadusa_status sampling_dev(vadusa_ctx* ctx, const vadusa_sampling* s, SamplingDev* o) {
+  if (!s) return fail(ctx, VADUSA_EINVAL, "sampling is NULL");
+  if (s->tau < 1) return fail(ctx, VADUSA_EINVAL, "tau must be >= 1");
+  if (!(s->temperature >= 0.f)) return fail(ctx, VADUSA_EINVAL, "temperature must be >= 0");
+  if (!(s->top_p > 0.f)) return fail(ctx, VADUSA_EINVAL, "top_p must be > 0");
+  if (s->accept_rule != 0 && s->accept_rule != 1) return fail(ctx, VADUSA_EINVAL, "accept_rule must be 0 or 1");
+  o->tau = s->tau;
+  o->temperature = s->temperature;
+  o->inv_temperature = s->temperature > 0.f ? (float)(1.0 / (double)s->temperature) : 1.f;
+  o->top_p = s->top_p;
+  o->eos_masked = s->eos_masked ? 1 : 0;
+  o->accept_rule = s->accept_rule;
+  o->eos_id = ctx->cfg.vocab - 1;
+  o->seed = s->seed;
+  return VADUSA_OK;
+}
+
+// ---- typed engine ------------------------------------------------------------------
+
+template <typename T, typename Epi>
+vadusa_status gemm(vadusa_ctx* ctx, const T* A, const T* W, int M, int N, int K, int batches, long long a_z,
+                   long long w_z, const Epi& epi) {
+  dim3 grid((N + 63) / 64, (M + 63) / 64, batches);
+  gemm_simt_kernel<T, Epi><<<grid, 256, 0, ctx->stream>>>(A, W, M, N, K, a_z, w_z, epi);
+  LAUNCH_CHECK();
+  return VADUSA_OK;
+}
+
+template <typename T>
+vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeView& tv, T* out) {
+  const vadusa_config& c = ctx->cfg;
+  const int dh = c.d_model / c.n_heads;
+  const KvGeom g = geom_of(ctx);
+  const float scale = (float)(1.0 / sqrt((double)dh));
+  dim3 grid(c.n_heads, ctx->batch);
+  const size_t smem = (size_t)(64 * dh * 3 + 64 + 64 * 64) * sizeof(float);   // = attention_smem(dh)
+  auto go = [&](auto kern) -> vadusa_status {
+    kern<<<grid, 256, smem, ctx->stream>>>(q, pool, ctx->block_table, wsptr<int32_t>(ctx, ctx->ws.ctx_len),
+                                           wsptr<int32_t>(ctx, ctx->ws.nvalid), tv, g, c.d_model, scale, out,
+                                           err_word(ctx));
+    LAUNCH_CHECK();
+    return VADUSA_OK;
+  };
+  if (dh == 64) return go(tree_attention_simt_kernel<T, 64>);
+  return go(tree_attention_simt_kernel<T, 32>);
+}
+
+// One forward pass of the base model over batch * tv.n_nodes rows (verify step).
+template <typename T>
+vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* override_tokens, T* attn_tap) {
+  const vadusa_config& c = ctx->cfg;
+  const int B = ctx->batch, N = tv.n_nodes, M = B * N, d = c.d_model, f = c.d_ffn, vp = vpad(&c);
+  const KvGeom g = geom_of(ctx);
+  float* x = wsptr<float>(ctx, ctx->ws.x);
+  T* a = wsptr<T>(ctx, ctx->ws.a);
+  T* q = wsptr<T>(ctx, ctx->ws.q);
+  T* o = wsptr<T>(ctx, ctx->ws.o);
+  T* mid = wsptr<T>(ctx, ctx->ws.mid);
+  T* hfinal = wsptr<T>(ctx, ctx->ws.hfinal);
+  float* logits = wsptr<float>(ctx, ctx->ws.logits);
+  int32_t* ctx_len = wsptr<int32_t>(ctx, ctx->ws.ctx_len);
+  int32_t* nvalid = wsptr<int32_t>(ctx, ctx->ws.nvalid);
+  const int ln_blocks = (M + 3) / 4;
+
+  tree_embed_kernel<T><<<M, 128, 0, ctx->stream>>>(
+      tv, override_tokens, wsptr<int32_t>(ctx, ctx->ws.root), wsptr<int32_t>(ctx, ctx->ws.topk), c.n_draft_heads,
+      c.draft_topk, ctx_len, nvalid, as<T>(ctx->emb_audio), as<T>(ctx->emb_phon), as<T>(ctx->pos),
+      c.vocab, c.n_phonemes, c.max_pos, d, wsptr<int32_t>(ctx, ctx->ws.tokens), x, err_word(ctx));
+  LAUNCH_CHECK();
+  for (int l = 0; l < c.n_layers; ++l) {
+    const LayerW& w = ctx->layers[l];
+    T* pool = reinterpret_cast<T*>(c.kv_pool) + (long long)l * g.layer_stride;
+    layernorm_kernel<T><<<ln_blocks, 128, 0, ctx->stream>>>(x, w.ln1_g, w.ln1_b, a, M, d, c.ln_eps);
+    LAUNCH_CHECK();
+    EpiQKV<T> eq{w.bqkv, q, pool, ctx->block_table, ctx_len, nvalid, err_word(ctx), g, N, d};
+    vadusa_status s = gemm<T>(ctx, a, as<T>(w.wqkv), M, 3 * d, d, 1, 0, 0, eq);
+    if (s) return s;
+    T* o_dst = attn_tap ? attn_tap + (long long)l * M * d : o;
+    s = attention<T>(ctx, q, pool, tv, o_dst);
+    if (s) return s;
+    EpiResidual eo{w.bo, x, d};
+    s = gemm<T>(ctx, o_dst, as<T>(w.wo), M, d, d, 1, 0, 0, eo);
+    if (s) return s;
+    layernorm_kernel<T><<<ln_blocks, 128, 0, ctx->stream>>>(x, w.ln2_g, w.ln2_b, a, M, d, c.ln_eps);
+    LAUNCH_CHECK();
+    EpiRelu<T> e1{w.b1, mid, f};
+    s = gemm<T>(ctx, a, as<T>(w.w1), M, f, d, 1, 0, 0, e1);
+    if (s) return s;
+    EpiResidual e2{w.b2, x, d};
+    s = gemm<T>(ctx, mid, as<T>(w.w2), M, d, f, 1, 0, 0, e2);
+    if (s) return s;
+  }
+  layernorm_kernel<T><<<ln_blocks, 128, 0, ctx->stream>>>(x, ctx->lnf_g, ctx->lnf_b,
+                                                          hfinal, M, d, c.ln_eps);
+  LAUNCH_CHECK();
+  EpiLogits el{logits, vp, 0};
+  return gemm<T>(ctx, hfinal, as<T>(ctx->lm), M, vp, d, 1, 0, 0, el);
+}
+
+template <typename T>
+vadusa_status draft(vadusa_ctx* ctx, const SamplingDev& sp) {
+  const vadusa_config& c = ctx->cfg;
+  const int B = ctx->batch, d = c.d_model, vp = vpad(&c), hd = c.n_draft_heads;
+  const T* hstar = wsptr<T>(ctx, ctx->ws.hstar);
+  T* z = wsptr<T>(ctx, ctx->ws.z);
+  float* dl = wsptr<float>(ctx, ctx->ws.dlogits);
+  const long long w_stride = ctx->dw_stride / (long long)sizeof(T), u_stride = ctx->du_stride / (long long)sizeof(T);
+  EpiDraftHidden<T> eh{ctx->db, hstar, z, d, B};
+  vadusa_status s = gemm<T>(ctx, hstar, as<T>(ctx->dw), B, d, d, hd, 0, w_stride, eh);
+  if (s) return s;
+  EpiLogits el{dl, vp, (long long)B * vp};
+  s = gemm<T>(ctx, z, as<T>(ctx->du), B, vp, d, hd, (long long)B * d, u_stride, el);
+  if (s) return s;
+  dim3 grid(hd + 1, B);
+  draft_select_kernel<<<grid, 256, 0, ctx->stream>>>(dl, wsptr<float>(ctx, ctx->ws.logits_star), vp, c.vocab, B, hd,
+                                                     c.draft_topk, wsptr<int32_t>(ctx, ctx->ws.ctx_len),
+                                                     wsptr<int32_t>(ctx, ctx->ws.nvalid), sp,
+                                                     wsptr<int32_t>(ctx, ctx->ws.topk),
+                                                     wsptr<int32_t>(ctx, ctx->ws.root));
+  LAUNCH_CHECK();
+  return VADUSA_OK;
+}
+
+// tokens = tree built from the draft (no model pass): used when the caller wants them.
+template <typename T>
+vadusa_status accept_commit(vadusa_ctx* ctx, const SamplingDev& sp, const int32_t* forced, const AcceptOut& out,
+                            int32_t* out_tokens, int out_cap, int target) {
+  const vadusa_config& c = ctx->cfg;
+  const int B = ctx->batch, vp = vpad(&c);
+  const KvGeom g = geom_of(ctx);
+  const TreeView tv = tree_of(ctx, false);
+  SeqState st = state_of(ctx, out_tokens, out_cap, target);
+  accept_kernel<<<B, 256, vp * sizeof(float), ctx->stream>>>(
+      wsptr<float>(ctx, ctx->ws.logits), vp, c.vocab, wsptr<int32_t>(ctx, ctx->ws.tokens), tv, ctx->block_table, g,
+      sp, forced, st, out, err_word(ctx));
+  LAUNCH_CHECK();
+  dim3 grid(c.n_layers + 1, B);
+  commit_kernel<T><<<grid, 256, 0, ctx->stream>>>(
+      reinterpret_cast<T*>(c.kv_pool), g, ctx->block_table, st, c.n_layers, tv.n_nodes,
+      wsptr<T>(ctx, ctx->ws.hfinal), c.d_model, wsptr<float>(ctx, ctx->ws.logits), vp, wsptr<T>(ctx, ctx->ws.hstar),
+      wsptr<float>(ctx, ctx->ws.logits_star), err_word(ctx));
+  LAUNCH_CHECK();
+  return VADUSA_OK;
+}
+
+template <typename T>
+vadusa_status prefill(vadusa_ctx* ctx, const int32_t* h_tokens, const int32_t* h_len, int stride) {
+  const vadusa_config& c = ctx->cfg;
+  const int B = ctx->batch, N = c.max_tree_nodes, vp = vpad(&c);
+  int longest = 0;
+  for (int b = 0; b < B; ++b) {
+    if (h_len[b] < 1 || h_len[b] > stride) return fail(ctx, VADUSA_EINVAL, "prefix length of sequence %d out of range", b);
+    longest = h_len[b] > longest ? h_len[b] : longest;
+  }
+  int32_t* d_nvalid = wsptr<int32_t>(ctx, ctx->ws.nvalid);
+  int32_t* d_stage = wsptr<int32_t>(ctx, ctx->ws.stage_tokens);
+  std::vector<int32_t> stage((size_t)B * N), nv(B);
+  const TreeView tv = tree_of(ctx, true);
+  SeqState st = state_of(ctx, nullptr, 0, 0);
+  for (int s0 = 0; s0 < longest; s0 += N) {
+    for (int b = 0; b < B; ++b) {
+      int n = h_len[b] - s0;
+      n = n < 0 ? 0 : (n > N ? N : n);
+      nv[b] = n;
+      for (int i = 0; i < N; ++i) stage[(size_t)b * N + i] = i < n ? h_tokens[(size_t)b * stride + s0 + i] : 0;
+    }
+    CU(cudaMemcpyAsync(d_nvalid, nv.data(), B * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaMemcpyAsync(d_stage, stage.data(), (size_t)B * N * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));   // the staging vectors are reused by the next chunk
+    vadusa_status s = forward<T>(ctx, tv, d_stage, nullptr);
+    if (s) return s;
+    prefill_advance_kernel<T><<<B, 256, 0, ctx->stream>>>(st, N, wsptr<T>(ctx, ctx->ws.hfinal), c.d_model,
+                                                          wsptr<float>(ctx, ctx->ws.logits), vp,
+                                                          wsptr<T>(ctx, ctx->ws.hstar),
+                                                          wsptr<float>(ctx, ctx->ws.logits_star));
+    LAUNCH_CHECK();
+  }
+  return VADUSA_OK;
+}
+
+size_t attention_smem(int dh) { return (size_t)(64 * dh * 3 + 64 + 64 * 64) * sizeof(float); }
+
+vadusa_status set_kernel_attributes(vadusa_ctx* ctx) {
+  CU(cudaFuncSetAttribute(tree_attention_simt_kernel<float, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(64)));
+  CU(cudaFuncSetAttribute(tree_attention_simt_kernel<float, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(32)));
+  CU(cudaFuncSetAttribute(tree_attention_simt_kernel<bf16, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(64)));
+  CU(cudaFuncSetAttribute(tree_attention_simt_kernel<bf16, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(32)));
+  return VADUSA_OK;
+}
+
+__global__ void fill_i32_kernel(int32_t* p, int n, int32_t v) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) p[i] = v;
+}
+
+vadusa_status set_active(vadusa_ctx* ctx, int value) {
+  fill_i32_kernel<<<(ctx->batch + 255) / 256, 256, 0, ctx->stream>>>(wsptr<int32_t>(ctx, ctx->ws.nvalid), ctx->batch,
+                                                                     value);
+  LAUNCH_CHECK();
+  return VADUSA_OK;
+}
+
+vadusa_status device_errors(vadusa_ctx* ctx) {
+  uint32_t e = 0;
+  CU(cudaMemcpyAsync(&e, err_word(ctx), sizeof(e), cudaMemcpyDeviceToHost, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  if (e & kErrTimeout) return fail(ctx, VADUSA_ETIMEOUT, "a bounded device-side wait expired (error word 0x%x)", e);
+  if (e & kErrCapacity)
+    return fail(ctx, VADUSA_ECAPACITY, "a sequence ran past its KV blocks, the position table or the token range (error word 0x%x)", e);
+  return VADUSA_OK;
+}
+
+#define DISPATCH(expr_f32, expr_bf16) (ctx->cfg.dtype == 1 ? (expr_bf16) : (expr_f32))
+
+vadusa_status need_batch(vadusa_ctx* ctx) {
+  if (!ctx) return VADUSA_EINVAL;
+  if (ctx->batch == 0) return fail(ctx, VADUSA_ESTATE, "vadusa_begin has not been called");
+  return VADUSA_OK;
+}
+
+}  // namespace
+
+// ---- C ABI -------------------------------------------------------------------------
+
+extern "C" {
+
+int64_t vadusa_workspace_bytes(const vadusa_config* cfg) {
+  if (check_config(cfg)) return -1;
+  return workspace_layout(cfg).total;
+}
+
+int64_t vadusa_weights_bytes(const vadusa_config* cfg) {
+  if (check_config(cfg)) return -1;
+  int64_t total = 0;
+  weight_layout(cfg, &total);
+  return total;
+}
+
+int64_t vadusa_kv_pool_bytes(const vadusa_config* cfg) {
+  if (check_config(cfg)) return -1;
+  return kv_pool_bytes(cfg);
+}
+
+int32_t vadusa_weight_count(const vadusa_config* cfg) {
+  if (check_config(cfg)) return -1;
+  return (int32_t)weight_layout(cfg, nullptr).size();
+}
+
+vadusa_status vadusa_weight_info(const vadusa_config* cfg, int32_t index, vadusa_tensor_info* h_out) {
+  if (check_config(cfg) || !h_out) return VADUSA_EINVAL;
+  auto v = weight_layout(cfg, nullptr);
+  if (index < 0 || index >= (int32_t)v.size()) return VADUSA_EINVAL;
+  const TensorDesc& t = v[index];
+  memset(h_out, 0, sizeof(*h_out));
+  snprintf(h_out->name, sizeof(h_out->name), "%s", t.name.c_str());
+  h_out->offset = t.offset; h_out->nbytes = t.nbytes;
+  h_out->rows = t.rows; h_out->cols = t.cols; h_out->rows_padded = t.rows_padded; h_out->is_matrix = t.is_matrix;
+  return VADUSA_OK;
+}
+
+vadusa_status vadusa_init(const vadusa_weights* weights, const vadusa_config* cfg, vadusa_ctx** h_out) {
+  if (!h_out) return VADUSA_EINVAL;
+  *h_out = nullptr;
+  vadusa_ctx* ctx = new (std::nothrow) vadusa_ctx();
+  if (!ctx) return VADUSA_ENOMEM;
+  *h_out = ctx;     // returned even on failure so that vadusa_last_error can be read; destroy it either way
+  if (const char* why = check_config(cfg)) return fail(ctx, VADUSA_EINVAL, "%s", why);
+  ctx->cfg = *cfg;
+  if (!weights || !weights->blob) return fail(ctx, VADUSA_EINVAL, "weights are NULL");
+  int64_t wbytes = 0;
+  ctx->wl = weight_layout(cfg, &wbytes);
+  if (weights->nbytes < wbytes) return fail(ctx, VADUSA_ENOMEM, "weight blob has %lld bytes, %lld needed", (long long)weights->nbytes, (long long)wbytes);
+  ctx->ws = workspace_layout(cfg);
+  if (!cfg->workspace || cfg->workspace_bytes < ctx->ws.total)
+    return fail(ctx, VADUSA_ENOMEM, "workspace has %lld bytes, %lld needed", (long long)cfg->workspace_bytes, (long long)ctx->ws.total);
+  if (((uintptr_t)cfg->workspace & 255) || ((uintptr_t)weights->blob & 255) || ((uintptr_t)cfg->kv_pool & 255))
+    return fail(ctx, VADUSA_EINVAL, "workspace, weight blob and KV pool must be 256-byte aligned");
+  if (!cfg->kv_pool || cfg->kv_pool_bytes < kv_pool_bytes(cfg))
+    return fail(ctx, VADUSA_ENOMEM, "KV pool has %lld bytes, %lld needed", (long long)cfg->kv_pool_bytes, (long long)kv_pool_bytes(cfg));
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
+    cudaGetLastError();
+    return fail(ctx, VADUSA_ECUDA, "no CUDA device: this library has no CPU path");
+  }
+  if (cfg->device < 0 || cfg->device >= ndev) return fail(ctx, VADUSA_EINVAL, "device ordinal out of range");
+  CU(cudaSetDevice(cfg->device));
+  cudaDeviceProp prop;
+  CU(cudaGetDeviceProperties(&prop, cfg->device));
+  if (prop.major != 10) return fail(ctx, VADUSA_ECUDA, "device is sm_%d%d; this library is built for sm_100a only", prop.major, prop.minor);
+  ctx->blob = reinterpret_cast<const char*>(weights->blob);
+  ctx->wsp = reinterpret_cast<char*>(cfg->workspace);
+  ctx->stream = reinterpret_cast<cudaStream_t>(cfg->stream);
+  resolve_weights(ctx);
+  if (vadusa_status s = set_kernel_attributes(ctx)) return s;
+  CU(cudaEventCreate(&ctx->ev0));
+  CU(cudaEventCreate(&ctx->ev1));
+  CU(cudaEventCreateWithFlags(&ctx->ev_poll, cudaEventDisableTiming));
+  CU(cudaMallocHost(&ctx->h_pinned, 4 * sizeof(int32_t)));
+  CU(cudaMemsetAsync(ctx->wsp, 0, ctx->ws.tokens, ctx->stream));     // scalars, per-sequence state, trees
+  // chain-shaped tree used by prefill: node i is the child of node i-1
+  int32_t par[64], dep[64], rnk[64];
+  unsigned long long anc[64];
+  for (int i = 0; i < 64; ++i) { par[i] = i - 1; dep[i] = i; rnk[i] = 0; anc[i] = i == 63 ? ~0ull : ((1ull << (i + 1)) - 1); }
+  CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.chain_parent, par, sizeof(par), cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.chain_depth, dep, sizeof(dep), cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.chain_rank, rnk, sizeof(rnk), cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.chain_anc, anc, sizeof(anc), cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  return VADUSA_OK;
+}
+
+vadusa_status vadusa_destroy(vadusa_ctx* ctx) {
+  if (!ctx) return VADUSA_EINVAL;
+  if (ctx->ev0) cudaEventDestroy(ctx->ev0);
+  if (ctx->ev1) cudaEventDestroy(ctx->ev1);
+  if (ctx->ev_poll) cudaEventDestroy(ctx->ev_poll);
+  if (ctx->h_pinned) cudaFreeHost(ctx->h_pinned);
+  delete ctx;
+  return VADUSA_OK;
+}
+
+const char* vadusa_last_error(const vadusa_ctx* ctx) { return ctx ? ctx->err : "context is NULL"; }
+
+vadusa_status vadusa_set_tree(vadusa_ctx* ctx, int32_t n_nodes, const int32_t* h_parent, const int32_t* h_rank,
+                              int32_t per_sequence) {
+  if (!ctx) return VADUSA_EINVAL;
+  if (!ctx->wsp) return fail(ctx, VADUSA_ESTATE, "context is not initialised");
+  if (!h_parent || !h_rank) return fail(ctx, VADUSA_EINVAL, "tree arrays are NULL");
+  if (n_nodes < 1 || n_nodes > ctx->cfg.max_tree_nodes) return fail(ctx, VADUSA_EINVAL, "n_nodes must be in 1..max_tree_nodes");
+  int copies = 1;
+  if (per_sequence) {
+    if (ctx->batch == 0) return fail(ctx, VADUSA_ESTATE, "per-sequence trees need vadusa_begin first");
+    copies = ctx->batch;
+  }
+  std::vector<int32_t> depth((size_t)copies * n_nodes);
+  std::vector<unsigned long long> anc((size_t)copies * n_nodes);
+  int max_rank = 0;
+  for (int s = 0; s < copies; ++s) {
+    const int32_t* par = h_parent + (size_t)s * n_nodes;
+    const int32_t* rnk = h_rank + (size_t)s * n_nodes;
+    int32_t* dep = depth.data() + (size_t)s * n_nodes;
+    unsigned long long* an = anc.data() + (size_t)s * n_nodes;
+    if (par[0] != -1) return fail(ctx, VADUSA_EINVAL, "node 0 must be the root (parent -1)");
+    dep[0] = 0; an[0] = 1ull;
+    for (int n = 1; n < n_nodes; ++n) {
+      if (par[n] < 0 || par[n] >= n) return fail(ctx, VADUSA_EINVAL, "node %d: parent %d must precede it", n, par[n]);
+      dep[n] = dep[par[n]] + 1;
+      an[n] = an[par[n]] | (1ull << n);
+      if (dep[n] > VADUSA_MAX_DEPTH) return fail(ctx, VADUSA_EINVAL, "node %d: deeper than %d", n, VADUSA_MAX_DEPTH);
+      if (!per_sequence) {
+        if (dep[n] > ctx->cfg.n_draft_heads) return fail(ctx, VADUSA_EINVAL, "node %d: depth %d exceeds the number of draft heads", n, dep[n]);
+        if (rnk[n] < 0 || rnk[n] >= ctx->cfg.draft_topk) return fail(ctx, VADUSA_EINVAL, "node %d: rank %d outside the draft top-k", n, rnk[n]);
+      } else if (rnk[n] < 0) {
+        return fail(ctx, VADUSA_EINVAL, "node %d: negative rank", n);
+      }
+      if (dep[n] < dep[n - 1]) return fail(ctx, VADUSA_EINVAL, "node %d: nodes must be ordered by depth", n);
+      // (depth, rank path) order: within a depth, parents ascend, and siblings ascend by rank
+      if (n > 1 && dep[n] == dep[n - 1]) {
+        if (par[n] < par[n - 1] || (par[n] == par[n - 1] && rnk[n] <= rnk[n - 1]))
+          return fail(ctx, VADUSA_EINVAL, "node %d: nodes of one depth must be in rank-path order", n);
+      }
+      max_rank = rnk[n] > max_rank ? rnk[n] : max_rank;
+    }
+  }
+  const size_t n4 = (size_t)copies * n_nodes * sizeof(int32_t);
+  CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.tree_parent, h_parent, n4, cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.tree_rank, h_rank, n4, cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.tree_depth, depth.data(), n4, cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.tree_anc, anc.data(), (size_t)copies * n_nodes * 8, cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  ctx->n_nodes = n_nodes;
+  ctx->tree_per_seq = per_sequence ? 1 : 0;
+  ctx->max_rank_used = max_rank;
+  ctx->have_draft = ctx->have_verify = false;
+  if (ctx->batch > 0) return set_active(ctx, ctx->n_nodes);
+  return VADUSA_OK;
+}
+
+vadusa_status vadusa_begin(vadusa_ctx* ctx, int32_t batch, const int32_t* block_table, const int32_t* h_ctx_len) {
+  if (!ctx) return VADUSA_EINVAL;
+  if (!ctx->wsp) return fail(ctx, VADUSA_ESTATE, "context is not initialised");
+  if (batch < 1 || batch > ctx->cfg.max_batch) return fail(ctx, VADUSA_EINVAL, "batch must be in 1..max_batch");
+  if (!block_table) return fail(ctx, VADUSA_EINVAL, "block_table is NULL");
+  if (ctx->tree_per_seq) { ctx->n_nodes = 0; ctx->tree_per_seq = 0; }
+  ctx->batch = batch;
+  ctx->block_table = block_table;
+  ctx->have_draft = ctx->have_verify = false;
+  CU(cudaMemsetAsync(ctx->wsp + ctx->ws.scalars, 0, 256, ctx->stream));
+  CU(cudaMemsetAsync(ctx->wsp + ctx->ws.gen_count, 0, batch * 4, ctx->stream));
+  if (h_ctx_len) {
+    for (int b = 0; b < batch; ++b)
+      if (h_ctx_len[b] < 0 || h_ctx_len[b] > (int64_t)ctx->cfg.max_blocks_per_seq * 64)
+        return fail(ctx, VADUSA_EINVAL, "context length of sequence %d out of range", b);
+    CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.ctx_len, h_ctx_len, batch * 4, cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+  } else {
+    CU(cudaMemsetAsync(ctx->wsp + ctx->ws.ctx_len, 0, batch * 4, ctx->stream));
+  }
+  return set_active(ctx, ctx->n_nodes);
+}
+
+vadusa_status vadusa_prefill(vadusa_ctx* ctx, const int32_t* h_tokens, const int32_t* h_len, int32_t stride) {
+  if (vadusa_status s = need_batch(ctx)) return s;
+  if (!h_tokens || !h_len || stride < 1) return fail(ctx, VADUSA_EINVAL, "prefill arguments are NULL or empty");
+  vadusa_status s = DISPATCH(prefill<float>(ctx, h_tokens, h_len, stride), prefill<bf16>(ctx, h_tokens, h_len, stride));
+  if (s) return s;
+  ctx->have_draft = ctx->have_verify = false;
+  return set_active(ctx, ctx->n_nodes);
+}
+
+vadusa_status vadusa_load_state(vadusa_ctx* ctx, const void* hstar, const float* logits_star) {
+  if (vadusa_status s = need_batch(ctx)) return s;
+  if (!hstar || !logits_star) return fail(ctx, VADUSA_EINVAL, "state pointers are NULL");
+  const vadusa_config& c = ctx->cfg;
+  CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.hstar, hstar, (size_t)ctx->batch * c.d_model * esize(&c), cudaMemcpyDeviceToDevice, ctx->stream));
+  CU(cudaMemcpy2DAsync(ctx->wsp + ctx->ws.logits_star, (size_t)vpad(&c) * 4, logits_star, (size_t)c.vocab * 4,
+                       (size_t)c.vocab * 4, ctx->batch, cudaMemcpyDeviceToDevice, ctx->stream));
+  return VADUSA_OK;
+}
+
+vadusa_status vadusa_draft(vadusa_ctx* ctx, const vadusa_sampling* sampling, int32_t* tree_tokens,
+                           int32_t* draft_topk_out) {
+  if (vadusa_status s = need_batch(ctx)) return s;
+  if (ctx->n_nodes == 0) return fail(ctx, VADUSA_ESTATE, "no tree set");
+  if (ctx->tree_per_seq && tree_tokens) return fail(ctx, VADUSA_EINVAL, "per-sequence topologies take their tokens from the override");
+  SamplingDev sp;
+  if (vadusa_status s = sampling_dev(ctx, sampling, &sp)) return s;
+  vadusa_status s = DISPATCH(draft<float>(ctx, sp), draft<bf16>(ctx, sp));
+  if (s) return s;
+  ctx->have_draft = true;
+  const vadusa_config& c = ctx->cfg;
+  if (draft_topk_out)
+    CU(cudaMemcpyAsync(draft_topk_out, ctx->wsp + ctx->ws.topk, (size_t)ctx->batch * c.n_draft_heads * c.draft_topk * 4,
+                       cudaMemcpyDeviceToDevice, ctx->stream));
+  if (tree_tokens) {
+    // tokens of the tree without a model pass: the embed kernel computes them; run it alone
+    const TreeView tv = tree_of(ctx, false);
+    const int M = ctx->batch * tv.n_nodes;
+    if (c.dtype == 1)
+      tree_embed_kernel<bf16><<<M, 128, 0, ctx->stream>>>(
+          tv, nullptr, wsptr<int32_t>(ctx, ctx->ws.root), wsptr<int32_t>(ctx, ctx->ws.topk), c.n_draft_heads, c.draft_topk,
+          wsptr<int32_t>(ctx, ctx->ws.ctx_len), wsptr<int32_t>(ctx, ctx->ws.nvalid), as<bf16>(ctx->emb_audio),
+          as<bf16>(ctx->emb_phon), as<bf16>(ctx->pos), c.vocab, c.n_phonemes, c.max_pos, c.d_model,
+          wsptr<int32_t>(ctx, ctx->ws.tokens), wsptr<float>(ctx, ctx->ws.x), err_word(ctx));
+    else
+      tree_embed_kernel<float><<<M, 128, 0, ctx->stream>>>(
+          tv, nullptr, wsptr<int32_t>(ctx, ctx->ws.root), wsptr<int32_t>(ctx, ctx->ws.topk), c.n_draft_heads, c.draft_topk,
+          wsptr<int32_t>(ctx, ctx->ws.ctx_len), wsptr<int32_t>(ctx, ctx->ws.nvalid), as<float>(ctx->emb_audio),
+          as<float>(ctx->emb_phon), as<float>(ctx->pos), c.vocab, c.n_phonemes, c.max_pos, c.d_model,
+          wsptr<int32_t>(ctx, ctx->ws.tokens), wsptr<float>(ctx, ctx->ws.x), err_word(ctx));
+    LAUNCH_CHECK();
+    CU(cudaMemcpyAsync(tree_tokens, ctx->wsp + ctx->ws.tokens, (size_t)M * 4, cudaMemcpyDeviceToDevice, ctx->stream));
+  }
+  return VADUSA_OK;
+}
+
+vadusa_status vadusa_verify_step(vadusa_ctx* ctx, const int32_t* tree_tokens_override, float* logits_out,
+                                 void* attn_tap, void* hidden_out) {
+  if (vadusa_status s = need_batch(ctx)) return s;
+  if (ctx->n_nodes == 0) return fail(ctx, VADUSA_ESTATE, "no tree set");
+  if (!tree_tokens_override && !ctx->have_draft) return fail(ctx, VADUSA_ESTATE, "verify without a draft or an override");
+  const TreeView tv = tree_of(ctx, false);
+  vadusa_status s = DISPATCH(forward<float>(ctx, tv, tree_tokens_override, reinterpret_cast<float*>(attn_tap)),
+                             forward<bf16>(ctx, tv, tree_tokens_override, reinterpret_cast<bf16*>(attn_tap)));
+  if (s) return s;
+  ctx->have_verify = true;
+  const vadusa_config& c = ctx->cfg;
+  const int M = ctx->batch * tv.n_nodes;
+  if (logits_out)
+    CU(cudaMemcpy2DAsync(logits_out, (size_t)c.vocab * 4, ctx->wsp + ctx->ws.logits, (size_t)vpad(&c) * 4,
+                         (size_t)c.vocab * 4, M, cudaMemcpyDeviceToDevice, ctx->stream));
+  if (hidden_out)
+    CU(cudaMemcpyAsync(hidden_out, ctx->wsp + ctx->ws.hfinal, (size_t)M * c.d_model * esize(&c), cudaMemcpyDeviceToDevice, ctx->stream));
+  return VADUSA_OK;
+}
+
+vadusa_status vadusa_accept_and_commit(vadusa_ctx* ctx, const vadusa_sampling* sampling, const int32_t* forced_best_node,
+                                       int32_t* accept_len, int32_t* path_nodes, int32_t* path_tokens,
+                                       int64_t* kv_slots, uint64_t* edge_bits, int32_t* next_root) {
+  if (vadusa_status s = need_batch(ctx)) return s;
+  if (!ctx->have_verify) return fail(ctx, VADUSA_ESTATE, "accept without a verify step");
+  SamplingDev sp;
+  if (vadusa_status s = sampling_dev(ctx, sampling, &sp)) return s;
+  AcceptOut out{accept_len, path_nodes, path_tokens, reinterpret_cast<long long*>(kv_slots),
+                reinterpret_cast<unsigned long long*>(edge_bits), next_root};
+  vadusa_status s = DISPATCH(accept_commit<float>(ctx, sp, forced_best_node, out, nullptr, 0, 0),
+                             accept_commit<bf16>(ctx, sp, forced_best_node, out, nullptr, 0, 0));
+  if (s) return s;
+  ctx->have_verify = ctx->have_draft = false;
+  return VADUSA_OK;
+}
+
+vadusa_status vadusa_generate(vadusa_ctx* ctx, const vadusa_sampling* sampling, int32_t max_new_tokens,
+                              int32_t max_iters, int32_t* out_tokens, int32_t* out_len, vadusa_stats* h_stats) {
+  if (vadusa_status s = need_batch(ctx)) return s;
+  if (ctx->n_nodes == 0 || ctx->tree_per_seq) return fail(ctx, VADUSA_ESTATE, "generate needs a shared tree template");
+  if (max_new_tokens < 1) return fail(ctx, VADUSA_EINVAL, "max_new_tokens must be positive");
+  SamplingDev sp;
+  if (vadusa_status s = sampling_dev(ctx, sampling, &sp)) return s;
+  const int64_t launches0 = ctx->launches;
+  const int limit = max_iters > 0 ? max_iters : max_new_tokens;
+  const TreeView tv = tree_of(ctx, false);
+  AcceptOut none{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  CU(cudaMemsetAsync(ctx->wsp + ctx->ws.gen_count, 0, ctx->batch * 4, ctx->stream));
+  CU(cudaMemsetAsync(done_word(ctx), 0, 4, ctx->stream));
+  if (vadusa_status s = set_active(ctx, ctx->n_nodes)) return s;
+  ctx->h_pinned[0] = 0;
+  bool poll_pending = false;
+  int iters = 0;
+  CU(cudaEventRecord(ctx->ev0, ctx->stream));
+  for (; iters < limit; ++iters) {
+    if (poll_pending && cudaEventQuery(ctx->ev_poll) == cudaSuccess) {
+      poll_pending = false;
+      if (ctx->h_pinned[0] >= ctx->batch) break;
+    }
+    vadusa_status s = DISPATCH(draft<float>(ctx, sp), draft<bf16>(ctx, sp));
+    if (s) return s;
+    s = DISPATCH(forward<float>(ctx, tv, nullptr, nullptr), forward<bf16>(ctx, tv, nullptr, nullptr));
+    if (s) return s;
+    s = DISPATCH(accept_commit<float>(ctx, sp, nullptr, none, out_tokens, max_new_tokens, max_new_tokens),
+                 accept_commit<bf16>(ctx, sp, nullptr, none, out_tokens, max_new_tokens, max_new_tokens));
+    if (s) return s;
+    if (!poll_pending && (iters & 7) == 7) {
+      CU(cudaMemcpyAsync(ctx->h_pinned, done_word(ctx), 4, cudaMemcpyDeviceToHost, ctx->stream));
+      CU(cudaEventRecord(ctx->ev_poll, ctx->stream));
+      poll_pending = true;
+    }
+  }
+  CU(cudaEventRecord(ctx->ev1, ctx->stream));
+  // lengths: min(gen_count, max_new_tokens) — computed on the host after the final sync
+  std::vector<int32_t> gen(ctx->batch);
+  CU(cudaMemcpyAsync(gen.data(), ctx->wsp + ctx->ws.gen_count, ctx->batch * 4, cudaMemcpyDeviceToHost, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  int64_t total = 0;
+  for (int b = 0; b < ctx->batch; ++b) { total += gen[b]; gen[b] = gen[b] > max_new_tokens ? max_new_tokens : gen[b]; }
+  if (out_len) CU(cudaMemcpyAsync(out_len, gen.data(), ctx->batch * 4, cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  if (h_stats) {
+    float ms = 0.f;
+    CU(cudaEventElapsedTime(&ms, ctx->ev0, ctx->ev1));
+    h_stats->iterations = iters;
+    h_stats->tokens_generated = total;
+    h_stats->elapsed_ms = ms;
+    h_stats->kernel_launches = ctx->launches - launches0;
+  }
+  ctx->have_draft = ctx->have_verify = false;
+  return device_errors(ctx);
+}
+
+vadusa_status vadusa_generate_host(vadusa_ctx* ctx, const vadusa_sampling* sampling, int32_t batch,
+                                   const int32_t* block_table, const int32_t* h_tokens, const int32_t* h_len,
+                                   int32_t stride, int32_t max_new_tokens, int32_t* h_out_tokens,
+                                   int32_t* h_out_len, vadusa_stats* h_stats) {
+  if (!ctx) return VADUSA_EINVAL;
+  if (!h_out_tokens || !h_out_len) return fail(ctx, VADUSA_EINVAL, "output pointers are NULL");
+  if (max_new_tokens < 1 || max_new_tokens > kGenHostCap)
+    return fail(ctx, VADUSA_EINVAL, "vadusa_generate_host: max_new_tokens must be in 1..%d", kGenHostCap);
+  vadusa_status s = vadusa_begin(ctx, batch, block_table, nullptr);
+  if (s) return s;
+  s = vadusa_prefill(ctx, h_tokens, h_len, stride);
+  if (s) return s;
+  int32_t* d_out = wsptr<int32_t>(ctx, ctx->ws.gen_out);
+  int32_t* d_len = wsptr<int32_t>(ctx, ctx->ws.gen_len);
+  s = vadusa_generate(ctx, sampling, max_new_tokens, 0, d_out, d_len, h_stats);
+  if (s == VADUSA_OK) {
+    cudaMemcpyAsync(h_out_tokens, d_out, (size_t)batch * max_new_tokens * 4, cudaMemcpyDeviceToHost, ctx->stream);
+    cudaMemcpyAsync(h_out_len, d_len, (size_t)batch * 4, cudaMemcpyDeviceToHost, ctx->stream);
+  }
+  CU(cudaStreamSynchronize(ctx->stream));
+  return s;
+}
+
+vadusa_status vadusa_get_lengths(vadusa_ctx* ctx, int32_t* h_ctx_len) {
+  if (vadusa_status s = need_batch(ctx)) return s;
+  if (!h_ctx_len) return fail(ctx, VADUSA_EINVAL, "h_ctx_len is NULL");
+  CU(cudaMemcpyAsync(h_ctx_len, ctx->wsp + ctx->ws.ctx_len, ctx->batch * 4, cudaMemcpyDeviceToHost, ctx->stream));
+  return device_errors(ctx);
+}
+
+vadusa_status vadusa_check(vadusa_ctx* ctx) {
+  if (!ctx || !ctx->wsp) return VADUSA_EINVAL;
+  return device_errors(ctx);
+}
+
+int64_t vadusa_kernel_launches(const vadusa_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

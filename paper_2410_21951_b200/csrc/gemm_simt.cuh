@@ -1,0 +1,137 @@
+// Plain FMA matrix product C[m,n] = sum_k A[m,k] * W[n,k] with fused epilogues.
+// This is the arithmetic of the fp32 model type (no tensor-core rounding); the
+// bf16 model type uses the tensor-core kernels and only falls back to this
+// file for shapes those do not cover.
+#pragma once
+#include "common.cuh"
+
+namespace vadusa {
+
+// ---- epilogues: called once per output element with the fp32 accumulator ----------
+
+// q/k/v projection (verify step, per layer): + bias, round to T; q goes to a dense
+// buffer, k and v go straight to the paged cache at slot ctx_len[b] + node.
+template <typename T>
+struct EpiQKV {
+  const float* bias;
+  T* q;
+  T* pool;                      // KV pool of this layer
+  const int32_t* block_table;
+  const int32_t* ctx_len;
+  const int32_t* nvalid;
+  uint32_t* err;
+  KvGeom geom;
+  int n_nodes, d;
+  __device__ __forceinline__ void operator()(int, int m, int n, float acc) const {
+    T r = from_f<T>(acc + bias[n]);
+    if (n < d) { q[(long long)m * d + n] = r; return; }
+    const int b = m / n_nodes, node = m % n_nodes;
+    if (node >= nvalid[b]) return;
+    const int pos = ctx_len[b] + node;
+    const long long blk = kv_block_of(block_table, geom, b, pos, err);
+    if (blk < 0) return;
+    const int c = n - d, kv = c / d, cc = c % d;
+    pool[geom.elem(blk, kv, cc / geom.head_dim, pos % kKvBlock) + cc % geom.head_dim] = r;
+  }
+};
+
+// output projection / second feed-forward matrix: x += acc + bias (fp32 residual stream)
+struct EpiResidual {
+  const float* bias;
+  float* x;
+  int ld;
+  __device__ __forceinline__ void operator()(int, int m, int n, float acc) const {
+    x[(long long)m * ld + n] += acc + bias[n];
+  }
+};
+
+// first feed-forward matrix: relu(acc + bias) rounded to T
+template <typename T>
+struct EpiRelu {
+  const float* bias;
+  T* out;
+  int ld;
+  __device__ __forceinline__ void operator()(int, int m, int n, float acc) const {
+    out[(long long)m * ld + n] = from_f<T>(fmaxf(acc + bias[n], 0.f));
+  }
+};
+
+// vocabulary heads: fp32 logits; z selects the draft head
+struct EpiLogits {
+  float* out;
+  int ld;
+  long long z_stride;
+  __device__ __forceinline__ void operator()(int z, int m, int n, float acc) const {
+    out[z * z_stride + (long long)m * ld + n] = acc;
+  }
+};
+
+// draft residual block (Sec. III-A.1): z = h + SiLU(acc + bias), rounded to T; z selects the head
+template <typename T>
+struct EpiDraftHidden {
+  const float* bias;     // [heads][d]
+  const T* h;            // [batch][d]
+  T* out;                // [heads][batch][d]
+  int d, batch;
+  __device__ __forceinline__ void operator()(int z, int m, int n, float acc) const {
+    const float t = acc + bias[z * d + n];
+    const float s = t / (1.0f + expf(-t));
+    out[((long long)z * batch + m) * d + n] = from_f<T>(to_f<T>(h[(long long)m * d + n]) + s);
+  }
+};
+
+// ---- kernel -----------------------------------------------------------------------
+// 64x64 tile, K step 16, 256 threads, 4x4 outputs per thread.  K must be a multiple of 16.
+// grid = (ceil(N/64), ceil(M/64), batches); A and W advance by a_z / w_z elements per batch.
+template <typename T, typename Epi>
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ A, const T* __restrict__ W,
+                                                        int M, int N, int K, long long a_z, long long w_z, Epi epi) {
+  __shared__ float As[16][64 + 4];
+  __shared__ float Ws[16][64 + 4];
+  const int z = blockIdx.z;
+  A += z * a_z; W += z * w_z;
+  const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int lr = threadIdx.x >> 2, lk = (threadIdx.x & 3) * 4;   // loader: row 0..63, k offset 0,4,8,12
+  float acc[4][4] = {};
+  for (int k0 = 0; k0 < K; k0 += 16) {
+    {
+      const int gm = m0 + lr, gn = n0 + lr;
+      float a[4] = {0.f, 0.f, 0.f, 0.f}, w[4] = {0.f, 0.f, 0.f, 0.f};
+      if (gm < M) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) a[i] = to_f<T>(A[(long long)gm * K + k0 + lk + i]);
+      }
+      if (gn < N) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) w[i] = to_f<T>(W[(long long)gn * K + k0 + lk + i]);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { As[lk + i][lr] = a[i]; Ws[lk + i][lr] = w[i]; }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      float a[4], w[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { a[i] = As[k][ty * 4 + i]; w[i] = Ws[k][tx * 4 + i]; }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], w[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = m0 + ty * 4 + i;
+    if (m >= M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tx * 4 + j;
+      if (n < N) epi(z, m, n, acc[i][j]);
+    }
+  }
+}
+
+}  // namespace vadusa

@@ -1,0 +1,186 @@
+"""Shared set-up of the GPU parity tests: runs the CUDA path and the CPU oracle on
+the same seeded inputs, iteration by iteration.
+
+Lockstep protocol: in every iteration the oracle drafts; the CUDA draft is
+compared with it wherever the oracle's decision margin exceeds MARGIN; the CUDA
+verify step then scores the oracle's tree tokens (override), logits are compared
+within the floating-point tolerance, and the accept/commit results are compared
+bit for bit when the oracle's acceptance margin exceeds MARGIN (otherwise the
+iteration is counted as undecidable and the CUDA path is told the oracle's
+choice so that both sides keep the same token history).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+
+import oracle as O
+import workloads as W
+
+MARGIN = 1e-3
+TOL = {"fp32": 1e-4, "bf16": 2e-2}
+MAX_PATH = 16
+
+
+def tokens_with_phonemes(shape, phon, prompt) -> np.ndarray:
+    """Prefix as the C ABI wants it: phoneme p is written vocab + p."""
+    return np.concatenate([np.asarray(phon, dtype=np.int32) + shape.vocab, np.asarray(prompt, dtype=np.int32)])
+
+
+def make_gpu(shape, weights, batch, n_nodes, tokens_per_seq, seed, draft_topk=10, spare_pages=3):
+    """Context whose block table (shuffled pages) covers tokens_per_seq[b] positions."""
+    import paper_2410_21951_b200 as P
+    table, total = W.shuffled_block_table(tokens_per_seq, 64, seed, spare_pages=spare_pages)
+    g = P.Vadusa(shape, weights, max_batch=batch, max_tree_nodes=n_nodes, max_blocks_per_seq=table.shape[1],
+                 kv_num_blocks=total, draft_topk=draft_topk)
+    return g, table
+
+
+def expected_slots(table: np.ndarray, b: int, S: int, n: int) -> List[int]:
+    return [int(table[b, (S + j) // 64]) * 64 + (S + j) % 64 for j in range(n)]
+
+
+def inject_kv(g, table, b: int, K: np.ndarray, V: np.ndarray):
+    """Write context rows K, V [L, S, H, dh] of sequence b into the paged pool."""
+    import torch
+    view = g.kv_view()
+    S = K.shape[1]
+    for p0 in range(0, S, 64):
+        n = min(64, S - p0)
+        blk = int(table[b, p0 // 64])
+        k = torch.from_numpy(np.ascontiguousarray(K[:, p0:p0 + n].transpose(0, 2, 1, 3))).to(g.dev).to(g.tdtype)
+        v = torch.from_numpy(np.ascontiguousarray(V[:, p0:p0 + n].transpose(0, 2, 1, 3))).to(g.dev).to(g.tdtype)
+        view[:, blk, 0, :, :n] = k
+        view[:, blk, 1, :, :n] = v
+
+
+def read_kv(g, table, b: int, S: int):
+    """Rows [L, S, H, dh] (float64) of sequence b from the paged pool."""
+    view = g.kv_view()
+    Ks, Vs = [], []
+    for p0 in range(0, S, 64):
+        n = min(64, S - p0)
+        blk = int(table[b, p0 // 64])
+        Ks.append(view[:, blk, 0, :, :n].float().cpu().numpy().transpose(0, 2, 1, 3))
+        Vs.append(view[:, blk, 1, :, :n].float().cpu().numpy().transpose(0, 2, 1, 3))
+    return np.concatenate(Ks, axis=1).astype(np.float64), np.concatenate(Vs, axis=1).astype(np.float64)
+
+
+@dataclass
+class LockstepReport:
+    iterations: int = 0
+    root_checked: int = 0
+    draft_heads_checked: int = 0
+    draft_heads_total: int = 0
+    accept_checked: int = 0
+    accept_undecidable: int = 0
+    max_logit_err: float = 0.0
+    max_attn_err: float = 0.0
+    accept_lens: List[int] = field(default_factory=list)
+
+
+def lockstep(g, table, model, states: Dict[int, "O.State"], template, sp_oracle, sp_gpu, n_iters: int,
+             dtype: str, oracle_mode: str = "tree", check_attn: bool = False,
+             planted: Optional[Dict[int, Sequence[int]]] = None) -> LockstepReport:
+    """Runs n_iters iterations.  `states` maps sequence index -> oracle state for the
+    sequences the oracle follows (the others run on the CUDA draft alone).
+    planted[b]: tokens the oracle's plain AR decoding produced for b; when given,
+    the true continuation is planted along the rank-0 path so that several tokens
+    are accepted."""
+    import torch
+    B, N, V, d, L = g.batch, template.n_nodes, model.V, model.d, model.L
+    dev = g.dev
+    rep = LockstepReport()
+    tree_tokens = torch.zeros(B, N, dtype=torch.int32, device=dev)
+    topk = torch.zeros(B, g.cfg.n_draft_heads, g.cfg.draft_topk, dtype=torch.int32, device=dev)
+    logits = torch.zeros(B, N, V, dtype=torch.float32, device=dev)
+    attn = torch.zeros(L, B, N, d, dtype=g.tdtype, device=dev) if check_attn else None
+    acc_len = torch.zeros(B, dtype=torch.int32, device=dev)
+    pnodes = torch.zeros(B, MAX_PATH, dtype=torch.int32, device=dev)
+    ptoks = torch.zeros(B, MAX_PATH, dtype=torch.int32, device=dev)
+    slots = torch.zeros(B, MAX_PATH, dtype=torch.int64, device=dev)
+    ebits = torch.zeros(B, dtype=torch.int64, device=dev)
+    nroot = torch.zeros(B, dtype=torch.int32, device=dev)
+    tol = TOL[dtype]
+    kused = int(template.rank.max()) + 1
+    rank0_path = [n for n in range(N) if all(r == 0 for r in template.rank_path(n))]
+    for it in range(n_iters):
+        g.draft(sp_gpu, tree_tokens=tree_tokens, topk_out=topk)
+        gpu_tokens = tree_tokens.cpu().numpy()
+        gpu_topk = topk.cpu().numpy()
+        gpu_len0 = g.lengths()
+        override = gpu_tokens.copy()
+        forced = np.full(B, -1, dtype=np.int32)
+        traces = {}
+        for b, st in states.items():
+            assert gpu_len0[b] == st.S
+            ov = None
+            if planted is not None:
+                # oracle's own draft first (on a throw-away copy), then plant the truth on the leftmost path
+                probe = O.vadusa_iteration(model, _clone_state(model, st), template, sp_oracle, mode=oracle_mode)
+                ov = probe.tree_tokens.copy()
+                done = len(st.tokens)
+                for j, n in enumerate(rank0_path):
+                    if done + j < len(planted[b]):
+                        ov[n] = planted[b][done + j]
+            tr = O.vadusa_iteration(model, st, template, sp_oracle, mode=oracle_mode, tokens_override=ov)
+            traces[b] = tr
+            if tr.margin_root > MARGIN:
+                assert gpu_tokens[b, 0] == tr.root, f"it {it} seq {b}: root {gpu_tokens[b, 0]} != {tr.root}"
+                rep.root_checked += 1
+            for h in range(model.n_draft):
+                rep.draft_heads_total += 1
+                used = int(template.rank[template.depth == h + 1].max()) + 1 if np.any(template.depth == h + 1) else 0
+                if used and tr.margin_draft[h] > MARGIN:
+                    assert np.array_equal(gpu_topk[b, h, :used], tr.topk[h, :used]), f"it {it} seq {b} head {h}"
+                    rep.draft_heads_checked += 1
+            override[b] = tr.tree_tokens
+            if not tr.margin_accept > MARGIN:
+                forced[b] = tr.best_node
+        g.verify_step(override=torch.from_numpy(override).to(dev), logits_out=logits, attn_tap=attn)
+        g.accept_and_commit(sp_gpu, forced_best=torch.from_numpy(forced).to(dev), accept_len=acc_len,
+                            path_nodes=pnodes, path_tokens=ptoks, kv_slots=slots, edge_bits=ebits, next_root=nroot)
+        lg = logits.cpu().numpy().astype(np.float64)
+        at = attn.float().cpu().numpy().astype(np.float64) if check_attn else None
+        al, pn, pt, sl = acc_len.cpu().numpy(), pnodes.cpu().numpy(), ptoks.cpu().numpy(), slots.cpu().numpy()
+        eb = ebits.cpu().numpy().astype(np.uint64)
+        for b, tr in traces.items():
+            err = float(np.abs(lg[b] - tr.node_logits).max())
+            rep.max_logit_err = max(rep.max_logit_err, err)
+            assert err <= tol, f"it {it} seq {b}: logits differ by {err}"
+            if check_attn and tr.attn is not None:
+                for l in range(L):
+                    e = float(np.abs(at[l, b] - tr.attn[l]).max())
+                    rep.max_attn_err = max(rep.max_attn_err, e)
+                    assert e <= tol, f"it {it} seq {b} layer {l}: attention outputs differ by {e}"
+            n_acc = tr.accept_len
+            assert al[b] == n_acc and list(pn[b, :n_acc]) == tr.path_nodes, \
+                f"it {it} seq {b}: path {list(pn[b, :al[b]])} != {tr.path_nodes} (margin {tr.margin_accept})"
+            assert list(pt[b, :n_acc]) == tr.path_tokens
+            assert np.all(pn[b, n_acc:] == -1) and np.all(pt[b, n_acc:] == -1)
+            assert list(sl[b, :n_acc]) == expected_slots(table, b, tr.S, n_acc)
+            if forced[b] < 0:
+                rep.accept_checked += 1
+                want = 1
+                acc = {0}
+                for n in range(1, N):
+                    p = int(template.parent[n])
+                    if p in acc and tr.edge_ok[n]:
+                        acc.add(n); want |= 1 << n
+                assert int(eb[b]) == want, f"it {it} seq {b}: edge bits {int(eb[b]):x} != {want:x}"
+            else:
+                rep.accept_undecidable += 1
+            rep.accept_lens.append(n_acc)
+        rep.iterations += 1
+    lens = g.lengths()
+    for b, st in states.items():
+        assert lens[b] == st.S
+    return rep
+
+
+def _clone_state(model, st):
+    kv = O.KVCache(model, capacity=st.kv.K.shape[1])
+    kv.extend(st.kv.K[:, :st.kv.n].copy(), st.kv.V[:, :st.kv.n].copy())
+    return O.State(kv=kv, tokens=list(st.tokens), h_star=st.h_star.copy(), logits_star=st.logits_star.copy(), seq=st.seq)
