@@ -35,10 +35,11 @@
  * Numeric types: dtype 0 keeps weights, K/V and activations in fp32 (plain
  *  fp32 FMA arithmetic).  dtype 1 keeps matrices, embeddings, K/V and the
  *  activations that feed a matrix product in bf16 (rounded to nearest even
- *  where produced: LayerNorm outputs, q/k/v, softmax weights before P.V,
- *  attention output, feed-forward hidden layer, final hidden state, draft
- *  residual block output) and accumulates in fp32; the residual stream,
- *  softmax statistics, logits and sampling keys are fp32.
+ *  where produced: LayerNorm outputs, q/k/v, attention output, feed-forward
+ *  hidden layer, final hidden state, draft residual block output) and
+ *  accumulates in fp32; the residual stream, softmax weights and statistics,
+ *  logits and sampling keys are fp32 (the softmax weights enter the P.V product
+ *  with at least 16 significant bits).
  */
 #ifndef VADUSA_H
 #define VADUSA_H
@@ -232,6 +233,20 @@ vadusa_status vadusa_generate_host(vadusa_ctx *ctx, const vadusa_sampling *sampl
 vadusa_status vadusa_get_lengths(vadusa_ctx *ctx, int32_t *h_ctx_len);  /* synchronises */
 vadusa_status vadusa_check(vadusa_ctx *ctx);                            /* synchronises; device error word */
 int64_t vadusa_kernel_launches(const vadusa_ctx *ctx);                  /* total kernels enqueued so far */
+
+/* ---- measurement ------------------------------------------------------------------ */
+/* Between vadusa_profile_begin and vadusa_profile_end every kernel launch of the library
+ * is bracketed by a pair of CUDA events on the context's stream.  vadusa_profile_end
+ * synchronises and returns, per kernel class, the number of launches and the summed
+ * device time.  h_out: host array of `capacity` >= 16 entries; *h_count entries are
+ * written.  The events perturb the stream slightly: take whole-step timings outside. */
+typedef struct {
+  char name[32];
+  int64_t launches;
+  double total_ms;
+} vadusa_kernel_time;
+vadusa_status vadusa_profile_begin(vadusa_ctx *ctx);
+vadusa_status vadusa_profile_end(vadusa_ctx *ctx, vadusa_kernel_time *h_out, int32_t capacity, int32_t *h_count);
 
 #ifdef __cplusplus
 }

@@ -135,6 +135,7 @@ class IterationTrace:
     path_tokens: List[int]
     margin_root: float
     margin_draft: np.ndarray         # [n_draft]
+    draft_gaps: np.ndarray           # [n_draft, kmax]: logit gap between candidates r and r+1 of each head
     margin_accept: float
     attn: Optional[List[np.ndarray]] = None     # per layer [N, d] (tree mode only)
     K: Optional[np.ndarray] = None              # [L, N, H, dh] rows of every node (tree/memo mode)
@@ -156,8 +157,13 @@ def _edge_margin(model: Model, logits, sp: Sampling, seq: int, pos: int, c: int)
     """Distance of candidate c from the boundary of the draw set at one node."""
     l32, keys, nuc = _keys_and_nucleus(model, logits, sp, seq, pos, noise=(sp.accept_rule == 0))
     m = float("inf")
-    if sp.temperature != 0.0 and sp.top_p < 1.0 and np.isfinite(l32[c]):
-        m = abs(nucleus_mass_before(l32, sp.temperature, c) - sp.top_p)
+    if sp.temperature != 0.0 and sp.top_p < 1.0:
+        # how close any prefix mass of the descending-probability order comes to top_p:
+        # the membership of every token, not only of c, shapes the draw set
+        z = l32.astype(np.float64) / float(sp.temperature)
+        p = np.exp(z - z.max()); p = np.sort(p / p.sum())[::-1]
+        before = np.concatenate([[0.0], np.cumsum(p)[:-1]])
+        m = float(np.min(np.abs(before - sp.top_p)))
     if not nuc[c]:
         return m
     ks = np.sort(keys[nuc].astype(np.float64))[::-1]
@@ -190,6 +196,10 @@ def vadusa_iteration(model: Model, st: State, template, sp: Sampling, mode: str 
         _draft_margin(masked_logits32(dl[i], model.eos_id, sp.eos_masked),
                       int(template.rank[template.depth == i + 1].max()) + 1 if np.any(template.depth == i + 1) else 0)
         for i in range(model.n_draft)])
+    draft_gaps = np.zeros((model.n_draft, kmax))
+    for i in range(model.n_draft):
+        srt = np.sort(masked_logits32(dl[i], model.eos_id, sp.eos_masked).astype(np.float64))[::-1]
+        draft_gaps[i] = srt[:kmax] - srt[1:kmax + 1]
     toks = build_tree_tokens(template, root, topk) if tokens_override is None \
         else np.asarray(tokens_override, dtype=np.int32).copy()
 
@@ -273,7 +283,7 @@ def vadusa_iteration(model: Model, st: State, template, sp: Sampling, mode: str 
     return IterationTrace(S=S, root=root, topk=topk, tree_tokens=toks, node_logits=node_logits,
                           node_h=node_h, edge_ok=edge_ok, accept_len=k_star + 1, best_node=best,
                           path_nodes=list(path), path_tokens=[int(toks[n]) for n in path],
-                          margin_root=_gap_top2(keys_s, nuc_s), margin_draft=margin_draft,
+                          margin_root=_gap_top2(keys_s, nuc_s), margin_draft=margin_draft, draft_gaps=draft_gaps,
                           margin_accept=margin_accept, attn=attn, K=node_K, V=node_V)
 
 

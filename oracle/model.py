@@ -12,10 +12,12 @@ pass under an explicit tree mask (Sec. II-A, "tree attention"); it exists to be
 checked against `forward_token` and to give taps for large cases.
 
 In a "bf16" model the quantities the model stores in bf16 are rounded (nearest
-even) where they are produced: LayerNorm outputs, q/k/v, the softmax weights
-that multiply V, the attention output, the feed-forward hidden layer, the final
-hidden state, and the draft heads' residual-block output.  Sums (residual
-stream, dot products, softmax denominators, logits) are never rounded.
+even) where they are produced: LayerNorm outputs, q/k/v, the attention output,
+the feed-forward hidden layer, the final hidden state, and the draft heads'
+residual-block output.  Sums and what feeds them without being stored (residual
+stream, dot products, softmax weights and denominators, logits) are never
+rounded, so the definition does not depend on the order in which keys are
+visited.
 """
 from __future__ import annotations
 
@@ -146,7 +148,7 @@ def forward_token(model: Model, kv: KVCache, kind: int, tok: int, pos: int, taps
         Km, Vm = kv.rows(l, kv.own + 1)                    # [t, H, dh], includes this token
         s = np.einsum("hd,thd->ht", q, Km) * m.scale        # [H, t]
         e = np.exp(s - s.max(axis=1, keepdims=True))
-        o = np.einsum("ht,thd->hd", m.R(e), Vm) / e.sum(axis=1, keepdims=True)
+        o = np.einsum("ht,thd->hd", e, Vm) / e.sum(axis=1, keepdims=True)
         o = m.R(o).reshape(m.d)
         if taps:
             attn_taps.append(o.copy())
@@ -193,8 +195,7 @@ def forward_tree(model: Model, kv: KVCache, kinds, toks, positions, mask: np.nda
         s_new = np.einsum("nhd,mhd->hnm", q, k) * m.scale + neg[None]
         s = np.concatenate([s_ctx, s_new], axis=2)
         e = np.exp(s - s.max(axis=2, keepdims=True))
-        er = m.R(e)
-        o = (np.einsum("hnt,thd->nhd", er[:, :, :S], Vc) + np.einsum("hnm,mhd->nhd", er[:, :, S:], v))
+        o = (np.einsum("hnt,thd->nhd", e[:, :, :S], Vc) + np.einsum("hnm,mhd->nhd", e[:, :, S:], v))
         o = o / e.sum(axis=2).T[:, :, None]
         o = m.R(o).reshape(N, m.d)
         attn.append(o.copy())

@@ -59,11 +59,15 @@ class Stats(C.Structure):
                 ("kernel_launches", C.c_int64)]
 
 
+class KernelTime(C.Structure):
+    _fields_ = [("name", C.c_char * 32), ("launches", C.c_int64), ("total_ms", C.c_double)]
+
+
 EXPORTS = ["vadusa_workspace_bytes", "vadusa_weights_bytes", "vadusa_kv_pool_bytes", "vadusa_weight_count",
            "vadusa_weight_info", "vadusa_init", "vadusa_destroy", "vadusa_last_error", "vadusa_set_tree",
            "vadusa_begin", "vadusa_prefill", "vadusa_load_state", "vadusa_draft", "vadusa_verify_step",
            "vadusa_accept_and_commit", "vadusa_generate", "vadusa_generate_host", "vadusa_get_lengths",
-           "vadusa_check", "vadusa_kernel_launches"]
+           "vadusa_check", "vadusa_kernel_launches", "vadusa_profile_begin", "vadusa_profile_end"]
 
 _lib = None
 
@@ -94,6 +98,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "vadusa_generate_host": (I32, [P, C.POINTER(Sampling), I32, P, P, P, I32, I32, P, P, C.POINTER(Stats)]),
         "vadusa_get_lengths": (I32, [P, P]), "vadusa_check": (I32, [P]),
         "vadusa_kernel_launches": (I64, [P]),
+        "vadusa_profile_begin": (I32, [P]),
+        "vadusa_profile_end": (I32, [P, C.POINTER(KernelTime), I32, C.POINTER(I32)]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib_, name)
@@ -294,6 +300,16 @@ class Vadusa:
 
     def kernel_launches(self) -> int:
         return int(self.L.vadusa_kernel_launches(self.ctx))
+
+    def profile_begin(self):
+        self._ck(self.L.vadusa_profile_begin(self.ctx))
+
+    def profile_end(self) -> Dict[str, tuple]:
+        """{kernel class: (launches, total_ms)} since profile_begin."""
+        arr = (KernelTime * 32)()
+        n = C.c_int32(0)
+        self._ck(self.L.vadusa_profile_end(self.ctx, arr, 32, C.byref(n)))
+        return {arr[i].name.decode(): (int(arr[i].launches), float(arr[i].total_ms)) for i in range(n.value)}
 
     # ---- helpers for tests and benchmarks: views of the caller-owned KV pool ----
     def kv_view(self):

@@ -32,12 +32,13 @@ struct SeqState {             // device state of the batch (all [batch] unless n
 // for an accepted parent p the keys of its logits row are formed once in shared memory
 // (they predict absolute position ctx_len + depth(p) + 1), then each child token c is
 // accepted iff fewer than tau tokens precede it in key order (and it lies in the nucleus).
-// dynamic shared memory: ld floats.
+// dynamic shared memory: 2 * ld floats.
 __global__ void __launch_bounds__(256) accept_kernel(
     const float* __restrict__ logits, int ld, int vocab, const int32_t* __restrict__ tokens, TreeView tree,
     const int32_t* __restrict__ block_table, KvGeom geom, SamplingDev sp,
     const int32_t* __restrict__ forced_best, SeqState st, AcceptOut out, uint32_t* err) {
-  extern __shared__ float keys[];
+  extern __shared__ float keys[];          // [ld] keys, then [ld] probabilities (nucleus only)
+  float* probs = keys + ld;
   __shared__ int s_parent[kMaxNodes], s_depth[kMaxNodes], s_tok[kMaxNodes];
   __shared__ int s_child[kMaxNodes], s_ok[kMaxNodes], s_nchild;
   __shared__ unsigned long long s_edges, s_acc;
@@ -90,31 +91,38 @@ __global__ void __launch_bounds__(256) accept_kernel(
       const uint64_t rs = noise_row_state(sp.seed, b, S + d + 1);
       const bool noise = sp.accept_rule == 0;
       for (int j = tid; j < vocab; j += blockDim.x) keys[j] = key_of(row[j], j, rs, sp, noise);
+      if (nuc) {
+        // Tokens outside the top-p nucleus cannot be drawn: give them the key -inf.  A token is
+        // inside iff the probability mass ahead of it (larger logit, or equal and lower id) is
+        // below top_p; probs[] holds exp((l - max) / T).
+        const RowStats rst = row_stats(row, vocab, sp, fscratch);
+        for (int j = tid; j < vocab; j += blockDim.x)
+          probs[j] = expf((masked_logit(row[j], j, sp) - rst.maxl) * sp.inv_temperature);
+        __syncthreads();
+        for (int j = tid; j < vocab; j += blockDim.x) {
+          const float lj = masked_logit(row[j], j, sp);
+          float m = 0.f;
+          for (int i = 0; i < vocab; ++i)
+            if (precedes(masked_logit(row[i], i, sp), i, lj, j)) m += probs[i];
+          if (!(m / rst.z < sp.top_p)) keys[j] = -INFINITY;
+        }
+      }
       __syncthreads();
       for (int i = warp; i < nchild; i += (blockDim.x >> 5)) {
         const int c = s_tok[s_child[i]];
-        int cnt = 0;
+        int cnt = sp.tau;                                            // not a speech token: never accepted
+        bool finite = false;
         if (c >= 0 && c < vocab) {
           const float kc = keys[c];
+          finite = kc > -INFINITY;
+          cnt = 0;
           for (int j = lane; j < vocab; j += 32) cnt += precedes(keys[j], j, kc, c) ? 1 : 0;
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-        } else {
-          cnt = sp.tau;                                              // not a speech token: never accepted
         }
-        if (lane == 0) s_ok[i] = (cnt < sp.tau && keys[min(max(c, 0), vocab - 1)] > -INFINITY) ? 1 : 0;
+        if (lane == 0) s_ok[i] = (cnt < sp.tau && finite) ? 1 : 0;
       }
       __syncthreads();
-      if (nuc) {
-        RowStats rst = row_stats(row, vocab, sp, fscratch);
-        for (int i = 0; i < nchild; ++i) {
-          if (!s_ok[i]) continue;                                    // uniform
-          const bool in = in_nucleus(row, vocab, s_tok[s_child[i]], rst, sp, fscratch);
-          __syncthreads();
-          if (tid == 0 && !in) s_ok[i] = 0;
-          __syncthreads();
-        }
-      }
       if (tid == 0) {
         for (int i = 0; i < nchild; ++i)
           if (s_ok[i]) { s_edges |= 1ull << s_child[i]; s_acc |= 1ull << s_child[i]; }

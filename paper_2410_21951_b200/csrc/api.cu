@@ -40,7 +40,17 @@ struct vadusa_ctx {
   cudaEvent_t ev0 = nullptr, ev1 = nullptr, ev_poll = nullptr;
   int32_t* h_pinned = nullptr;     // [2]: done_count, err
   char err[512] = {0};
+  // per-kernel timing (vadusa_profile_begin/end): one event pair per launch
+  struct ProfRec { cudaEvent_t a, b; int cls; };
+  bool prof_on = false, prof_pending = false;
+  std::vector<ProfRec> prof;
 };
+
+enum KClass { K_EMBED, K_LAYERNORM, K_GEMM_QKV, K_ATTENTION, K_GEMM_OUT, K_GEMM_FFN1, K_GEMM_FFN2, K_GEMM_LM,
+              K_DRAFT_HIDDEN, K_DRAFT_LOGITS, K_DRAFT_SELECT, K_ACCEPT, K_COMMIT, K_MISC, K_NCLASS };
+static const char* const kClassName[K_NCLASS] = {
+    "tree_embed", "layernorm", "gemm_qkv", "tree_attention", "gemm_out", "gemm_ffn1", "gemm_ffn2", "gemm_lm",
+    "draft_hidden", "draft_logits", "draft_select", "accept", "commit", "misc"};
 
 namespace {
 
@@ -65,7 +75,19 @@ vadusa_status fail(vadusa_ctx* c, vadusa_status s, const char* fmt, ...) {
     cudaError_t e_ = cudaGetLastError();                                                           \
     if (e_ != cudaSuccess) return fail(ctx, VADUSA_ECUDA, "kernel launch: %s", cudaGetErrorString(e_)); \
     ctx->launches++;                                                                               \
+    if (ctx->prof_pending) { cudaEventRecord(ctx->prof.back().b, ctx->stream); ctx->prof_pending = false; } \
   } while (0)
+
+// Call right before a kernel launch: when profiling is on, brackets the launch with events.
+void PROF(vadusa_ctx* c, int cls) {
+  if (!c->prof_on) return;
+  vadusa_ctx::ProfRec r;
+  r.cls = cls;
+  if (cudaEventCreate(&r.a) != cudaSuccess || cudaEventCreate(&r.b) != cudaSuccess) return;
+  cudaEventRecord(r.a, c->stream);
+  c->prof.push_back(r);
+  c->prof_pending = true;
+}
 
 template <typename P> P* wsptr(vadusa_ctx* c, int64_t off) { return reinterpret_cast<P*>(c->wsp + off); }
 
@@ -168,9 +190,10 @@ vadusa_status sampling_dev(vadusa_ctx* ctx, const vadusa_sampling* s, SamplingDe
 // ---- typed engine ------------------------------------------------------------------
 
 template <typename T, typename Epi>
-vadusa_status gemm(vadusa_ctx* ctx, const T* A, const T* W, int M, int N, int K, int batches, long long a_z,
+vadusa_status gemm(vadusa_ctx* ctx, int cls, const T* A, const T* W, int M, int N, int K, int batches, long long a_z,
                    long long w_z, const Epi& epi) {
   dim3 grid((N + 63) / 64, (M + 63) / 64, batches);
+  PROF(ctx, cls);
   gemm_simt_kernel<T, Epi><<<grid, 256, 0, ctx->stream>>>(A, W, M, N, K, a_z, w_z, epi);
   LAUNCH_CHECK();
   return VADUSA_OK;
@@ -185,6 +208,7 @@ vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeVi
   dim3 grid(c.n_heads, ctx->batch);
   const size_t smem = (size_t)(64 * dh * 3 + 64 + 64 * 64) * sizeof(float);   // = attention_smem(dh)
   auto go = [&](auto kern) -> vadusa_status {
+    PROF(ctx, K_ATTENTION);
     kern<<<grid, 256, smem, ctx->stream>>>(q, pool, ctx->block_table, wsptr<int32_t>(ctx, ctx->ws.ctx_len),
                                            wsptr<int32_t>(ctx, ctx->ws.nvalid), tv, g, c.d_model, scale, out,
                                            err_word(ctx));
@@ -212,6 +236,7 @@ vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* overri
   int32_t* nvalid = wsptr<int32_t>(ctx, ctx->ws.nvalid);
   const int ln_blocks = (M + 3) / 4;
 
+  PROF(ctx, K_EMBED);
   tree_embed_kernel<T><<<M, 128, 0, ctx->stream>>>(
       tv, override_tokens, wsptr<int32_t>(ctx, ctx->ws.root), wsptr<int32_t>(ctx, ctx->ws.topk), c.n_draft_heads,
       c.draft_topk, ctx_len, nvalid, as<T>(ctx->emb_audio), as<T>(ctx->emb_phon), as<T>(ctx->pos),
@@ -220,31 +245,34 @@ vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* overri
   for (int l = 0; l < c.n_layers; ++l) {
     const LayerW& w = ctx->layers[l];
     T* pool = reinterpret_cast<T*>(c.kv_pool) + (long long)l * g.layer_stride;
+    PROF(ctx, K_LAYERNORM);
     layernorm_kernel<T><<<ln_blocks, 128, 0, ctx->stream>>>(x, w.ln1_g, w.ln1_b, a, M, d, c.ln_eps);
     LAUNCH_CHECK();
     EpiQKV<T> eq{w.bqkv, q, pool, ctx->block_table, ctx_len, nvalid, err_word(ctx), g, N, d};
-    vadusa_status s = gemm<T>(ctx, a, as<T>(w.wqkv), M, 3 * d, d, 1, 0, 0, eq);
+    vadusa_status s = gemm<T>(ctx, K_GEMM_QKV, a, as<T>(w.wqkv), M, 3 * d, d, 1, 0, 0, eq);
     if (s) return s;
     T* o_dst = attn_tap ? attn_tap + (long long)l * M * d : o;
     s = attention<T>(ctx, q, pool, tv, o_dst);
     if (s) return s;
     EpiResidual eo{w.bo, x, d};
-    s = gemm<T>(ctx, o_dst, as<T>(w.wo), M, d, d, 1, 0, 0, eo);
+    s = gemm<T>(ctx, K_GEMM_OUT, o_dst, as<T>(w.wo), M, d, d, 1, 0, 0, eo);
     if (s) return s;
+    PROF(ctx, K_LAYERNORM);
     layernorm_kernel<T><<<ln_blocks, 128, 0, ctx->stream>>>(x, w.ln2_g, w.ln2_b, a, M, d, c.ln_eps);
     LAUNCH_CHECK();
     EpiRelu<T> e1{w.b1, mid, f};
-    s = gemm<T>(ctx, a, as<T>(w.w1), M, f, d, 1, 0, 0, e1);
+    s = gemm<T>(ctx, K_GEMM_FFN1, a, as<T>(w.w1), M, f, d, 1, 0, 0, e1);
     if (s) return s;
     EpiResidual e2{w.b2, x, d};
-    s = gemm<T>(ctx, mid, as<T>(w.w2), M, d, f, 1, 0, 0, e2);
+    s = gemm<T>(ctx, K_GEMM_FFN2, mid, as<T>(w.w2), M, d, f, 1, 0, 0, e2);
     if (s) return s;
   }
+  PROF(ctx, K_LAYERNORM);
   layernorm_kernel<T><<<ln_blocks, 128, 0, ctx->stream>>>(x, ctx->lnf_g, ctx->lnf_b,
                                                           hfinal, M, d, c.ln_eps);
   LAUNCH_CHECK();
   EpiLogits el{logits, vp, 0};
-  return gemm<T>(ctx, hfinal, as<T>(ctx->lm), M, vp, d, 1, 0, 0, el);
+  return gemm<T>(ctx, K_GEMM_LM, hfinal, as<T>(ctx->lm), M, vp, d, 1, 0, 0, el);
 }
 
 template <typename T>
@@ -256,12 +284,13 @@ vadusa_status draft(vadusa_ctx* ctx, const SamplingDev& sp) {
   float* dl = wsptr<float>(ctx, ctx->ws.dlogits);
   const long long w_stride = ctx->dw_stride / (long long)sizeof(T), u_stride = ctx->du_stride / (long long)sizeof(T);
   EpiDraftHidden<T> eh{ctx->db, hstar, z, d, B};
-  vadusa_status s = gemm<T>(ctx, hstar, as<T>(ctx->dw), B, d, d, hd, 0, w_stride, eh);
+  vadusa_status s = gemm<T>(ctx, K_DRAFT_HIDDEN, hstar, as<T>(ctx->dw), B, d, d, hd, 0, w_stride, eh);
   if (s) return s;
   EpiLogits el{dl, vp, (long long)B * vp};
-  s = gemm<T>(ctx, z, as<T>(ctx->du), B, vp, d, hd, (long long)B * d, u_stride, el);
+  s = gemm<T>(ctx, K_DRAFT_LOGITS, z, as<T>(ctx->du), B, vp, d, hd, (long long)B * d, u_stride, el);
   if (s) return s;
   dim3 grid(hd + 1, B);
+  PROF(ctx, K_DRAFT_SELECT);
   draft_select_kernel<<<grid, 256, 0, ctx->stream>>>(dl, wsptr<float>(ctx, ctx->ws.logits_star), vp, c.vocab, B, hd,
                                                      c.draft_topk, wsptr<int32_t>(ctx, ctx->ws.ctx_len),
                                                      wsptr<int32_t>(ctx, ctx->ws.nvalid), sp,
@@ -280,11 +309,13 @@ vadusa_status accept_commit(vadusa_ctx* ctx, const SamplingDev& sp, const int32_
   const KvGeom g = geom_of(ctx);
   const TreeView tv = tree_of(ctx, false);
   SeqState st = state_of(ctx, out_tokens, out_cap, target);
-  accept_kernel<<<B, 256, vp * sizeof(float), ctx->stream>>>(
+  PROF(ctx, K_ACCEPT);
+  accept_kernel<<<B, 256, 2 * vp * sizeof(float), ctx->stream>>>(
       wsptr<float>(ctx, ctx->ws.logits), vp, c.vocab, wsptr<int32_t>(ctx, ctx->ws.tokens), tv, ctx->block_table, g,
       sp, forced, st, out, err_word(ctx));
   LAUNCH_CHECK();
   dim3 grid(c.n_layers + 1, B);
+  PROF(ctx, K_COMMIT);
   commit_kernel<T><<<grid, 256, 0, ctx->stream>>>(
       reinterpret_cast<T*>(c.kv_pool), g, ctx->block_table, st, c.n_layers, tv.n_nodes,
       wsptr<T>(ctx, ctx->ws.hfinal), c.d_model, wsptr<float>(ctx, ctx->ws.logits), vp, wsptr<T>(ctx, ctx->ws.hstar),
@@ -465,6 +496,7 @@ vadusa_status vadusa_destroy(vadusa_ctx* ctx) {
   if (ctx->ev1) cudaEventDestroy(ctx->ev1);
   if (ctx->ev_poll) cudaEventDestroy(ctx->ev_poll);
   if (ctx->h_pinned) cudaFreeHost(ctx->h_pinned);
+  for (auto& r : ctx->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
   delete ctx;
   return VADUSA_OK;
 }
@@ -609,6 +641,7 @@ vadusa_status vadusa_verify_step(vadusa_ctx* ctx, const int32_t* tree_tokens_ove
   if (vadusa_status s = need_batch(ctx)) return s;
   if (ctx->n_nodes == 0) return fail(ctx, VADUSA_ESTATE, "no tree set");
   if (!tree_tokens_override && !ctx->have_draft) return fail(ctx, VADUSA_ESTATE, "verify without a draft or an override");
+  if (!tree_tokens_override && ctx->tree_per_seq) return fail(ctx, VADUSA_ESTATE, "per-sequence topologies need a token override");
   const TreeView tv = tree_of(ctx, false);
   vadusa_status s = DISPATCH(forward<float>(ctx, tv, tree_tokens_override, reinterpret_cast<float*>(attn_tap)),
                              forward<bf16>(ctx, tv, tree_tokens_override, reinterpret_cast<bf16*>(attn_tap)));
@@ -733,5 +766,40 @@ vadusa_status vadusa_check(vadusa_ctx* ctx) {
 }
 
 int64_t vadusa_kernel_launches(const vadusa_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+vadusa_status vadusa_profile_begin(vadusa_ctx* ctx) {
+  if (!ctx || !ctx->wsp) return VADUSA_EINVAL;
+  for (auto& r : ctx->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+  ctx->prof.clear();
+  ctx->prof_on = true;
+  ctx->prof_pending = false;
+  return VADUSA_OK;
+}
+
+vadusa_status vadusa_profile_end(vadusa_ctx* ctx, vadusa_kernel_time* h_out, int32_t capacity, int32_t* h_count) {
+  if (!ctx || !ctx->wsp) return VADUSA_EINVAL;
+  if (!h_out || !h_count || capacity < K_NCLASS) return fail(ctx, VADUSA_EINVAL, "profile output needs room for %d entries", (int)K_NCLASS);
+  ctx->prof_on = false;
+  CU(cudaStreamSynchronize(ctx->stream));
+  double total[K_NCLASS] = {0};
+  int64_t count[K_NCLASS] = {0};
+  for (auto& r : ctx->prof) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, r.a, r.b) == cudaSuccess) { total[r.cls] += ms; count[r.cls]++; }
+    cudaEventDestroy(r.a); cudaEventDestroy(r.b);
+  }
+  ctx->prof.clear();
+  int n = 0;
+  for (int k = 0; k < K_NCLASS; ++k) {
+    if (!count[k]) continue;
+    memset(&h_out[n], 0, sizeof(h_out[n]));
+    snprintf(h_out[n].name, sizeof(h_out[n].name), "%s", kClassName[k]);
+    h_out[n].launches = count[k];
+    h_out[n].total_ms = total[k];
+    ++n;
+  }
+  *h_count = n;
+  return VADUSA_OK;
+}
 
 }  // extern "C"

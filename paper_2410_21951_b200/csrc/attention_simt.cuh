@@ -71,8 +71,8 @@ __global__ void __launch_bounds__(256) tree_attention_simt_kernel(
       const float corr = expf(mrun[i] - mnew);
       lrun[i] = lrun[i] * corr + warp_sum(p0 + p1);
       mrun[i] = mnew;
-      Ps[n * 64 + lane] = round_as<T>(p0);
-      Ps[n * 64 + lane + 32] = round_as<T>(p1);
+      Ps[n * 64 + lane] = p0;
+      Ps[n * 64 + lane + 32] = p1;
 #pragma unroll
       for (int c = 0; c < R; ++c) O[i][c] *= corr;
       __syncwarp();

@@ -1,0 +1,294 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on
+the same seeded inputs.  Integers (tokens, accepted lengths, paths, KV slots,
+edge bits) must match bit for bit wherever the oracle's decision margin exceeds
+1e-3; logits and attention outputs within 1e-4 (fp32 models) / 2e-2 (bf16)."""
+import numpy as np
+import pytest
+
+import oracle as O
+import workloads as W
+from harness import (MARGIN, MARGINS, TOL, expected_slots, inject_kv, lockstep, make_gpu, read_kv, tokens_with_phonemes)
+
+pytestmark = pytest.mark.gpu
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def _sampling(wl, seed=7, tau=None, temperature=None, top_p=1.0, accept_rule=0):
+    import paper_2410_21951_b200 as P
+    tau = wl.tau if tau is None else tau
+    t = wl.temperature if temperature is None else temperature
+    return (O.Sampling(tau=tau, temperature=t, top_p=top_p, seed=seed, accept_rule=accept_rule),
+            P.Sampling.make(tau=tau, temperature=t, top_p=top_p, seed=seed, accept_rule=accept_rule))
+
+
+def _prefill_both(wl, g, table, model, seqs, oracle_chunk=128):
+    """GPU prefill of every sequence of the workload; oracle prefill of `seqs`."""
+    prefixes = [W.prefix_for(wl, b) for b in range(wl.batch)]
+    toks = [tokens_with_phonemes(wl.shape, ph, pr) for ph, pr in prefixes]
+    stride = max(len(t) for t in toks)
+    mat = np.zeros((wl.batch, stride), dtype=np.int32)
+    for b, t in enumerate(toks):
+        mat[b, :len(t)] = t
+    g.begin(table)
+    g.prefill(mat, [len(t) for t in toks])
+    states = {b: O.prefill_blocked(model, prefixes[b][0], prefixes[b][1], seq=b, chunk=oracle_chunk) for b in seqs}
+    lens = g.lengths()
+    for b, st in states.items():
+        assert lens[b] == st.S == len(toks[b])
+    return states, toks
+
+
+def _setup(wl, n_iters, seqs, seed=11, extra=0):
+    w = W.make_weights(wl.shape, wl.seed())
+    model = O.Model.from_shape(wl.shape, w)
+    tpl = W.static_template(wl.tree_nodes, wl.tree_caps)
+    need = []
+    for b in range(wl.batch):
+        ph, pr = W.prefix_for(wl, b)
+        need.append(len(ph) + len(pr) + n_iters * (tpl.max_depth + 1) + wl.tree_nodes + extra)
+    g, table = make_gpu(wl.shape, w, wl.batch, wl.tree_nodes, need, seed)
+    g.set_tree(tpl.parent, tpl.rank)
+    return w, model, tpl, g, table
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_toy_lockstep_prefill_and_kv(dtype):
+    """Small model, several tiles worth of context after prefill, ragged prefix; also
+    checks that the committed K/V rows equal the oracle's."""
+    wl = W.toy_workload(dtype=dtype, d_model=128, n_heads=2, d_ffn=256, vocab=203, tree_nodes=16, tree_caps=(6, 3, 2),
+                        tau=3, temperature=1.0, batch=3, phoneme_len=(20, 70), prompt_len=90, index=11)
+    w, model, tpl, g, table = _setup(wl, 6, range(3))
+    states, _ = _prefill_both(wl, g, table, model, range(3), oracle_chunk=37)
+    so, sg = _sampling(wl)
+    rep = lockstep(g, table, model, states, tpl, so, sg, 6, dtype, oracle_mode="memo", check_attn=True)
+    assert rep.accept_checked > 0 and rep.root_checked > 0 and rep.draft_sets_checked > 0
+    for b, st in states.items():
+        K, V = read_kv(g, table, b, st.S)
+        assert np.abs(K - st.kv.K[:, :st.S]).max() <= TOL[dtype]
+        assert np.abs(V - st.kv.V[:, :st.S]).max() <= TOL[dtype]
+    g.check()
+
+
+@pytest.mark.parametrize("dtype,tau,temperature,top_p,rule", [("fp32", 2, 0.9, 0.8, 0), ("fp32", 3, 1.0, 1.0, 1),
+                                                               ("bf16", 5, 0.8, 1.0, 0), ("fp32", 1, 0.0, 1.0, 0)])
+def test_toy_planted_paths_are_accepted(dtype, tau, temperature, top_p, rule):
+    """The true continuation planted on the leftmost branch: several tokens are committed
+    per iteration and K/V rows move; nucleus and plain top-tau rules included."""
+    wl = W.toy_workload(dtype=dtype, d_model=64, n_heads=2, d_ffn=128, vocab=61, tree_nodes=12, tree_caps=(4, 3, 2),
+                        batch=2, phoneme_len=(9, 9), prompt_len=60, index=12)
+    w, model, tpl, g, table = _setup(wl, 8, range(2))
+    states, _ = _prefill_both(wl, g, table, model, range(2))
+    so, sg = _sampling(wl, seed=3, tau=tau, temperature=temperature, top_p=top_p, accept_rule=rule)
+    # truth under tolerance 1 (plain AR with the same noise)
+    so1 = O.Sampling(tau=1, temperature=temperature, top_p=top_p, seed=3, accept_rule=rule)
+    planted = {}
+    for b in range(2):
+        ph, pr = W.prefix_for(wl, b)
+        planted[b] = O.ar_decode(model, O.prefill(model, ph, pr, seq=b), so1, 40)
+    rep = lockstep(g, table, model, states, tpl, so, sg, 8, dtype, oracle_mode="memo", planted=planted)
+    if rule == 0:            # under rule 1 the noisy truth need not be among the plain top-tau
+        assert max(rep.accept_lens) == tpl.max_depth + 1
+    if tau == 1:
+        for b, st in states.items():
+            assert st.tokens == planted[b][:len(st.tokens)]
+    g.check()
+
+
+def test_c1_generate_matches_oracle_and_plain_ar():
+    """BASELINE config 1 end to end: free-running vadusa_generate (greedy, tolerance 1, 100
+    tokens) equals the oracle's speculative decoding and plain AR decoding token for token
+    up to the first position where the oracle's top-2 margin is below 1e-3."""
+    torch = _torch()
+    wl = W.workload("C1")
+    w, model, tpl, g, table = _setup(wl, wl.gen_tokens, [0])
+    states, toks = _prefill_both(wl, g, table, model, [0])
+    so, sg = _sampling(wl)
+    ph, pr = W.prefix_for(wl, 0)
+    ar_state = O.prefill(model, ph, pr)
+    truth, first_thin = [], None
+    for i in range(wl.gen_tokens):
+        l32 = O.sampling.masked_logits32(ar_state.logits_star, model.eos_id, True)
+        top2 = np.sort(l32)[-2:]
+        if first_thin is None and top2[1] - top2[0] <= MARGIN:
+            first_thin = i
+        truth += O.ar_decode(model, ar_state, so, 1)
+    out = torch.zeros(1, wl.gen_tokens, dtype=torch.int32, device=g.dev)
+    out_len = torch.zeros(1, dtype=torch.int32, device=g.dev)
+    stats = g.generate(sg, wl.gen_tokens, out, out_len)
+    got = out.cpu().numpy()[0]
+    n = wl.gen_tokens if first_thin is None else first_thin
+    assert n > 20
+    assert list(got[:n]) == truth[:n]
+    assert int(out_len.cpu()[0]) == wl.gen_tokens
+    assert stats.iterations <= wl.gen_tokens and stats.tokens_generated >= wl.gen_tokens and stats.kernel_launches > 0
+    # host-to-host entry gives the same tokens
+    mat = toks[0][None, :].copy()
+    h_out = np.zeros((1, wl.gen_tokens), dtype=np.int32); h_len = np.zeros(1, dtype=np.int32)
+    bt = torch.from_numpy(np.pad(table, ((0, 0), (0, g.cfg.max_blocks_per_seq - table.shape[1])), constant_values=-1)).to(g.dev)
+    g.generate_host(sg, bt, mat, np.array([mat.shape[1]], dtype=np.int32), wl.gen_tokens, h_out, h_len)
+    assert np.array_equal(h_out[0], got) and h_len[0] == wl.gen_tokens
+
+
+def test_c1_lockstep_full():
+    wl = W.workload("C1")
+    w, model, tpl, g, table = _setup(wl, 40, [0])
+    states, _ = _prefill_both(wl, g, table, model, [0])
+    so, sg = _sampling(wl)
+    rep = lockstep(g, table, model, states, tpl, so, sg, 40, "fp32", oracle_mode="memo", check_attn=True)
+    assert rep.max_logit_err <= 1e-4 and rep.accept_checked >= 35
+    g.check()
+
+
+def test_c2_lockstep_sampled_iterations():
+    """BASELINE config 2 (12 layers, d 1024, 64-node tree, tau 3, T 1.0): prefill of the
+    325-token prefix and the first iterations in lockstep."""
+    wl = W.workload("C2")
+    w, model, tpl, g, table = _setup(wl, 4, [0])
+    states, _ = _prefill_both(wl, g, table, model, [0])
+    so, sg = _sampling(wl)
+    rep = lockstep(g, table, model, states, tpl, so, sg, 4, "bf16", oracle_mode="tree", check_attn=True)
+    assert rep.iterations == 4
+    g.check()
+
+
+def test_c3_batch16_vocab2049_sampled_sequences():
+    """BASELINE config 3 (batch 16, vocab 2049, 42-node tree, tau 5, T 0.8): all sequences
+    run on the GPU, the oracle follows two of them."""
+    wl = W.workload("C3")
+    w, model, tpl, g, table = _setup(wl, 3, [0, 9])
+    states, _ = _prefill_both(wl, g, table, model, [0, 9])
+    so, sg = _sampling(wl)
+    rep = lockstep(g, table, model, states, tpl, so, sg, 3, "bf16", oracle_mode="tree")
+    assert rep.iterations == 3
+    g.check()
+
+
+def _random_context(model, S, rng, scale=1.0):
+    K = O.round_bf16(rng.standard_normal((model.L, S, model.H, model.dh)) * scale)
+    V = O.round_bf16(rng.standard_normal((model.L, S, model.H, model.dh)) * scale)
+    return K, V
+
+
+@pytest.mark.parametrize("name", ["C4", "C5"])
+def test_long_ragged_contexts_with_injected_kv(name):
+    """BASELINE configs 4 and 5 at full batch and context lengths: the KV cache holds
+    seeded random bf16 rows (so no prefill is needed on either side), tree tokens and the
+    carried state are random; the oracle scores three sampled sequences (shortest, longest,
+    one other).  C5 uses a random topology per sequence."""
+    torch = _torch()
+    wl = W.workload(name)
+    w = W.make_weights(wl.shape, wl.seed())
+    model = O.Model.from_shape(wl.shape, w)
+    B, N = wl.batch, wl.tree_nodes
+    lens = W.ragged_lengths(B, wl.context_len[0], wl.context_len[1], wl.seed(900))
+    g, table = make_gpu(wl.shape, w, B, N, [int(s) + N + 8 for s in lens], wl.seed(1))
+    g.begin(table, ctx_len=lens)
+    if wl.random_topology:
+        tpls = [W.random_topology(N, wl.topology_max_depth, wl.seed(100 + b)) for b in range(B)]
+        g.set_tree(np.stack([t.parent for t in tpls]), np.stack([t.rank for t in tpls]), per_sequence=True)
+    else:
+        tpls = [W.static_template(N, wl.tree_caps)] * B
+        g.set_tree(tpls[0].parent, tpls[0].rank)
+    order = np.argsort(lens)
+    picks = [int(order[0]), int(order[-1]), int(order[B // 2])]
+    rng = np.random.default_rng(wl.seed(2))
+    # every sequence gets random K/V on the GPU; the sampled ones also in the oracle
+    view = g.kv_view()
+    view.normal_()                                           # all pages: seeded below for the sampled ones
+    states = {}
+    for b in picks:
+        K, V = _random_context(model, int(lens[b]), rng)
+        inject_kv(g, table, b, K, V)
+        kv = O.KVCache(model, capacity=int(lens[b]) + 80)
+        kv.extend(K, V)
+        states[b] = kv
+    toks = rng.integers(0, wl.shape.vocab - 1, size=(B, N)).astype(np.int32)
+    logits = torch.zeros(B, N, wl.shape.vocab, dtype=torch.float32, device=g.dev)
+    attn = torch.zeros(model.L, B, N, model.d, dtype=g.tdtype, device=g.dev)
+    g.verify_step(override=torch.from_numpy(toks).to(g.dev), logits_out=logits, attn_tap=attn)
+    so, sg = _sampling(wl, seed=5)
+    acc = torch.zeros(B, dtype=torch.int32, device=g.dev)
+    pn = torch.zeros(B, 16, dtype=torch.int32, device=g.dev)
+    sl = torch.zeros(B, 16, dtype=torch.int64, device=g.dev)
+    eb = torch.zeros(B, dtype=torch.int64, device=g.dev)
+    g.accept_and_commit(sg, accept_len=acc, path_nodes=pn, kv_slots=sl, edge_bits=eb)
+    lg = logits.cpu().numpy().astype(np.float64)
+    at = attn.float().cpu().numpy().astype(np.float64)
+    for b in picks:
+        tpl = tpls[b]
+        mask = np.zeros((N, N), dtype=bool)
+        for n in range(N):
+            mask[n, tpl.node_path(n)] = True
+        S = int(lens[b])
+        out = O.forward_tree(model, states[b], [0] * N, toks[b], S + tpl.depth, mask)
+        e_l = np.abs(lg[b] - out.logits).max()
+        e_a = max(np.abs(at[l, b] - out.attn[l]).max() for l in range(model.L))
+        print(f"{name} seq {b} (context {int(lens[b])}): max |logit err| {e_l:.2e}, max |attn err| {e_a:.2e}")
+        assert e_l <= TOL["bf16"] and e_a <= TOL["bf16"]
+        # accept decision of the oracle on its own logits
+        draws = {n: O.draws_at(model, out.logits[n], so, b, S + int(tpl.depth[n]) + 1) for n in range(N)}
+        ok = O.tree_edge_accepts(tpl.parent, toks[b], draws)
+        best, path = O.accept_from_edges(tpl.parent, tpl.depth, ok)
+        margin = min(O.decode._edge_margin(model, out.logits[int(tpl.parent[n])], so, b,
+                                           S + int(tpl.depth[int(tpl.parent[n])]) + 1, int(toks[b, n]))
+                     for n in range(1, N))
+        if margin > MARGINS["bf16"]:
+            assert int(acc[b]) == len(path) and list(pn[b, :len(path)].cpu().numpy()) == path
+            assert list(sl[b, :len(path)].cpu().numpy()) == expected_slots(table, b, S, len(path))
+    assert np.array_equal(g.lengths(), lens + acc.cpu().numpy())
+    g.check()
+
+
+def test_capacity_error_is_reported_not_faulted():
+    """A block table too short for context + tree: the device flags it, no access goes out
+    of bounds, and the next synchronising call returns ECAPACITY."""
+    import paper_2410_21951_b200 as P
+    torch = _torch()
+    wl = W.toy_workload(dtype="fp32", d_model=64, n_heads=2, d_ffn=128, vocab=61, tree_nodes=12, tree_caps=(4, 3, 2))
+    w = W.make_weights(wl.shape, wl.seed())
+    tpl = W.static_template(wl.tree_nodes, wl.tree_caps)
+    g, table = make_gpu(wl.shape, w, 1, wl.tree_nodes, [64], 1, spare_pages=0)      # one block only
+    g.set_tree(tpl.parent, tpl.rank)
+    g.begin(table, ctx_len=[60])                                                     # 60 + 12 nodes > 64
+    toks = torch.zeros(1, wl.tree_nodes, dtype=torch.int32, device=g.dev)
+    g.verify_step(override=toks)
+    with pytest.raises(P.VadusaError) as e:
+        g.check()
+    assert e.value.status == 4
+
+
+def test_call_order_and_argument_errors():
+    import paper_2410_21951_b200 as P
+    torch = _torch()
+    wl = W.toy_workload(dtype="fp32", d_model=64, n_heads=2, d_ffn=128, vocab=61, tree_nodes=12, tree_caps=(4, 3, 2))
+    w = W.make_weights(wl.shape, wl.seed())
+    g, table = make_gpu(wl.shape, w, 2, wl.tree_nodes, [200, 200], 1)
+    sp = P.Sampling.make(tau=1)
+    with pytest.raises(P.VadusaError) as e:
+        g.verify_step()
+    assert e.value.status == 5                              # no batch begun
+    g.begin(table)
+    with pytest.raises(P.VadusaError) as e:
+        g.draft(sp)
+    assert e.value.status == 5                              # no tree
+    bad_parent = np.array([-1, 0, 0, 5], dtype=np.int32)    # node 3's parent does not precede it
+    with pytest.raises(P.VadusaError) as e:
+        g.set_tree(bad_parent, np.zeros(4, dtype=np.int32))
+    assert e.value.status == 1
+    tpl = W.static_template(wl.tree_nodes, wl.tree_caps)
+    with pytest.raises(P.VadusaError):                      # siblings out of rank order
+        g.set_tree(tpl.parent, tpl.rank[::-1].copy())
+    g.set_tree(tpl.parent, tpl.rank)
+    with pytest.raises(P.VadusaError) as e:
+        g.verify_step()
+    assert e.value.status == 5                              # no draft, no override
+    with pytest.raises(P.VadusaError) as e:
+        g.accept_and_commit(sp)
+    assert e.value.status == 5
+    with pytest.raises(P.VadusaError) as e:
+        g.draft(P.Sampling.make(tau=0))
+    assert e.value.status == 1
