@@ -3,12 +3,17 @@
 #include <cuda_runtime.h>
 #include <stdarg.h>
 
+#include <type_traits>
+
+#include <map>
 #include <new>
+#include <tuple>
 
 #include "accept.cuh"
 #include "attention_simt.cuh"
 #include "elementwise.cuh"
 #include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
 #include "layout.h"
 #include "select.cuh"
 
@@ -40,6 +45,10 @@ struct vadusa_ctx {
   cudaEvent_t ev0 = nullptr, ev1 = nullptr, ev_poll = nullptr;
   int32_t* h_pinned = nullptr;     // [2]: done_count, err
   char err[512] = {0};
+  // TMA descriptors of the operands of the tensor-core products, made on first use
+  typedef std::tuple<const void*, int, int, int, int, long long> MapKey;   // ptr, rows, K, box rows, batches, batch stride
+  std::map<MapKey, CUtensorMap> maps;
+  void* encode_fn = nullptr;       // cuTensorMapEncodeTiled, resolved through the runtime
   // per-kernel timing (vadusa_profile_begin/end): one event pair per launch
   struct ProfRec { cudaEvent_t a, b; int cls; };
   bool prof_on = false, prof_pending = false;
@@ -199,6 +208,92 @@ vadusa_status gemm(vadusa_ctx* ctx, int cls, const T* A, const T* W, int M, int 
   return VADUSA_OK;
 }
 
+// ---- tensor-core products (bf16 models) ------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Descriptor of a row-major bf16 matrix [batches][rows][K] read in boxes of box_rows x 64
+// elements with the 128-byte swizzle; rows outside the matrix read as zero.
+vadusa_status tensor_map(vadusa_ctx* ctx, const void* ptr, int rows, int K, int box_rows, int batches,
+                         long long batch_stride_elems, const CUtensorMap** out) {
+  vadusa_ctx::MapKey key(ptr, rows, K, box_rows, batches, batch_stride_elems);
+  auto it = ctx->maps.find(key);
+  if (it == ctx->maps.end()) {
+    if (!ctx->encode_fn) return fail(ctx, VADUSA_ECUDA, "cuTensorMapEncodeTiled is not available");
+    CUtensorMap m;
+    cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)batches};
+    cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)(batches > 1 ? batch_stride_elems : (long long)rows * K) * 2};
+    cuuint32_t box[3] = {(cuuint32_t)kGemmBK, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_fn)(
+        &m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(ctx, VADUSA_ECUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    it = ctx->maps.emplace(key, m).first;
+  }
+  *out = &it->second;
+  return VADUSA_OK;
+}
+
+template <int TN, typename Epi>
+vadusa_status launch_gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void* W, int w_rows, int M, int N, int K,
+                             int batches, long long x_z, long long w_z, int ksplit, const Epi& epi) {
+  using Cfg = GemmTcCfg<TN>;
+  static bool attr_done = false;
+  if (!attr_done) {
+    CU(cudaFuncSetAttribute(gemm_tc_kernel<TN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
+    attr_done = true;
+  }
+  const CUtensorMap *mw, *mx;
+  if (vadusa_status s = tensor_map(ctx, W, w_rows, K, kGemmRowsW, batches, w_z, &mw)) return s;
+  if (vadusa_status s = tensor_map(ctx, X, M, K, TN, batches, x_z, &mx)) return s;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3((N + kGemmRowsW - 1) / kGemmRowsW, (M + TN - 1) / TN, batches * ksplit);
+  lc.blockDim = dim3(128);
+  lc.dynamicSmemBytes = Cfg::kSmemBytes;
+  lc.stream = ctx->stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = ksplit;
+  lc.attrs = at; lc.numAttrs = 1;
+  PROF(ctx, cls);
+  CU(cudaLaunchKernelEx(&lc, gemm_tc_kernel<TN, Epi>, *mw, *mx, M, N, K / kGemmBK / ksplit, ksplit, epi, err_word(ctx)));
+  LAUNCH_CHECK();
+  return VADUSA_OK;
+}
+
+// Tile width by token count; K split so that about one CTA per SM streams weights.
+template <typename Epi>
+vadusa_status gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void* W, int w_rows, int M, int N, int K,
+                      int batches, long long x_z, long long w_z, const Epi& epi) {
+  const int tn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 1024 ? 128 : 256;
+  const int tiles = ((N + kGemmRowsW - 1) / kGemmRowsW) * ((M + tn - 1) / tn) * batches;
+  const int chunks = K / kGemmBK;
+  int ksplit = 1;
+  while (ksplit < 8 && tiles * ksplit < 148 && chunks % (ksplit * 2) == 0 && ksplit * 2 <= tn) ksplit *= 2;
+  switch (tn) {
+    case 16: return launch_gemm_tc<16>(ctx, cls, X, W, w_rows, M, N, K, batches, x_z, w_z, ksplit, epi);
+    case 32: return launch_gemm_tc<32>(ctx, cls, X, W, w_rows, M, N, K, batches, x_z, w_z, ksplit, epi);
+    case 64: return launch_gemm_tc<64>(ctx, cls, X, W, w_rows, M, N, K, batches, x_z, w_z, ksplit, epi);
+    case 128: return launch_gemm_tc<128>(ctx, cls, X, W, w_rows, M, N, K, batches, x_z, w_z, ksplit, epi);
+    default: return launch_gemm_tc<256>(ctx, cls, X, W, w_rows, M, N, K, batches, x_z, w_z, ksplit, epi);
+  }
+}
+
+// Product dispatch by model type: fp32 models use plain FMA arithmetic, bf16 models the
+// tensor cores (K must be a multiple of 64 there, else the FMA kernel serves).
+template <typename T, typename Epi>
+vadusa_status product(vadusa_ctx* ctx, int cls, const T* X, const T* W, int w_rows, int M, int N, int K, int batches,
+                      long long x_z, long long w_z, const Epi& epi) {
+  if constexpr (std::is_same<T, bf16>::value) {
+    if (K % kGemmBK == 0) return gemm_tc(ctx, cls, X, W, w_rows, M, N, K, batches, x_z, w_z, epi);
+  }
+  return gemm<T>(ctx, cls, X, W, M, N, K, batches, x_z, w_z, epi);
+}
+
 template <typename T>
 vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeView& tv, T* out) {
   const vadusa_config& c = ctx->cfg;
@@ -249,22 +344,23 @@ vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* overri
     layernorm_kernel<T><<<ln_blocks, 128, 0, ctx->stream>>>(x, w.ln1_g, w.ln1_b, a, M, d, c.ln_eps);
     LAUNCH_CHECK();
     EpiQKV<T> eq{w.bqkv, q, pool, ctx->block_table, ctx_len, nvalid, err_word(ctx), g, N, d};
-    vadusa_status s = gemm<T>(ctx, K_GEMM_QKV, a, as<T>(w.wqkv), M, 3 * d, d, 1, 0, 0, eq);
+    vadusa_status s = product<T>(ctx, K_GEMM_QKV, a, as<T>(w.wqkv), 3 * d, M, 3 * d, d, 1, 0, 0, eq);
     if (s) return s;
-    T* o_dst = attn_tap ? attn_tap + (long long)l * M * d : o;
-    s = attention<T>(ctx, q, pool, tv, o_dst);
+    s = attention<T>(ctx, q, pool, tv, o);
     if (s) return s;
+    if (attn_tap)
+      CU(cudaMemcpyAsync(attn_tap + (long long)l * M * d, o, (size_t)M * d * sizeof(T), cudaMemcpyDeviceToDevice, ctx->stream));
     EpiResidual eo{w.bo, x, d};
-    s = gemm<T>(ctx, K_GEMM_OUT, o_dst, as<T>(w.wo), M, d, d, 1, 0, 0, eo);
+    s = product<T>(ctx, K_GEMM_OUT, o, as<T>(w.wo), d, M, d, d, 1, 0, 0, eo);
     if (s) return s;
     PROF(ctx, K_LAYERNORM);
     layernorm_kernel<T><<<ln_blocks, 128, 0, ctx->stream>>>(x, w.ln2_g, w.ln2_b, a, M, d, c.ln_eps);
     LAUNCH_CHECK();
     EpiRelu<T> e1{w.b1, mid, f};
-    s = gemm<T>(ctx, K_GEMM_FFN1, a, as<T>(w.w1), M, f, d, 1, 0, 0, e1);
+    s = product<T>(ctx, K_GEMM_FFN1, a, as<T>(w.w1), f, M, f, d, 1, 0, 0, e1);
     if (s) return s;
     EpiResidual e2{w.b2, x, d};
-    s = gemm<T>(ctx, K_GEMM_FFN2, mid, as<T>(w.w2), M, d, f, 1, 0, 0, e2);
+    s = product<T>(ctx, K_GEMM_FFN2, mid, as<T>(w.w2), d, M, d, f, 1, 0, 0, e2);
     if (s) return s;
   }
   PROF(ctx, K_LAYERNORM);
@@ -272,7 +368,7 @@ vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* overri
                                                           hfinal, M, d, c.ln_eps);
   LAUNCH_CHECK();
   EpiLogits el{logits, vp, 0};
-  return gemm<T>(ctx, K_GEMM_LM, hfinal, as<T>(ctx->lm), M, vp, d, 1, 0, 0, el);
+  return product<T>(ctx, K_GEMM_LM, hfinal, as<T>(ctx->lm), vp, M, vp, d, 1, 0, 0, el);
 }
 
 template <typename T>
@@ -283,11 +379,12 @@ vadusa_status draft(vadusa_ctx* ctx, const SamplingDev& sp) {
   T* z = wsptr<T>(ctx, ctx->ws.z);
   float* dl = wsptr<float>(ctx, ctx->ws.dlogits);
   const long long w_stride = ctx->dw_stride / (long long)sizeof(T), u_stride = ctx->du_stride / (long long)sizeof(T);
-  EpiDraftHidden<T> eh{ctx->db, hstar, z, d, B};
-  vadusa_status s = gemm<T>(ctx, K_DRAFT_HIDDEN, hstar, as<T>(ctx->dw), B, d, d, hd, 0, w_stride, eh);
+  if (hd > 1 && w_stride != (long long)d * d) return fail(ctx, VADUSA_EINVAL, "draft matrices are not contiguous");
+  EpiDraftHiddenFlat<T> eh{ctx->db, hstar, z, d, B};
+  vadusa_status s = product<T>(ctx, K_DRAFT_HIDDEN, hstar, as<T>(ctx->dw), hd * d, B, hd * d, d, 1, 0, 0, eh);
   if (s) return s;
   EpiLogits el{dl, vp, (long long)B * vp};
-  s = gemm<T>(ctx, K_DRAFT_LOGITS, z, as<T>(ctx->du), B, vp, d, hd, (long long)B * d, u_stride, el);
+  s = product<T>(ctx, K_DRAFT_LOGITS, z, as<T>(ctx->du), vp, B, vp, d, hd, (long long)B * d, u_stride, el);
   if (s) return s;
   dim3 grid(hd + 1, B);
   PROF(ctx, K_DRAFT_SELECT);
@@ -472,6 +569,15 @@ vadusa_status vadusa_init(const vadusa_weights* weights, const vadusa_config* cf
   ctx->wsp = reinterpret_cast<char*>(cfg->workspace);
   ctx->stream = reinterpret_cast<cudaStream_t>(cfg->stream);
   resolve_weights(ctx);
+  {
+    cudaDriverEntryPointQueryResult qres;
+    void* fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      ctx->encode_fn = fn;
+    else
+      cudaGetLastError();
+  }
   if (vadusa_status s = set_kernel_attributes(ctx)) return s;
   CU(cudaEventCreate(&ctx->ev0));
   CU(cudaEventCreate(&ctx->ev1));

@@ -80,6 +80,21 @@ struct EpiDraftHidden {
   }
 };
 
+// the same with the heads' matrices stacked along the feature axis: n = head * d + column
+template <typename T>
+struct EpiDraftHiddenFlat {
+  const float* bias;     // [heads * d]
+  const T* h;            // [batch][d]
+  T* out;                // [heads][batch][d]
+  int d, batch;
+  __device__ __forceinline__ void operator()(int, int m, int n, float acc) const {
+    const int head = n / d, col = n - head * d;
+    const float t = acc + bias[n];
+    const float s = t / (1.0f + expf(-t));
+    out[((long long)head * batch + m) * d + col] = from_f<T>(to_f<T>(h[(long long)m * d + col]) + s);
+  }
+};
+
 // ---- kernel -----------------------------------------------------------------------
 // 64x64 tile, K step 16, 256 threads, 4x4 outputs per thread.  K must be a multiple of 16.
 // grid = (ceil(N/64), ceil(M/64), batches); A and W advance by a_z / w_z elements per batch.

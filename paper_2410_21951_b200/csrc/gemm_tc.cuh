@@ -1,0 +1,149 @@
+// bf16 projections on the 5th-generation tensor cores (tcgen05.mma, TMEM accumulator,
+// TMA-staged operands):  C[m, n] = sum_k X[m, k] * W[n, k], fp32 accumulation.
+//
+// The weight tile is the MMA's 128-row operand (A) and the token tile its narrow operand
+// (B, TN = 16..256 tokens), so with few tokens (batch 1: 64 tree nodes) a CTA still streams
+// a full 128 x 64 weight tile per MMA group and the kernel is bound by weight streaming.
+// The accumulator D[128 features][TN tokens] lives in tensor memory: lane = feature.
+//
+// Work split: grid.x = feature tiles of 128, grid.y = token tiles of TN, grid.z = batch *
+// ksplit.  With ksplit > 1 the CTAs of one cluster (1,1,ksplit) each take a K slice, park
+// their partial tile in shared memory, and reduce it over distributed shared memory in a
+// fixed order (deterministic), each CTA finishing TN/ksplit tokens of the tile.
+//
+// Warp roles (128 threads): warp 0 lane 0 issues TMA loads into a ring of stages, warp 1
+// owns the TMEM allocation and its lane 0 issues the MMAs, all four warps run the epilogue.
+// Weight tiles of the first stages are requested before griddepcontrol.wait, so under
+// programmatic dependent launch they stream while the producer of X is still running.
+#pragma once
+#include "tc.cuh"
+
+namespace vadusa {
+
+constexpr int kGemmBK = 64;                 // K elements per stage (128 bytes per row: one swizzle row)
+constexpr int kGemmRowsW = 128;             // weight rows per tile
+constexpr int kGemmSmemBudget = 196 * 1024;
+
+template <int TN> struct GemmTcCfg {
+  static constexpr int kStageBytes = kGemmRowsW * kGemmBK * 2 + TN * kGemmBK * 2;
+  static constexpr int kStagesMax = kGemmSmemBudget / kStageBytes;
+  static constexpr int kStages = kStagesMax > 8 ? 8 : kStagesMax;
+  static constexpr int kTmemCols = TN < 32 ? 32 : TN;
+  static constexpr int kRingBytes = kStages * kStageBytes;
+  static constexpr int kSmemBytes = kRingBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+template <int TN, typename Epi>
+__global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW,
+                                                      const __grid_constant__ CUtensorMap tmX, int M, int N,
+                                                      int chunks_per_split, int ksplit, Epi epi, uint32_t* err) {
+  using Cfg = GemmTcCfg<TN>;
+  constexpr int S = Cfg::kStages;
+  constexpr uint32_t kWBytes = kGemmRowsW * kGemmBK * 2, kXBytes = TN * kGemmBK * 2;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* ring_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bars = base + Cfg::kRingBytes;          // full[S], empty[S], accum, tmem holder
+  const uint32_t full0 = bars, empty0 = bars + 8 * S, accum_bar = bars + 16 * S, holder = bars + 16 * S + 8;
+  volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(ring_ptr + Cfg::kRingBytes + 16 * S + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * kGemmRowsW, m0 = blockIdx.y * TN;
+  const int zb = blockIdx.z / ksplit, ks = blockIdx.z % ksplit;
+  const int chunk0 = ks * chunks_per_split, nchunks = chunks_per_split;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    mbar_init(accum_bar, 1);
+    mbar_fence_init();
+    tma_prefetch_desc(&tmW);
+    tma_prefetch_desc(&tmX);
+  }
+  if (warp == 1) { tmem_alloc(holder, Cfg::kTmemCols); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *holder_ptr;
+
+  if (warp == 0 && lane == 0) {
+    // ---- TMA producer
+    const int pre = nchunks < S ? nchunks : S;
+    for (int i = 0; i < pre; ++i) {                      // weights do not depend on the upstream kernel
+      mbar_expect_tx(full0 + 8 * i, kWBytes + kXBytes);
+      tma_load_3d(base + i * Cfg::kStageBytes, &tmW, full0 + 8 * i, (chunk0 + i) * kGemmBK, n0, zb);
+    }
+    grid_dep_wait();
+    for (int i = 0; i < pre; ++i)
+      tma_load_3d(base + i * Cfg::kStageBytes + kWBytes, &tmX, full0 + 8 * i, (chunk0 + i) * kGemmBK, m0, zb);
+    for (int i = pre; i < nchunks; ++i) {
+      const int s = i % S;
+      if (!mbar_wait(empty0 + 8 * s, ((i / S) - 1) & 1, err)) break;
+      mbar_expect_tx(full0 + 8 * s, kWBytes + kXBytes);
+      tma_load_3d(base + s * Cfg::kStageBytes, &tmW, full0 + 8 * s, (chunk0 + i) * kGemmBK, n0, zb);
+      tma_load_3d(base + s * Cfg::kStageBytes + kWBytes, &tmX, full0 + 8 * s, (chunk0 + i) * kGemmBK, m0, zb);
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---- MMA issuer
+    constexpr uint32_t idesc = umma_idesc_bf16(kGemmRowsW, TN < 16 ? 16 : TN);
+    for (int i = 0; i < nchunks; ++i) {
+      const int s = i % S;
+      if (!mbar_wait(full0 + 8 * s, (i / S) & 1, err)) break;
+      tc_fence_after();
+      const uint32_t wa = base + s * Cfg::kStageBytes, xa = wa + kWBytes;
+#pragma unroll
+      for (int k = 0; k < kGemmBK / 16; ++k)
+        umma_bf16(tmem, umma_desc_k_sw128(wa + 32 * k), umma_desc_k_sw128(xa + 32 * k), idesc, (i | k) != 0);
+      umma_commit(empty0 + 8 * s);                       // stage reusable once these MMAs have read it
+    }
+    umma_commit(accum_bar);                              // accumulator complete
+  }
+  __syncwarp();
+  // every thread (grid_dep_wait must precede any global access of upstream-produced data)
+  grid_dep_wait();
+  mbar_wait(accum_bar, 0, err);
+  tc_fence_after();
+  grid_dep_launch();
+
+  // ---- epilogue: warp w reads TMEM lanes 32w .. 32w+31 (features n0 + 32w + lane)
+  const int n = n0 + 32 * warp + lane;
+  const uint32_t trow = tmem + ((uint32_t)(32 * warp) << 16);
+  if (ksplit == 1) {
+    constexpr int CH = TN < 32 ? 16 : 32;
+#pragma unroll 1
+    for (int c0 = 0; c0 < TN; c0 += CH) {
+      float v[CH];
+      if (CH == 32) tmem_ld32(trow + c0, v); else tmem_ld16(trow + c0, v);
+      if (n < N) {
+#pragma unroll
+        for (int j = 0; j < CH; ++j)
+          if (m0 + c0 + j < M) epi(zb, m0 + c0 + j, n, v[j]);
+      }
+    }
+  } else {
+    // park the partial tile as P[token][feature] (the ring is idle: all MMAs have completed)
+    float* P = reinterpret_cast<float*>(ring_ptr);
+    constexpr int CH = TN < 32 ? 16 : 32;
+#pragma unroll 1
+    for (int c0 = 0; c0 < TN; c0 += CH) {
+      float v[CH];
+      if (CH == 32) tmem_ld32(trow + c0, v); else tmem_ld16(trow + c0, v);
+#pragma unroll
+      for (int j = 0; j < CH; ++j) P[(c0 + j) * kGemmRowsW + threadIdx.x] = v[j];
+    }
+    cluster_sync_all();
+    const int per = TN / ksplit;
+    const int nn = n0 + threadIdx.x;
+    for (int t = ks * per; t < (ks + 1) * per; ++t) {
+      float acc = 0.f;
+      const uint32_t a = base + (uint32_t)(t * kGemmRowsW + threadIdx.x) * 4u;
+      for (int peer = 0; peer < ksplit; ++peer) acc += ld_peer_f32(a, peer);
+      if (nn < N && m0 + t < M) epi(zb, m0 + t, nn, acc);
+    }
+    cluster_sync_all();                                  // peers may still be reading this CTA's tile
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, Cfg::kTmemCols);
+}
+
+}  // namespace vadusa
