@@ -11,6 +11,7 @@
 
 #include "accept.cuh"
 #include "attention_simt.cuh"
+#include "attention_tc.cuh"
 #include "elementwise.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
@@ -310,6 +311,37 @@ vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeVi
     LAUNCH_CHECK();
     return VADUSA_OK;
   };
+  if constexpr (std::is_same<T, bf16>::value) {
+    if (dh == 64) {
+      // tensor-core kernel; KV splits so that about two CTAs per SM exist even at batch 1
+      int splits = 1;
+      while (splits < 8 && c.n_heads * ctx->batch * splits * 2 <= 296) splits *= 2;
+      const CUtensorMap *mq, *mkv;
+      const int M = ctx->batch * tv.n_nodes;
+      if (vadusa_status s = tensor_map(ctx, q, M, c.d_model, 64, 1, 0, &mq)) return s;
+      const long long rows = (long long)c.kv_num_blocks * 2 * c.n_heads * kKvBlock;
+      if (rows > 0x7fffffffLL) return fail(ctx, VADUSA_EINVAL, "KV pool too large for one tensor map");
+      if (vadusa_status s = tensor_map(ctx, c.kv_pool, (int)rows, 64, 64, c.n_layers, g.layer_stride, &mkv)) return s;
+      const int layer = (int)((reinterpret_cast<const char*>(pool) - reinterpret_cast<const char*>(c.kv_pool)) /
+                              (g.layer_stride * (long long)sizeof(bf16)));
+      cudaLaunchConfig_t lc = {};
+      lc.gridDim = dim3(c.n_heads, ctx->batch, splits);
+      lc.blockDim = dim3(128);
+      lc.dynamicSmemBytes = kAttSmemBytes;
+      lc.stream = ctx->stream;
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = splits;
+      lc.attrs = at; lc.numAttrs = 1;
+      PROF(ctx, K_ATTENTION);
+      CU(cudaLaunchKernelEx(&lc, tree_attention_tc_kernel, *mq, *mkv, layer, ctx->block_table,
+                            (const int32_t*)wsptr<int32_t>(ctx, ctx->ws.ctx_len),
+                            (const int32_t*)wsptr<int32_t>(ctx, ctx->ws.nvalid), tv, g, c.d_model,
+                            scale * 1.4426950408889634f, splits, reinterpret_cast<bf16*>(out), err_word(ctx)));
+      LAUNCH_CHECK();
+      return VADUSA_OK;
+    }
+  }
   if (dh == 64) return go(tree_attention_simt_kernel<T, 64>);
   return go(tree_attention_simt_kernel<T, 32>);
 }
@@ -329,7 +361,6 @@ vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* overri
   float* logits = wsptr<float>(ctx, ctx->ws.logits);
   int32_t* ctx_len = wsptr<int32_t>(ctx, ctx->ws.ctx_len);
   int32_t* nvalid = wsptr<int32_t>(ctx, ctx->ws.nvalid);
-  const int ln_blocks = (M + 3) / 4;
 
   PROF(ctx, K_EMBED);
   tree_embed_kernel<T><<<M, 128, 0, ctx->stream>>>(
@@ -341,7 +372,7 @@ vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* overri
     const LayerW& w = ctx->layers[l];
     T* pool = reinterpret_cast<T*>(c.kv_pool) + (long long)l * g.layer_stride;
     PROF(ctx, K_LAYERNORM);
-    layernorm_kernel<T><<<ln_blocks, 128, 0, ctx->stream>>>(x, w.ln1_g, w.ln1_b, a, M, d, c.ln_eps);
+    layernorm_kernel<T><<<M, 256, 0, ctx->stream>>>(x, w.ln1_g, w.ln1_b, a, M, d, c.ln_eps);
     LAUNCH_CHECK();
     EpiQKV<T> eq{w.bqkv, q, pool, ctx->block_table, ctx_len, nvalid, err_word(ctx), g, N, d};
     vadusa_status s = product<T>(ctx, K_GEMM_QKV, a, as<T>(w.wqkv), 3 * d, M, 3 * d, d, 1, 0, 0, eq);
@@ -354,7 +385,7 @@ vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* overri
     s = product<T>(ctx, K_GEMM_OUT, o, as<T>(w.wo), d, M, d, d, 1, 0, 0, eo);
     if (s) return s;
     PROF(ctx, K_LAYERNORM);
-    layernorm_kernel<T><<<ln_blocks, 128, 0, ctx->stream>>>(x, w.ln2_g, w.ln2_b, a, M, d, c.ln_eps);
+    layernorm_kernel<T><<<M, 256, 0, ctx->stream>>>(x, w.ln2_g, w.ln2_b, a, M, d, c.ln_eps);
     LAUNCH_CHECK();
     EpiRelu<T> e1{w.b1, mid, f};
     s = product<T>(ctx, K_GEMM_FFN1, a, as<T>(w.w1), f, M, f, d, 1, 0, 0, e1);
@@ -364,7 +395,7 @@ vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* overri
     if (s) return s;
   }
   PROF(ctx, K_LAYERNORM);
-  layernorm_kernel<T><<<ln_blocks, 128, 0, ctx->stream>>>(x, ctx->lnf_g, ctx->lnf_b,
+  layernorm_kernel<T><<<M, 256, 0, ctx->stream>>>(x, ctx->lnf_g, ctx->lnf_b,
                                                           hfinal, M, d, c.ln_eps);
   LAUNCH_CHECK();
   EpiLogits el{logits, vp, 0};
@@ -463,6 +494,7 @@ vadusa_status set_kernel_attributes(vadusa_ctx* ctx) {
   CU(cudaFuncSetAttribute(tree_attention_simt_kernel<float, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(32)));
   CU(cudaFuncSetAttribute(tree_attention_simt_kernel<bf16, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(64)));
   CU(cudaFuncSetAttribute(tree_attention_simt_kernel<bf16, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(32)));
+  CU(cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmemBytes));
   return VADUSA_OK;
 }
 

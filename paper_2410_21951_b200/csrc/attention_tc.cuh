@@ -1,0 +1,281 @@
+// Tree-masked decode attention over the paged bf16 KV cache on the tcgen05 tensor cores
+// (head_dim 64).  Node n of sequence b attends to every cached position < ctx_len[b] and to
+// the tree slots ctx_len[b] + m whose bit m is set in anc[n] (paper Sec. II-A, tree attention).
+//
+// One CTA per (head, sequence, KV split); the splits of one (head, sequence) form a cluster.
+// Per 64-key page:  TMA brings the page's K and V tiles (8 KB each, 128-byte swizzle);
+//   S = Q K^T      tcgen05.mma, A = Q tile (rows 64..127 zero), B = K tile, D in TMEM cols 0..63
+//   softmax        one thread per node row reads its 64 scores from TMEM, keeps the running
+//                  max / sum, and writes the weights back to TMEM as two bf16 halves
+//                  (p = hi + lo, 16 significant bits) over the score columns
+//   O_tile = P V   tcgen05.mma with A from TMEM (hi then lo), B = V tile (MN-major), D in cols 64..127
+//   the row's thread folds O_tile into its fp32 register accumulator while the next page runs.
+// Splits are merged over distributed shared memory in a fixed order.
+// Warps: 0-1 softmax rows, warp 2 lane 0 TMA producer, warp 3 TMEM owner and MMA issuer.
+#pragma once
+#include "tc.cuh"
+
+namespace vadusa {
+
+constexpr int kAttStages = 3;
+constexpr int kAttTileBytes = 64 * 64 * 2;                                   // one K or V page tile
+constexpr int kAttSmemBytes = 2 * kAttTileBytes /*Q, 128 rows*/ + kAttStages * 2 * kAttTileBytes + 1024 + 256;
+
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// D[tmem] (+)= A[tmem] * B[smem] for one K step of 16 elements (A: lane = row, 8 columns of bf16 pairs).
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, bool accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"((uint32_t)accumulate)
+      : "memory");
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
+}
+
+__global__ void __launch_bounds__(128) tree_attention_tc_kernel(
+    const __grid_constant__ CUtensorMap tmQ,    // q [1][batch * n_nodes][d_model], box 64 x 64
+    const __grid_constant__ CUtensorMap tmKV,   // pool [layers][blocks * 2 * heads * 64][64], box 64 x 64
+    int layer, const int32_t* __restrict__ block_table, const int32_t* __restrict__ ctx_len,
+    const int32_t* __restrict__ nvalid, TreeView tree, KvGeom geom, int d_model, float scale_log2e, int splits,
+    bf16* __restrict__ out, uint32_t* err) {
+  constexpr int S = kAttStages;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t q_addr = base, ring = base + 2 * kAttTileBytes;
+  uint8_t* ring_ptr = base_ptr + 2 * kAttTileBytes;
+  const uint32_t bars = ring + S * 2 * kAttTileBytes;
+  const uint32_t full0 = bars, empty0 = bars + 8 * S, bar_q = bars + 16 * S, bar_s = bar_q + 8, bar_p = bar_q + 16,
+                 bar_o = bar_q + 24, holder = bar_q + 32;
+  volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(ring_ptr + S * 2 * kAttTileBytes + 16 * S + 32);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int h = blockIdx.x, b = blockIdx.y, split = blockIdx.z;
+  const int N = tree.n_nodes;
+
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    mbar_init(bar_q, 1); mbar_init(bar_s, 1); mbar_init(bar_p, 64); mbar_init(bar_o, 1);
+    mbar_fence_init();
+    tma_prefetch_desc(&tmQ);
+    tma_prefetch_desc(&tmKV);
+  }
+  {  // rows 64..127 of the Q operand are zero
+    uint4* z = reinterpret_cast<uint4*>(base_ptr + kAttTileBytes);
+    for (int i = tid; i < kAttTileBytes / 16; i += 128) z[i] = make_uint4(0, 0, 0, 0);
+    fence_proxy_async_smem();
+  }
+  if (warp == 3) { tmem_alloc(holder, 128); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *holder_ptr;
+
+  grid_dep_wait();                            // q, K/V rows, lengths come from upstream kernels
+  const int nv = nvalid[b], ctx = ctx_len[b];
+  const int total = ctx + nv;
+  const int npages = nv > 0 ? (total + kKvBlock - 1) / kKvBlock : 0;
+  const int per = (npages + splits - 1) / splits;
+  const int p0 = split * per, p1 = min(npages, p0 + per);
+  const int ntiles = max(0, p1 - p0);
+
+  float o_acc[64];
+  float m_run = -INFINITY, l_run = 0.f;
+
+  if (warp == 2 && lane == 0) {
+    // ---- TMA producer
+    if (ntiles > 0) {
+      mbar_expect_tx(bar_q, kAttTileBytes);
+      tma_load_3d(q_addr, &tmQ, bar_q, h * 64, b * N, 0);
+    }
+    for (int i = 0; i < ntiles; ++i) {
+      const int s = i % S;
+      if (i >= S && !mbar_wait(empty0 + 8 * s, ((i / S) - 1) & 1, err)) break;
+      long long blk = kv_block_of(block_table, geom, b, (p0 + i) * kKvBlock, err);
+      if (blk < 0) blk = 0;                   // flagged; stay inside the pool
+      const int row = (int)((blk * 2 * geom.n_heads + h) * kKvBlock);
+      mbar_expect_tx(full0 + 8 * s, 2 * kAttTileBytes);
+      tma_load_3d(ring + s * 2 * kAttTileBytes, &tmKV, full0 + 8 * s, 0, row, layer);
+      tma_load_3d(ring + s * 2 * kAttTileBytes + kAttTileBytes, &tmKV, full0 + 8 * s, 0, row + geom.n_heads * kKvBlock, layer);
+    }
+  } else if (warp == 3 && lane == 0) {
+    // ---- MMA issuer
+    constexpr uint32_t idesc_qk = umma_idesc_bf16(128, 64);
+    constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 64) | (1u << 16);       // B (V tile) is MN-major
+    bool ok = ntiles == 0 || mbar_wait(bar_q, 0, err);
+    for (int i = 0; i < ntiles && ok; ++i) {
+      const int s = i % S;
+      if (!mbar_wait(full0 + 8 * s, (i / S) & 1, err)) break;
+      tc_fence_after();
+      const uint32_t ka = ring + s * 2 * kAttTileBytes, va = ka + kAttTileBytes;
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        umma_bf16(tmem, umma_desc_k_sw128(q_addr + 32 * k), umma_desc_k_sw128(ka + 32 * k), idesc_qk, k != 0);
+      umma_commit(bar_s);
+      if (!mbar_wait(bar_p, i & 1, err)) break;
+      tc_fence_after();
+#pragma unroll
+      for (int k = 0; k < 4; ++k)            // 16 keys per step: 8 TMEM columns of A, 16 rows (2048 bytes) of V
+        umma_bf16_ts(tmem + 64, tmem + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, k != 0);
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        umma_bf16_ts(tmem + 64, tmem + 32 + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, true);
+      umma_commit(empty0 + 8 * s);
+      umma_commit(bar_o);
+    }
+  } else if (warp < 2) {
+    // ---- softmax: thread tid owns node row tid (TMEM lane tid)
+#pragma unroll
+    for (int e = 0; e < 64; ++e) o_acc[e] = 0.f;
+    const unsigned long long amask = tid < nv ? tree.anc[tree.off(b) + tid] : 0ull;
+    const uint32_t trow = tmem + ((uint32_t)(32 * warp) << 16);
+    float corr_prev = 0.f;
+    for (int i = 0; i < ntiles; ++i) {
+      if (!mbar_wait(bar_s, i & 1, err)) break;
+      tc_fence_after();
+      float sc[64];
+      tmem_ld32(trow, sc);
+      tmem_ld32(trow + 32, sc + 32);
+      if (i > 0) {                            // fold the previous page's P V (complete: issued before this S)
+        float ot[32];
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          tmem_ld32(trow + 64 + 32 * half, ot);
+#pragma unroll
+          for (int e = 0; e < 32; ++e) o_acc[32 * half + e] = fmaf(o_acc[32 * half + e], corr_prev, ot[e]);
+        }
+      }
+      const int key0 = (p0 + i) * kKvBlock;
+      float mx = -INFINITY;
+      if (key0 + kKvBlock <= ctx) {           // whole page inside the context: every key visible
+#pragma unroll
+        for (int j = 0; j < 64; ++j) { sc[j] *= scale_log2e; mx = fmaxf(mx, sc[j]); }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 64; ++j) {
+          const int p = key0 + j;
+          const bool vis = p < ctx || (p < total && ((amask >> ((p - ctx) & 63)) & 1ull));
+          sc[j] = vis ? sc[j] * scale_log2e : -INFINITY;
+          mx = fmaxf(mx, sc[j]);
+        }
+        if (key0 + kKvBlock > total) {        // rows of V past the tree may hold anything: zero them
+          const int valid = total - key0;
+          if (tid >= valid) {
+            uint4* vr = reinterpret_cast<uint4*>(ring_ptr + (i % S) * 2 * kAttTileBytes + kAttTileBytes + tid * 128);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) vr[c] = make_uint4(0, 0, 0, 0);
+          }
+          fence_proxy_async_smem();
+        }
+      }
+      const float m_new = fmaxf(m_run, mx);
+      corr_prev = (m_run == -INFINITY) ? 0.f : exp2f(m_run - m_new);
+      float psum = 0.f;
+      uint32_t hi[32], lo[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const float pa = (m_new == -INFINITY) ? 0.f : exp2f(sc[2 * j] - m_new);
+        const float pb = (m_new == -INFINITY) ? 0.f : exp2f(sc[2 * j + 1] - m_new);
+        psum += pa + pb;
+        const bf16 ha = __float2bfloat16_rn(pa), hb = __float2bfloat16_rn(pb);
+        hi[j] = (uint32_t)__bfloat16_as_ushort(ha) | ((uint32_t)__bfloat16_as_ushort(hb) << 16);
+        lo[j] = pack_bf16(pa - __bfloat162float(ha), pb - __bfloat162float(hb));
+      }
+      l_run = l_run * corr_prev + psum;
+      m_run = m_new;
+      tmem_st32(trow, hi);
+      tmem_st32(trow + 32, lo);
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(bar_p);
+    }
+    if (ntiles > 0 && mbar_wait(bar_o, (ntiles - 1) & 1, err)) {
+      tc_fence_after();
+      float ot[32];
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        tmem_ld32(trow + 64 + 32 * half, ot);
+#pragma unroll
+        for (int e = 0; e < 32; ++e) o_acc[32 * half + e] = fmaf(o_acc[32 * half + e], corr_prev, ot[e]);
+      }
+    }
+  }
+  __syncwarp();
+  grid_dep_launch();
+
+  // ---- output
+  if (splits == 1) {
+    if (warp < 2 && tid < N) {
+      const float inv = (tid < nv && l_run > 0.f) ? 1.f / l_run : 0.f;
+      uint4* dst = reinterpret_cast<uint4*>(out + ((long long)b * N + tid) * d_model + h * 64);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        uint4 v;
+        v.x = pack_bf16(o_acc[8 * c + 0] * inv, o_acc[8 * c + 1] * inv);
+        v.y = pack_bf16(o_acc[8 * c + 2] * inv, o_acc[8 * c + 3] * inv);
+        v.z = pack_bf16(o_acc[8 * c + 4] * inv, o_acc[8 * c + 5] * inv);
+        v.w = pack_bf16(o_acc[8 * c + 6] * inv, o_acc[8 * c + 7] * inv);
+        dst[c] = v;
+      }
+    }
+  } else {
+    // partial results to shared memory: O[64 nodes][64] fp32, then m[64], l[64] (the ring is idle)
+    __syncthreads();
+    float* Op = reinterpret_cast<float*>(ring_ptr);
+    float* mp = Op + 64 * 64;
+    float* lp = mp + 64;
+    if (warp < 2) {
+#pragma unroll
+      for (int e = 0; e < 64; ++e) Op[tid * 64 + ((e + tid) & 63)] = o_acc[e];   // skewed: conflict-free
+      mp[tid] = m_run;
+      lp[tid] = l_run;
+    }
+    cluster_sync_all();
+    const int per_n = 64 / splits;
+    const int e = tid & 63;
+    for (int n = split * per_n + (tid >> 6); n < (split + 1) * per_n; n += 2) {
+      float mm[8], ll[8], oo[8];
+      float M = -INFINITY;
+#pragma unroll
+      for (int p = 0; p < 8; ++p)
+        if (p < splits) {
+          mm[p] = ld_peer_f32(ring + (uint32_t)(64 * 64 + n) * 4u, p);
+          ll[p] = ld_peer_f32(ring + (uint32_t)(64 * 64 + 64 + n) * 4u, p);
+          oo[p] = ld_peer_f32(ring + (uint32_t)(n * 64 + ((e + n) & 63)) * 4u, p);
+          M = fmaxf(M, mm[p]);
+        }
+      float L = 0.f, o = 0.f;
+#pragma unroll
+      for (int p = 0; p < 8; ++p)
+        if (p < splits) {
+          const float w = (mm[p] == -INFINITY) ? 0.f : exp2f(mm[p] - M);
+          L = fmaf(ll[p], w, L);
+          o = fmaf(oo[p], w, o);
+        }
+      if (n < N) out[((long long)b * N + n) * d_model + h * 64 + e] = __float2bfloat16_rn((n < nv && L > 0.f) ? o / L : 0.f);
+    }
+    cluster_sync_all();
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 3) tmem_dealloc(tmem, 128);
+}
+
+}  // namespace vadusa

@@ -37,22 +37,37 @@ __global__ void tree_embed_kernel(TreeView tree, const int32_t* __restrict__ ove
   for (int i = threadIdx.x; i < d; i += blockDim.x) x[(long long)m * d + i] = to_f<T>(e[i]) + to_f<T>(p[i]);
 }
 
-// One warp per row: y = (x - mean) / sqrt(var + eps) * g + b, rounded to T.
+// One block per row: y = (x - mean) / sqrt(var + eps) * g + b, rounded to T.  The row is read
+// once into registers (up to 8 values per thread, d <= 8 * blockDim.x).
 template <typename T>
-__global__ void layernorm_kernel(const float* __restrict__ x, const float* __restrict__ g,
-                                 const float* __restrict__ bta, T* __restrict__ y, int rows, int d, float eps) {
-  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  if (row >= rows) return;
+__global__ void __launch_bounds__(256) layernorm_kernel(const float* __restrict__ x, const float* __restrict__ g,
+                                                        const float* __restrict__ bta, T* __restrict__ y, int rows, int d,
+                                                        float eps) {
+  __shared__ float red[8];
+  const int row = blockIdx.x;
   const float* xr = x + (long long)row * d;
+  float v[8];
+  int cnt = 0;
   float s = 0.f;
-  for (int i = lane; i < d; i += 32) s += xr[i];
-  const float mean = warp_sum(s) / (float)d;
-  float v = 0.f;
-  for (int i = lane; i < d; i += 32) { float t = xr[i] - mean; v += t * t; }
-  const float rstd = 1.0f / sqrtf(warp_sum(v) / (float)d + eps);
+  for (int i = threadIdx.x; i < d; i += blockDim.x) { v[cnt] = xr[i]; s += v[cnt]; ++cnt; }
+  s = warp_sum(s);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = s;
+  __syncthreads();
+  float tot = 0.f;
+  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];
+  const float mean = tot / (float)d;
+  __syncthreads();
+  float q = 0.f;
+  for (int c = 0; c < cnt; ++c) { const float t = v[c] - mean; q += t * t; }
+  q = warp_sum(q);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = q;
+  __syncthreads();
+  float var = 0.f;
+  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) var += red[w];
+  const float rstd = 1.0f / sqrtf(var / (float)d + eps);
   T* yr = y + (long long)row * d;
-  for (int i = lane; i < d; i += 32) yr[i] = from_f<T>((xr[i] - mean) * rstd * g[i] + bta[i]);
+  cnt = 0;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) { yr[i] = from_f<T>((v[cnt] - mean) * rstd * g[i] + bta[i]); ++cnt; }
 }
 
 }  // namespace vadusa

@@ -131,13 +131,27 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
       for (int j = 0; j < CH; ++j) P[(c0 + j) * kGemmRowsW + threadIdx.x] = v[j];
     }
     cluster_sync_all();
+    // CTA ks finishes tokens [ks*per, (ks+1)*per): a thread sums four consecutive features of
+    // one token over the peers (16-byte loads, fixed peer order), warp w takes every 4th token.
     const int per = TN / ksplit;
-    const int nn = n0 + threadIdx.x;
-    for (int t = ks * per; t < (ks + 1) * per; ++t) {
-      float acc = 0.f;
-      const uint32_t a = base + (uint32_t)(t * kGemmRowsW + threadIdx.x) * 4u;
-      for (int peer = 0; peer < ksplit; ++peer) acc += ld_peer_f32(a, peer);
-      if (nn < N && m0 + t < M) epi(zb, m0 + t, nn, acc);
+    const int n4 = (threadIdx.x & 31) * 4;
+    for (int t = ks * per + warp; t < (ks + 1) * per; t += 4) {
+      const uint32_t a = base + (uint32_t)(t * kGemmRowsW + n4) * 4u;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      float4 part[8];
+#pragma unroll
+      for (int peer = 0; peer < 8; ++peer)
+        if (peer < ksplit) part[peer] = ld_peer_f32x4(a, peer);
+#pragma unroll
+      for (int peer = 0; peer < 8; ++peer)
+        if (peer < ksplit) { acc.x += part[peer].x; acc.y += part[peer].y; acc.z += part[peer].z; acc.w += part[peer].w; }
+      if (m0 + t < M) {
+        const int nn = n0 + n4;
+        if (nn + 0 < N) epi(zb, m0 + t, nn + 0, acc.x);
+        if (nn + 1 < N) epi(zb, m0 + t, nn + 1, acc.y);
+        if (nn + 2 < N) epi(zb, m0 + t, nn + 2, acc.z);
+        if (nn + 3 < N) epi(zb, m0 + t, nn + 3, acc.w);
+      }
     }
     cluster_sync_all();                                  // peers may still be reading this CTA's tile
   }

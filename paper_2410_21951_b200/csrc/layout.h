@@ -21,7 +21,7 @@ inline const char* check_config(const vadusa_config* c) {
   if (c->abi_version != VADUSA_ABI_VERSION) return "config.abi_version does not match this library";
   if (c->dtype != 0 && c->dtype != 1) return "dtype must be 0 (fp32) or 1 (bf16)";
   if (c->n_layers < 1 || c->n_layers > 64) return "n_layers out of range";
-  if (c->d_model < 64 || c->d_model % 64) return "d_model must be a positive multiple of 64";
+  if (c->d_model < 64 || c->d_model % 64 || c->d_model > 2048) return "d_model must be a multiple of 64 in 64..2048";
   if (c->n_heads < 1 || c->d_model % c->n_heads) return "n_heads must divide d_model";
   {
     int dh = c->d_model / c->n_heads;

@@ -149,4 +149,13 @@ __device__ __forceinline__ float ld_peer_f32(uint32_t local_addr, uint32_t peer)
   return v;
 }
 
+__device__ __forceinline__ float4 ld_peer_f32x4(uint32_t local_addr, uint32_t peer) {
+  uint32_t remote;
+  float4 v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(peer));
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote) : "memory");
+  return v;
+}
+
 }  // namespace vadusa
