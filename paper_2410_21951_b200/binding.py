@@ -188,7 +188,8 @@ class Vadusa:
         self.blob = torch.from_numpy(pack_weights(self.cfg, weights)).to(self.dev)
         self.kv_pool = torch.zeros(self.L.vadusa_kv_pool_bytes(C.byref(self.cfg)), dtype=torch.uint8, device=self.dev)
         self.workspace = torch.zeros(self.L.vadusa_workspace_bytes(C.byref(self.cfg)), dtype=torch.uint8, device=self.dev)
-        self.stream = stream if stream is not None else torch.cuda.current_stream(self.dev)
+        # a stream of its own: the legacy default stream cannot be captured into CUDA graphs
+        self.stream = stream if stream is not None else torch.cuda.Stream(self.dev)
         self.cfg.kv_pool, self.cfg.kv_pool_bytes = self.kv_pool.data_ptr(), self.kv_pool.numel()
         self.cfg.workspace, self.cfg.workspace_bytes = self.workspace.data_ptr(), self.workspace.numel()
         self.cfg.stream = self.stream.cuda_stream
@@ -221,6 +222,18 @@ class Vadusa:
         if st:
             raise VadusaError(st, self.L.vadusa_last_error(self.ctx).decode())
 
+    def _enter(self):
+        """Order the library's stream after the caller's current stream (inputs are ready)."""
+        cur = self.torch.cuda.current_stream(self.dev)
+        if cur != self.stream:
+            self.stream.wait_stream(cur)
+
+    def _leave(self):
+        """Order the caller's current stream after the library's stream (outputs are ready)."""
+        cur = self.torch.cuda.current_stream(self.dev)
+        if cur != self.stream:
+            cur.wait_stream(self.stream)
+
     @staticmethod
     def _p(t):
         return None if t is None else C.c_void_p(t.data_ptr())
@@ -231,14 +244,17 @@ class Vadusa:
 
     # ---- set-up ----
     def set_tree(self, parent: np.ndarray, rank: np.ndarray, per_sequence: bool = False):
+        self._enter()
         parent = np.ascontiguousarray(parent, dtype=np.int32)
         rank = np.ascontiguousarray(rank, dtype=np.int32)
         n = parent.shape[-1]
         self._ck(self.L.vadusa_set_tree(self.ctx, n, self._h(parent), self._h(rank), int(per_sequence)))
         self.n_nodes = n
+        self._leave()
 
     def begin(self, block_table, ctx_len: Optional[Sequence[int]] = None):
         """block_table: int32 [batch, max_blocks_per_seq] (numpy or device tensor)."""
+        self._enter()
         torch = self.torch
         if not isinstance(block_table, torch.Tensor):
             bt = np.full((len(block_table), self.cfg.max_blocks_per_seq), -1, dtype=np.int32)
@@ -249,44 +265,59 @@ class Vadusa:
         self.batch = block_table.shape[0]
         cl = None if ctx_len is None else np.ascontiguousarray(ctx_len, dtype=np.int32)
         self._ck(self.L.vadusa_begin(self.ctx, self.batch, self._p(block_table), self._h(cl)))
+        self._leave()
 
     def prefill(self, tokens: np.ndarray, lengths: Sequence[int]):
+        self._enter()
         tokens = np.ascontiguousarray(tokens, dtype=np.int32)
         lengths = np.ascontiguousarray(lengths, dtype=np.int32)
         self._ck(self.L.vadusa_prefill(self.ctx, self._h(tokens), self._h(lengths), tokens.shape[1]))
+        self._leave()
 
     def load_state(self, hstar, logits_star):
+        self._enter()
         self._ck(self.L.vadusa_load_state(self.ctx, self._p(hstar), self._p(logits_star)))
+        self._leave()
 
     # ---- hot path ----
     def draft(self, sp: Sampling, tree_tokens=None, topk_out=None):
+        self._enter()
         self._ck(self.L.vadusa_draft(self.ctx, C.byref(sp), self._p(tree_tokens), self._p(topk_out)))
+        self._leave()
 
     def verify_step(self, override=None, logits_out=None, attn_tap=None, hidden_out=None):
+        self._enter()
         self._ck(self.L.vadusa_verify_step(self.ctx, self._p(override), self._p(logits_out), self._p(attn_tap),
                                            self._p(hidden_out)))
+        self._leave()
 
     def accept_and_commit(self, sp: Sampling, forced_best=None, accept_len=None, path_nodes=None, path_tokens=None,
                           kv_slots=None, edge_bits=None, next_root=None):
+        self._enter()
         self._ck(self.L.vadusa_accept_and_commit(self.ctx, C.byref(sp), self._p(forced_best), self._p(accept_len),
                                                  self._p(path_nodes), self._p(path_tokens), self._p(kv_slots),
                                                  self._p(edge_bits), self._p(next_root)))
+        self._leave()
 
     def generate(self, sp: Sampling, max_new_tokens: int, out_tokens, out_len, max_iters: int = 0) -> Stats:
+        self._enter()
         st = Stats()
         self._ck(self.L.vadusa_generate(self.ctx, C.byref(sp), max_new_tokens, max_iters, self._p(out_tokens),
                                         self._p(out_len), C.byref(st)))
+        self._leave()
         return st
 
     def generate_host(self, sp: Sampling, block_table, tokens: np.ndarray, lengths: np.ndarray,
                       max_new_tokens: int, out_tokens: np.ndarray, out_len: np.ndarray) -> Stats:
         """Host buffers in, host buffers out (block_table is a device tensor)."""
+        self._enter()
         st = Stats()
         self._keep["block_table"] = block_table
         self.batch = block_table.shape[0]
         self._ck(self.L.vadusa_generate_host(self.ctx, C.byref(sp), self.batch, self._p(block_table), self._h(tokens),
                                              self._h(lengths), tokens.shape[1], max_new_tokens, self._h(out_tokens),
                                              self._h(out_len), C.byref(st)))
+        self._leave()
         return st
 
     # ---- state ----

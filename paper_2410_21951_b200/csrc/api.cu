@@ -7,6 +7,7 @@
 
 #include <map>
 #include <new>
+#include <string>
 #include <tuple>
 
 #include "accept.cuh"
@@ -50,6 +51,9 @@ struct vadusa_ctx {
   typedef std::tuple<const void*, int, int, int, int, long long> MapKey;   // ptr, rows, K, box rows, batches, batch stride
   std::map<MapKey, CUtensorMap> maps;
   void* encode_fn = nullptr;       // cuTensorMapEncodeTiled, resolved through the runtime
+  // CUDA graphs of the launch sequences of the hot calls, keyed by their baked-in arguments
+  struct GraphRec { cudaGraphExec_t exec = nullptr; int seen = 0; int64_t launches = 0; };
+  std::map<std::string, GraphRec> graphs;
   // per-kernel timing (vadusa_profile_begin/end): one event pair per launch
   struct ProfRec { cudaEvent_t a, b; int cls; };
   bool prof_on = false, prof_pending = false;
@@ -186,6 +190,7 @@ vadusa_status sampling_dev(vadusa_ctx* ctx, const vadusa_sampling* s, SamplingDe
   if (!(s->temperature >= 0.f)) return fail(ctx, VADUSA_EINVAL, "temperature must be >= 0");
   if (!(s->top_p > 0.f)) return fail(ctx, VADUSA_EINVAL, "top_p must be > 0");
   if (s->accept_rule != 0 && s->accept_rule != 1) return fail(ctx, VADUSA_EINVAL, "accept_rule must be 0 or 1");
+  memset(o, 0, sizeof(*o));            // the bytes of this struct key the graph cache: no stray padding
   o->tau = s->tau;
   o->temperature = s->temperature;
   o->inv_temperature = s->temperature > 0.f ? (float)(1.0 / (double)s->temperature) : 1.f;
@@ -245,23 +250,28 @@ vadusa_status launch_gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void
   using Cfg = GemmTcCfg<TN>;
   static bool attr_done = false;
   if (!attr_done) {
-    CU(cudaFuncSetAttribute(gemm_tc_kernel<TN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
+    CU(cudaFuncSetAttribute(gemm_tc_kernel<TN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemMax));
     attr_done = true;
   }
+  const int chunks = K / kGemmBK / ksplit;
+  const int smem = Cfg::smem_for(chunks, ksplit);
   const CUtensorMap *mw, *mx;
   if (vadusa_status s = tensor_map(ctx, W, w_rows, K, kGemmRowsW, batches, w_z, &mw)) return s;
   if (vadusa_status s = tensor_map(ctx, X, M, K, TN, batches, x_z, &mx)) return s;
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3((N + kGemmRowsW - 1) / kGemmRowsW, (M + TN - 1) / TN, batches * ksplit);
   lc.blockDim = dim3(128);
-  lc.dynamicSmemBytes = Cfg::kSmemBytes;
+  lc.dynamicSmemBytes = smem;
   lc.stream = ctx->stream;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = ksplit;
-  lc.attrs = at; lc.numAttrs = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // the kernel calls griddepcontrol.wait
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at; lc.numAttrs = 2;
   PROF(ctx, cls);
-  CU(cudaLaunchKernelEx(&lc, gemm_tc_kernel<TN, Epi>, *mw, *mx, M, N, K / kGemmBK / ksplit, ksplit, epi, err_word(ctx)));
+  CU(cudaLaunchKernelEx(&lc, gemm_tc_kernel<TN, Epi>, *mw, *mx, M, N, chunks, ksplit, Cfg::stages_for(chunks),
+                        Cfg::ring_for(chunks, ksplit), epi, err_word(ctx)));
   LAUNCH_CHECK();
   return VADUSA_OK;
 }
@@ -329,10 +339,12 @@ vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeVi
       lc.blockDim = dim3(128);
       lc.dynamicSmemBytes = kAttSmemBytes;
       lc.stream = ctx->stream;
-      cudaLaunchAttribute at[1];
+      cudaLaunchAttribute at[2];
       at[0].id = cudaLaunchAttributeClusterDimension;
       at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = splits;
-      lc.attrs = at; lc.numAttrs = 1;
+      at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      at[1].val.programmaticStreamSerializationAllowed = 1;
+      lc.attrs = at; lc.numAttrs = 2;
       PROF(ctx, K_ATTENTION);
       CU(cudaLaunchKernelEx(&lc, tree_attention_tc_kernel, *mq, *mkv, layer, ctx->block_table,
                             (const int32_t*)wsptr<int32_t>(ctx, ctx->ws.ctx_len),
@@ -344,6 +356,22 @@ vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeVi
   }
   if (dh == 64) return go(tree_attention_simt_kernel<T, 64>);
   return go(tree_attention_simt_kernel<T, 32>);
+}
+
+template <typename T>
+vadusa_status layernorm(vadusa_ctx* ctx, const float* x, const float* g, const float* b, T* y, int rows) {
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(rows);
+  lc.blockDim = dim3(256);
+  lc.stream = ctx->stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;       // the kernel calls griddepcontrol.wait
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at; lc.numAttrs = 1;
+  PROF(ctx, K_LAYERNORM);
+  CU(cudaLaunchKernelEx(&lc, layernorm_kernel<T>, x, g, b, y, rows, ctx->cfg.d_model, ctx->cfg.ln_eps));
+  LAUNCH_CHECK();
+  return VADUSA_OK;
 }
 
 // One forward pass of the base model over batch * tv.n_nodes rows (verify step).
@@ -371,11 +399,10 @@ vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* overri
   for (int l = 0; l < c.n_layers; ++l) {
     const LayerW& w = ctx->layers[l];
     T* pool = reinterpret_cast<T*>(c.kv_pool) + (long long)l * g.layer_stride;
-    PROF(ctx, K_LAYERNORM);
-    layernorm_kernel<T><<<M, 256, 0, ctx->stream>>>(x, w.ln1_g, w.ln1_b, a, M, d, c.ln_eps);
-    LAUNCH_CHECK();
+    vadusa_status s = layernorm<T>(ctx, x, w.ln1_g, w.ln1_b, a, M);
+    if (s) return s;
     EpiQKV<T> eq{w.bqkv, q, pool, ctx->block_table, ctx_len, nvalid, err_word(ctx), g, N, d};
-    vadusa_status s = product<T>(ctx, K_GEMM_QKV, a, as<T>(w.wqkv), 3 * d, M, 3 * d, d, 1, 0, 0, eq);
+    s = product<T>(ctx, K_GEMM_QKV, a, as<T>(w.wqkv), 3 * d, M, 3 * d, d, 1, 0, 0, eq);
     if (s) return s;
     s = attention<T>(ctx, q, pool, tv, o);
     if (s) return s;
@@ -384,9 +411,8 @@ vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* overri
     EpiResidual eo{w.bo, x, d};
     s = product<T>(ctx, K_GEMM_OUT, o, as<T>(w.wo), d, M, d, d, 1, 0, 0, eo);
     if (s) return s;
-    PROF(ctx, K_LAYERNORM);
-    layernorm_kernel<T><<<M, 256, 0, ctx->stream>>>(x, w.ln2_g, w.ln2_b, a, M, d, c.ln_eps);
-    LAUNCH_CHECK();
+    s = layernorm<T>(ctx, x, w.ln2_g, w.ln2_b, a, M);
+    if (s) return s;
     EpiRelu<T> e1{w.b1, mid, f};
     s = product<T>(ctx, K_GEMM_FFN1, a, as<T>(w.w1), f, M, f, d, 1, 0, 0, e1);
     if (s) return s;
@@ -394,10 +420,7 @@ vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* overri
     s = product<T>(ctx, K_GEMM_FFN2, mid, as<T>(w.w2), d, M, d, f, 1, 0, 0, e2);
     if (s) return s;
   }
-  PROF(ctx, K_LAYERNORM);
-  layernorm_kernel<T><<<M, 256, 0, ctx->stream>>>(x, ctx->lnf_g, ctx->lnf_b,
-                                                          hfinal, M, d, c.ln_eps);
-  LAUNCH_CHECK();
+  if (vadusa_status s = layernorm<T>(ctx, x, ctx->lnf_g, ctx->lnf_b, hfinal, M)) return s;
   EpiLogits el{logits, vp, 0};
   return product<T>(ctx, K_GEMM_LM, hfinal, as<T>(ctx->lm), vp, M, vp, d, 1, 0, 0, el);
 }
@@ -520,6 +543,51 @@ vadusa_status device_errors(vadusa_ctx* ctx) {
   return VADUSA_OK;
 }
 
+// Key of a launch sequence: a tag plus the raw bytes of everything baked into its kernels' arguments.
+struct KeyBuilder {
+  std::string k;
+  explicit KeyBuilder(const char* tag) : k(tag) {}
+  template <typename V> KeyBuilder& add(const V& v) { k.append(reinterpret_cast<const char*>(&v), sizeof(V)); return *this; }
+};
+
+// Runs `body` (which only enqueues work on ctx->stream) eagerly the first time a key is seen,
+// captures it into a CUDA graph the second time, and replays the graph afterwards.  The legacy
+// default stream cannot be captured, and profiling wants separate launches: both run eagerly.
+template <typename F>
+vadusa_status run_graphed(vadusa_ctx* ctx, const std::string& key, F&& body) {
+  if (ctx->stream == nullptr || ctx->prof_on) return body();
+  if (ctx->graphs.size() > 64) {
+    for (auto& kv : ctx->graphs) if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
+    ctx->graphs.clear();
+  }
+  vadusa_ctx::GraphRec& r = ctx->graphs[key];
+  if (r.exec) {
+    CU(cudaGraphLaunch(r.exec, ctx->stream));
+    ctx->launches += r.launches;
+    return VADUSA_OK;
+  }
+  if (r.seen++ == 0) return body();
+  const int64_t l0 = ctx->launches;
+  CU(cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal));
+  vadusa_status s = body();
+  cudaGraph_t graph = nullptr;
+  cudaError_t ce = cudaStreamEndCapture(ctx->stream, &graph);
+  if (s != VADUSA_OK || ce != cudaSuccess || !graph) {
+    if (graph) cudaGraphDestroy(graph);
+    cudaGetLastError();
+    if (s != VADUSA_OK) return s;
+    return fail(ctx, VADUSA_ECUDA, "stream capture failed: %s", cudaGetErrorString(ce));
+  }
+  ce = cudaGraphInstantiate(&r.exec, graph, 0);
+  cudaGraphDestroy(graph);
+  if (ce != cudaSuccess) { r.exec = nullptr; return fail(ctx, VADUSA_ECUDA, "cudaGraphInstantiate: %s", cudaGetErrorString(ce)); }
+  r.launches = ctx->launches - l0;
+  ctx->launches = l0;
+  CU(cudaGraphLaunch(r.exec, ctx->stream));
+  ctx->launches += r.launches;
+  return VADUSA_OK;
+}
+
 #define DISPATCH(expr_f32, expr_bf16) (ctx->cfg.dtype == 1 ? (expr_bf16) : (expr_f32))
 
 vadusa_status need_batch(vadusa_ctx* ctx) {
@@ -635,6 +703,7 @@ vadusa_status vadusa_destroy(vadusa_ctx* ctx) {
   if (ctx->ev_poll) cudaEventDestroy(ctx->ev_poll);
   if (ctx->h_pinned) cudaFreeHost(ctx->h_pinned);
   for (auto& r : ctx->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+  for (auto& kv : ctx->graphs) if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
   delete ctx;
   return VADUSA_OK;
 }
@@ -745,32 +814,38 @@ vadusa_status vadusa_draft(vadusa_ctx* ctx, const vadusa_sampling* sampling, int
   if (ctx->tree_per_seq && tree_tokens) return fail(ctx, VADUSA_EINVAL, "per-sequence topologies take their tokens from the override");
   SamplingDev sp;
   if (vadusa_status s = sampling_dev(ctx, sampling, &sp)) return s;
-  vadusa_status s = DISPATCH(draft<float>(ctx, sp), draft<bf16>(ctx, sp));
+  const vadusa_config& c = ctx->cfg;
+  const std::string key = KeyBuilder("draft").add(sp).add(tree_tokens).add(draft_topk_out).add(ctx->batch)
+                              .add(ctx->n_nodes).add(ctx->tree_per_seq).add(ctx->block_table).k;
+  vadusa_status s = run_graphed(ctx, key, [&]() -> vadusa_status {
+    vadusa_status s = DISPATCH(draft<float>(ctx, sp), draft<bf16>(ctx, sp));
+    if (s) return s;
+    if (draft_topk_out)
+      CU(cudaMemcpyAsync(draft_topk_out, ctx->wsp + ctx->ws.topk, (size_t)ctx->batch * c.n_draft_heads * c.draft_topk * 4,
+                         cudaMemcpyDeviceToDevice, ctx->stream));
+    if (tree_tokens) {
+      // tokens of the tree without a model pass: the embed kernel computes them; run it alone
+      const TreeView tv = tree_of(ctx, false);
+      const int M = ctx->batch * tv.n_nodes;
+      if (c.dtype == 1)
+        tree_embed_kernel<bf16><<<M, 128, 0, ctx->stream>>>(
+            tv, nullptr, wsptr<int32_t>(ctx, ctx->ws.root), wsptr<int32_t>(ctx, ctx->ws.topk), c.n_draft_heads, c.draft_topk,
+            wsptr<int32_t>(ctx, ctx->ws.ctx_len), wsptr<int32_t>(ctx, ctx->ws.nvalid), as<bf16>(ctx->emb_audio),
+            as<bf16>(ctx->emb_phon), as<bf16>(ctx->pos), c.vocab, c.n_phonemes, c.max_pos, c.d_model,
+            wsptr<int32_t>(ctx, ctx->ws.tokens), wsptr<float>(ctx, ctx->ws.x), err_word(ctx));
+      else
+        tree_embed_kernel<float><<<M, 128, 0, ctx->stream>>>(
+            tv, nullptr, wsptr<int32_t>(ctx, ctx->ws.root), wsptr<int32_t>(ctx, ctx->ws.topk), c.n_draft_heads, c.draft_topk,
+            wsptr<int32_t>(ctx, ctx->ws.ctx_len), wsptr<int32_t>(ctx, ctx->ws.nvalid), as<float>(ctx->emb_audio),
+            as<float>(ctx->emb_phon), as<float>(ctx->pos), c.vocab, c.n_phonemes, c.max_pos, c.d_model,
+            wsptr<int32_t>(ctx, ctx->ws.tokens), wsptr<float>(ctx, ctx->ws.x), err_word(ctx));
+      LAUNCH_CHECK();
+      CU(cudaMemcpyAsync(tree_tokens, ctx->wsp + ctx->ws.tokens, (size_t)M * 4, cudaMemcpyDeviceToDevice, ctx->stream));
+    }
+    return VADUSA_OK;
+  });
   if (s) return s;
   ctx->have_draft = true;
-  const vadusa_config& c = ctx->cfg;
-  if (draft_topk_out)
-    CU(cudaMemcpyAsync(draft_topk_out, ctx->wsp + ctx->ws.topk, (size_t)ctx->batch * c.n_draft_heads * c.draft_topk * 4,
-                       cudaMemcpyDeviceToDevice, ctx->stream));
-  if (tree_tokens) {
-    // tokens of the tree without a model pass: the embed kernel computes them; run it alone
-    const TreeView tv = tree_of(ctx, false);
-    const int M = ctx->batch * tv.n_nodes;
-    if (c.dtype == 1)
-      tree_embed_kernel<bf16><<<M, 128, 0, ctx->stream>>>(
-          tv, nullptr, wsptr<int32_t>(ctx, ctx->ws.root), wsptr<int32_t>(ctx, ctx->ws.topk), c.n_draft_heads, c.draft_topk,
-          wsptr<int32_t>(ctx, ctx->ws.ctx_len), wsptr<int32_t>(ctx, ctx->ws.nvalid), as<bf16>(ctx->emb_audio),
-          as<bf16>(ctx->emb_phon), as<bf16>(ctx->pos), c.vocab, c.n_phonemes, c.max_pos, c.d_model,
-          wsptr<int32_t>(ctx, ctx->ws.tokens), wsptr<float>(ctx, ctx->ws.x), err_word(ctx));
-    else
-      tree_embed_kernel<float><<<M, 128, 0, ctx->stream>>>(
-          tv, nullptr, wsptr<int32_t>(ctx, ctx->ws.root), wsptr<int32_t>(ctx, ctx->ws.topk), c.n_draft_heads, c.draft_topk,
-          wsptr<int32_t>(ctx, ctx->ws.ctx_len), wsptr<int32_t>(ctx, ctx->ws.nvalid), as<float>(ctx->emb_audio),
-          as<float>(ctx->emb_phon), as<float>(ctx->pos), c.vocab, c.n_phonemes, c.max_pos, c.d_model,
-          wsptr<int32_t>(ctx, ctx->ws.tokens), wsptr<float>(ctx, ctx->ws.x), err_word(ctx));
-    LAUNCH_CHECK();
-    CU(cudaMemcpyAsync(tree_tokens, ctx->wsp + ctx->ws.tokens, (size_t)M * 4, cudaMemcpyDeviceToDevice, ctx->stream));
-  }
   return VADUSA_OK;
 }
 
@@ -781,17 +856,23 @@ vadusa_status vadusa_verify_step(vadusa_ctx* ctx, const int32_t* tree_tokens_ove
   if (!tree_tokens_override && !ctx->have_draft) return fail(ctx, VADUSA_ESTATE, "verify without a draft or an override");
   if (!tree_tokens_override && ctx->tree_per_seq) return fail(ctx, VADUSA_ESTATE, "per-sequence topologies need a token override");
   const TreeView tv = tree_of(ctx, false);
-  vadusa_status s = DISPATCH(forward<float>(ctx, tv, tree_tokens_override, reinterpret_cast<float*>(attn_tap)),
-                             forward<bf16>(ctx, tv, tree_tokens_override, reinterpret_cast<bf16*>(attn_tap)));
-  if (s) return s;
-  ctx->have_verify = true;
   const vadusa_config& c = ctx->cfg;
   const int M = ctx->batch * tv.n_nodes;
-  if (logits_out)
-    CU(cudaMemcpy2DAsync(logits_out, (size_t)c.vocab * 4, ctx->wsp + ctx->ws.logits, (size_t)vpad(&c) * 4,
-                         (size_t)c.vocab * 4, M, cudaMemcpyDeviceToDevice, ctx->stream));
-  if (hidden_out)
-    CU(cudaMemcpyAsync(hidden_out, ctx->wsp + ctx->ws.hfinal, (size_t)M * c.d_model * esize(&c), cudaMemcpyDeviceToDevice, ctx->stream));
+  const std::string key = KeyBuilder("verify").add(tree_tokens_override).add(logits_out).add(attn_tap).add(hidden_out)
+                              .add(ctx->batch).add(ctx->n_nodes).add(ctx->tree_per_seq).add(ctx->block_table).k;
+  vadusa_status s = run_graphed(ctx, key, [&]() -> vadusa_status {
+    vadusa_status s = DISPATCH(forward<float>(ctx, tv, tree_tokens_override, reinterpret_cast<float*>(attn_tap)),
+                               forward<bf16>(ctx, tv, tree_tokens_override, reinterpret_cast<bf16*>(attn_tap)));
+    if (s) return s;
+    if (logits_out)
+      CU(cudaMemcpy2DAsync(logits_out, (size_t)c.vocab * 4, ctx->wsp + ctx->ws.logits, (size_t)vpad(&c) * 4,
+                           (size_t)c.vocab * 4, M, cudaMemcpyDeviceToDevice, ctx->stream));
+    if (hidden_out)
+      CU(cudaMemcpyAsync(hidden_out, ctx->wsp + ctx->ws.hfinal, (size_t)M * c.d_model * esize(&c), cudaMemcpyDeviceToDevice, ctx->stream));
+    return VADUSA_OK;
+  });
+  if (s) return s;
+  ctx->have_verify = true;
   return VADUSA_OK;
 }
 
@@ -804,8 +885,12 @@ vadusa_status vadusa_accept_and_commit(vadusa_ctx* ctx, const vadusa_sampling* s
   if (vadusa_status s = sampling_dev(ctx, sampling, &sp)) return s;
   AcceptOut out{accept_len, path_nodes, path_tokens, reinterpret_cast<long long*>(kv_slots),
                 reinterpret_cast<unsigned long long*>(edge_bits), next_root};
-  vadusa_status s = DISPATCH(accept_commit<float>(ctx, sp, forced_best_node, out, nullptr, 0, 0),
-                             accept_commit<bf16>(ctx, sp, forced_best_node, out, nullptr, 0, 0));
+  const std::string key = KeyBuilder("accept").add(sp).add(forced_best_node).add(out).add(ctx->batch).add(ctx->n_nodes)
+                              .add(ctx->tree_per_seq).add(ctx->block_table).k;
+  vadusa_status s = run_graphed(ctx, key, [&]() -> vadusa_status {
+    return DISPATCH(accept_commit<float>(ctx, sp, forced_best_node, out, nullptr, 0, 0),
+                    accept_commit<bf16>(ctx, sp, forced_best_node, out, nullptr, 0, 0));
+  });
   if (s) return s;
   ctx->have_verify = ctx->have_draft = false;
   return VADUSA_OK;
@@ -825,6 +910,8 @@ vadusa_status vadusa_generate(vadusa_ctx* ctx, const vadusa_sampling* sampling, 
   CU(cudaMemsetAsync(ctx->wsp + ctx->ws.gen_count, 0, ctx->batch * 4, ctx->stream));
   CU(cudaMemsetAsync(done_word(ctx), 0, 4, ctx->stream));
   if (vadusa_status s = set_active(ctx, ctx->n_nodes)) return s;
+  const std::string iter_key = KeyBuilder("iteration").add(sp).add(out_tokens).add(max_new_tokens).add(ctx->batch)
+                                   .add(ctx->n_nodes).add(ctx->block_table).k;
   ctx->h_pinned[0] = 0;
   bool poll_pending = false;
   int iters = 0;
@@ -834,12 +921,14 @@ vadusa_status vadusa_generate(vadusa_ctx* ctx, const vadusa_sampling* sampling, 
       poll_pending = false;
       if (ctx->h_pinned[0] >= ctx->batch) break;
     }
-    vadusa_status s = DISPATCH(draft<float>(ctx, sp), draft<bf16>(ctx, sp));
-    if (s) return s;
-    s = DISPATCH(forward<float>(ctx, tv, nullptr, nullptr), forward<bf16>(ctx, tv, nullptr, nullptr));
-    if (s) return s;
-    s = DISPATCH(accept_commit<float>(ctx, sp, nullptr, none, out_tokens, max_new_tokens, max_new_tokens),
-                 accept_commit<bf16>(ctx, sp, nullptr, none, out_tokens, max_new_tokens, max_new_tokens));
+    vadusa_status s = run_graphed(ctx, iter_key, [&]() -> vadusa_status {
+      vadusa_status s = DISPATCH(draft<float>(ctx, sp), draft<bf16>(ctx, sp));
+      if (s) return s;
+      s = DISPATCH(forward<float>(ctx, tv, nullptr, nullptr), forward<bf16>(ctx, tv, nullptr, nullptr));
+      if (s) return s;
+      return DISPATCH(accept_commit<float>(ctx, sp, nullptr, none, out_tokens, max_new_tokens, max_new_tokens),
+                      accept_commit<bf16>(ctx, sp, nullptr, none, out_tokens, max_new_tokens, max_new_tokens));
+    });
     if (s) return s;
     if (!poll_pending && (iters & 7) == 7) {
       CU(cudaMemcpyAsync(ctx->h_pinned, done_word(ctx), 4, cudaMemcpyDeviceToHost, ctx->stream));

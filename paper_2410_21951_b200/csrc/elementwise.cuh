@@ -44,6 +44,10 @@ __global__ void __launch_bounds__(256) layernorm_kernel(const float* __restrict_
                                                         const float* __restrict__ bta, T* __restrict__ y, int rows, int d,
                                                         float eps) {
   __shared__ float red[8];
+  // launched as a programmatic dependent: let the next kernel start its prologue, then wait
+  // for the producer of x
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int row = blockIdx.x;
   const float* xr = x + (long long)row * d;
   float v[8];

@@ -29,23 +29,31 @@ template <int TN> struct GemmTcCfg {
   static constexpr int kStagesMax = kGemmSmemBudget / kStageBytes;
   static constexpr int kStages = kStagesMax > 8 ? 8 : kStagesMax;
   static constexpr int kTmemCols = TN < 32 ? 32 : TN;
-  static constexpr int kRingBytes = kStages * kStageBytes;
-  static constexpr int kSmemBytes = kRingBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  // Shared memory needed for `chunks` K chunks per CTA: no more stages than chunks (so that
+  // several CTAs fit on an SM), but room for the split-K partial tile TN x 128 fp32.
+  static int stages_for(int chunks) { return chunks < kStages ? chunks : kStages; }
+  static int ring_for(int chunks, int ksplit) {
+    int ring = stages_for(chunks) * kStageBytes;
+    const int part = ksplit > 1 ? TN * kGemmRowsW * 4 : 0;
+    return ring < part ? part : ring;
+  }
+  static int smem_for(int chunks, int ksplit) { return ring_for(chunks, ksplit) + 1024 /*alignment*/ + 256 /*barriers*/; }
+  static constexpr int kSmemMax = kStages * kStageBytes + 1024 + 256;
 };
 
 template <int TN, typename Epi>
 __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW,
                                                       const __grid_constant__ CUtensorMap tmX, int M, int N,
-                                                      int chunks_per_split, int ksplit, Epi epi, uint32_t* err) {
+                                                      int chunks_per_split, int ksplit, int S, int ring_bytes,
+                                                      Epi epi, uint32_t* err) {
   using Cfg = GemmTcCfg<TN>;
-  constexpr int S = Cfg::kStages;
   constexpr uint32_t kWBytes = kGemmRowsW * kGemmBK * 2, kXBytes = TN * kGemmBK * 2;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* ring_ptr = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t bars = base + Cfg::kRingBytes;          // full[S], empty[S], accum, tmem holder
+  const uint32_t bars = base + ring_bytes;               // full[S], empty[S], accum, tmem holder
   const uint32_t full0 = bars, empty0 = bars + 8 * S, accum_bar = bars + 16 * S, holder = bars + 16 * S + 8;
-  volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(ring_ptr + Cfg::kRingBytes + 16 * S + 8);
+  volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(ring_ptr + ring_bytes + 16 * S + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n0 = blockIdx.x * kGemmRowsW, m0 = blockIdx.y * TN;
