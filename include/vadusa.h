@@ -248,6 +248,35 @@ typedef struct {
 vadusa_status vadusa_profile_begin(vadusa_ctx *ctx);
 vadusa_status vadusa_profile_end(vadusa_ctx *ctx, vadusa_kernel_time *h_out, int32_t capacity, int32_t *h_count);
 
+/* ---- for callers that cannot allocate device memory ---------------------------------- */
+/* (The paper has no counterpart to this call; it exists for deployment reasons only.)
+ * The draft heads' top-k, like the draft-head part of vadusa_draft, but without a context
+ * and without a workspace: the intermediate results (the residual-block outputs and the
+ * heads' logits) live in a fixed 2 MiB device array compiled into the library, which every
+ * GPU that loads the library holds until the process exits.  It is meant for code that may
+ * not call cudaMalloc: a plug-in inside another framework's memory plan, a real-time audio
+ * loop that must not touch the allocator once it runs, a process whose device memory was
+ * handed out completely before this library was loaded.  The call makes no allocation of
+ * any kind, on the host or on the device.
+ *   draft_w [heads][d_model][d_model], draft_u [heads][ceil(vocab/128)*128][d_model] in the
+ *   model dtype (0 fp32, 1 bf16; the layout of the weight blob), draft_b fp32 [heads][d_model],
+ *   hstar [batch][d_model] in the model dtype, topk_out int32 [batch][heads][topk]; all device
+ *   memory of the current device.  Work is enqueued on `stream`; the call does not synchronise.
+ * Limits: batch <= 64 and heads * batch * (d_model * sizeof(dtype) + ceil(vocab/128)*128 * 4)
+ *   + 768 <= vadusa_static_scratch_bytes(); larger requests return VADUSA_ENOMEM with a message
+ *   in vadusa_static_last_error().  The arithmetic is the plain-FMA one for both dtypes.
+ * The first call on a device looks up the array's device address (with that device current):
+ *   make that first call outside any stream capture.
+ * All calls on one GPU share the array and it keeps what the last call left there; every
+ *   call overwrites what it reads, so nothing needs clearing, but two calls that overlap on
+ *   the GPU (different streams, no ordering between them) race on it. */
+vadusa_status vadusa_draft_topk_static(const void *draft_w, const float *draft_b, const void *draft_u,
+                                       const void *hstar, int32_t dtype, int32_t batch, int32_t d_model,
+                                       int32_t vocab, int32_t n_draft_heads, int32_t topk, int32_t eos_masked,
+                                       int32_t *topk_out, void *stream);
+int64_t vadusa_static_scratch_bytes(void);
+const char *vadusa_static_last_error(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -67,7 +67,8 @@ EXPORTS = ["vadusa_workspace_bytes", "vadusa_weights_bytes", "vadusa_kv_pool_byt
            "vadusa_weight_info", "vadusa_init", "vadusa_destroy", "vadusa_last_error", "vadusa_set_tree",
            "vadusa_begin", "vadusa_prefill", "vadusa_load_state", "vadusa_draft", "vadusa_verify_step",
            "vadusa_accept_and_commit", "vadusa_generate", "vadusa_generate_host", "vadusa_get_lengths",
-           "vadusa_check", "vadusa_kernel_launches", "vadusa_profile_begin", "vadusa_profile_end"]
+           "vadusa_check", "vadusa_kernel_launches", "vadusa_profile_begin", "vadusa_profile_end",
+           "vadusa_draft_topk_static", "vadusa_static_scratch_bytes", "vadusa_static_last_error"]
 
 _lib = None
 
@@ -98,6 +99,9 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "vadusa_generate_host": (I32, [P, C.POINTER(Sampling), I32, P, P, P, I32, I32, P, P, C.POINTER(Stats)]),
         "vadusa_get_lengths": (I32, [P, P]), "vadusa_check": (I32, [P]),
         "vadusa_kernel_launches": (I64, [P]),
+        "vadusa_draft_topk_static": (I32, [P, P, P, P, I32, I32, I32, I32, I32, I32, I32, P, P]),
+        "vadusa_static_scratch_bytes": (I64, []),
+        "vadusa_static_last_error": (C.c_char_p, []),
         "vadusa_profile_begin": (I32, [P]),
         "vadusa_profile_end": (I32, [P, C.POINTER(KernelTime), I32, C.POINTER(I32)]),
     }
@@ -168,6 +172,20 @@ def pack_weights(cfg: Config, weights: Dict[str, np.ndarray]) -> np.ndarray:
         raw = raw.reshape(-1)
         blob[t.offset:t.offset + raw.size] = raw
     return blob
+
+
+def draft_topk_static(draft_w, draft_b, draft_u, hstar, dtype: int, batch: int, d_model: int, vocab: int,
+                      n_draft_heads: int, topk: int, eos_masked: bool, topk_out, stream=None):
+    """vadusa_draft_topk_static: device tensors in, device tensor out, no allocation in the library.
+    `stream` is a torch stream (None: the legacy default stream)."""
+    L = lib()
+    st = L.vadusa_draft_topk_static(C.c_void_p(draft_w.data_ptr()), C.c_void_p(draft_b.data_ptr()),
+                                    C.c_void_p(draft_u.data_ptr()), C.c_void_p(hstar.data_ptr()), dtype, batch,
+                                    d_model, vocab, n_draft_heads, topk, int(bool(eos_masked)),
+                                    C.c_void_p(topk_out.data_ptr()),
+                                    C.c_void_p(stream.cuda_stream) if stream is not None else None)
+    if st:
+        raise VadusaError(st, L.vadusa_static_last_error().decode())
 
 
 class Vadusa:

@@ -17,7 +17,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libvadusa.so")
 STAMP = LIB + ".srchash"
-UNITS = ["api.cu"]
+UNITS = ["api.cu", "noalloc.cu"]
 
 
 def _sources():
