@@ -394,14 +394,16 @@ vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* overri
   tree_embed_kernel<T><<<M, 128, 0, ctx->stream>>>(
       tv, override_tokens, wsptr<int32_t>(ctx, ctx->ws.root), wsptr<int32_t>(ctx, ctx->ws.topk), c.n_draft_heads,
       c.draft_topk, ctx_len, nvalid, as<T>(ctx->emb_audio), as<T>(ctx->emb_phon), as<T>(ctx->pos),
-      c.vocab, c.n_phonemes, c.max_pos, d, wsptr<int32_t>(ctx, ctx->ws.tokens), x, err_word(ctx));
+      c.vocab, c.n_phonemes, c.max_pos, d, wsptr<int32_t>(ctx, ctx->ws.tokens), x, ctx->block_table, g,
+      wsptr<long long>(ctx, ctx->ws.kv_row), err_word(ctx));
   LAUNCH_CHECK();
   for (int l = 0; l < c.n_layers; ++l) {
     const LayerW& w = ctx->layers[l];
     T* pool = reinterpret_cast<T*>(c.kv_pool) + (long long)l * g.layer_stride;
     vadusa_status s = layernorm<T>(ctx, x, w.ln1_g, w.ln1_b, a, M);
     if (s) return s;
-    EpiQKV<T> eq{w.bqkv, q, pool, ctx->block_table, ctx_len, nvalid, err_word(ctx), g, N, d};
+    EpiQKV<T> eq{w.bqkv, q, pool, wsptr<long long>(ctx, ctx->ws.kv_row), (long long)c.n_heads * kKvBlock * g.head_dim,
+                 kKvBlock * g.head_dim, g.head_dim, d};
     s = product<T>(ctx, K_GEMM_QKV, a, as<T>(w.wqkv), 3 * d, M, 3 * d, d, 1, 0, 0, eq);
     if (s) return s;
     s = attention<T>(ctx, q, pool, tv, o);
@@ -832,13 +834,15 @@ vadusa_status vadusa_draft(vadusa_ctx* ctx, const vadusa_sampling* sampling, int
             tv, nullptr, wsptr<int32_t>(ctx, ctx->ws.root), wsptr<int32_t>(ctx, ctx->ws.topk), c.n_draft_heads, c.draft_topk,
             wsptr<int32_t>(ctx, ctx->ws.ctx_len), wsptr<int32_t>(ctx, ctx->ws.nvalid), as<bf16>(ctx->emb_audio),
             as<bf16>(ctx->emb_phon), as<bf16>(ctx->pos), c.vocab, c.n_phonemes, c.max_pos, c.d_model,
-            wsptr<int32_t>(ctx, ctx->ws.tokens), wsptr<float>(ctx, ctx->ws.x), err_word(ctx));
+            wsptr<int32_t>(ctx, ctx->ws.tokens), wsptr<float>(ctx, ctx->ws.x), ctx->block_table, geom_of(ctx),
+            (long long*)nullptr, err_word(ctx));
       else
         tree_embed_kernel<float><<<M, 128, 0, ctx->stream>>>(
             tv, nullptr, wsptr<int32_t>(ctx, ctx->ws.root), wsptr<int32_t>(ctx, ctx->ws.topk), c.n_draft_heads, c.draft_topk,
             wsptr<int32_t>(ctx, ctx->ws.ctx_len), wsptr<int32_t>(ctx, ctx->ws.nvalid), as<float>(ctx->emb_audio),
             as<float>(ctx->emb_phon), as<float>(ctx->pos), c.vocab, c.n_phonemes, c.max_pos, c.d_model,
-            wsptr<int32_t>(ctx, ctx->ws.tokens), wsptr<float>(ctx, ctx->ws.x), err_word(ctx));
+            wsptr<int32_t>(ctx, ctx->ws.tokens), wsptr<float>(ctx, ctx->ws.x), ctx->block_table, geom_of(ctx),
+            (long long*)nullptr, err_word(ctx));
       LAUNCH_CHECK();
       CU(cudaMemcpyAsync(tree_tokens, ctx->wsp + ctx->ws.tokens, (size_t)M * 4, cudaMemcpyDeviceToDevice, ctx->stream));
     }

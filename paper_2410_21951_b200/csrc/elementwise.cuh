@@ -6,7 +6,7 @@ namespace vadusa {
 
 // One block per tree node row m = b * n_nodes + n.
 // token = override ? override[m] : (n == 0 ? root[b] : topk[b][depth-1][rank]);
-// position = ctx_len[b] + depth[n]; x[m] = E[token] + P[position] (fp32).
+// position = ctx_len[b] + depth[n]; x[m] = E[token] + P[position] (fp32); kv_row[m] = cache slot of the node.
 // Token ids >= vocab address the phoneme table.
 template <typename T>
 __global__ void tree_embed_kernel(TreeView tree, const int32_t* __restrict__ override_tokens,
@@ -15,7 +15,9 @@ __global__ void tree_embed_kernel(TreeView tree, const int32_t* __restrict__ ove
                                   const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ nvalid,
                                   const T* __restrict__ emb_audio, const T* __restrict__ emb_phon,
                                   const T* __restrict__ pos_table, int vocab, int n_phonemes, int max_pos, int d,
-                                  int32_t* __restrict__ tokens_out, float* __restrict__ x, uint32_t* err) {
+                                  int32_t* __restrict__ tokens_out, float* __restrict__ x,
+                                  const int32_t* __restrict__ block_table, KvGeom geom, long long* __restrict__ kv_row,
+                                  uint32_t* err) {
   const int m = blockIdx.x;
   const int b = m / tree.n_nodes, n = m % tree.n_nodes;
   const int to = tree.off(b);
@@ -32,7 +34,18 @@ __global__ void tree_embed_kernel(TreeView tree, const int32_t* __restrict__ ove
   if (tok >= 0 && tok < vocab) e = emb_audio + (long long)tok * d;
   else if (tok >= vocab && tok < vocab + n_phonemes) e = emb_phon + (long long)(tok - vocab) * d;
   else { if (live && threadIdx.x == 0) atomicOr(err, kErrCapacity); e = emb_audio; }
-  if (threadIdx.x == 0) tokens_out[m] = tok;
+  if (threadIdx.x == 0) {
+    tokens_out[m] = tok;
+    // where this node's K/V rows go: slot ctx_len + n behind the context (the q/k/v product's
+    // epilogue reads this instead of walking the block table per element)
+    long long row = -1;
+    if (live && kv_row) {
+      const int slot = ctx_len[b] + n;
+      const long long blk = kv_block_of(block_table, geom, b, slot, err);
+      if (blk >= 0) row = geom.elem(blk, 0, 0, slot % kKvBlock);
+    }
+    if (kv_row) kv_row[m] = row;
+  }
   const T* p = pos_table + (long long)pos * d;
   for (int i = threadIdx.x; i < d; i += blockDim.x) x[(long long)m * d + i] = to_f<T>(e[i]) + to_f<T>(p[i]);
 }

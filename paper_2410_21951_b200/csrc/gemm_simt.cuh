@@ -7,31 +7,48 @@
 
 namespace vadusa {
 
-// ---- epilogues: called once per output element with the fp32 accumulator ----------
+// ---- epilogues: called with the fp32 accumulator, one element at a time (operator()) or
+// four consecutive features of one token at a time (vec4; n is a multiple of 4) ----------
 
-// q/k/v projection (verify step, per layer): + bias, round to T; q goes to a dense
-// buffer, k and v go straight to the paged cache at slot ctx_len[b] + node.
+template <typename T> __device__ __forceinline__ void store4(T* p, float a, float b, float c, float d);
+template <> __device__ __forceinline__ void store4<float>(float* p, float a, float b, float c, float d) {
+  *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
+}
+template <> __device__ __forceinline__ void store4<bf16>(bf16* p, float a, float b, float c, float d) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+  uint2 v;
+  v.x = *reinterpret_cast<uint32_t*>(&lo);
+  v.y = *reinterpret_cast<uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(p) = v;
+}
+
+// q/k/v projection (verify step, per layer): + bias, round to T; q goes to a dense buffer,
+// k and v go straight to the paged cache at the node's slot (kv_row[m], written by the
+// embedding kernel of the same pass; -1: the row is not scored).
 template <typename T>
 struct EpiQKV {
   const float* bias;
   T* q;
   T* pool;                      // KV pool of this layer
-  const int32_t* block_table;
-  const int32_t* ctx_len;
-  const int32_t* nvalid;
-  uint32_t* err;
-  KvGeom geom;
-  int n_nodes, d;
+  const long long* kv_row;      // [M] element offset of the row's K slot for head 0
+  long long kv_stride;          // elements from a K row to the V row of the same head
+  int tile_elems;               // elements between heads: 64 * head_dim
+  int head_dim, d;
+  __device__ __forceinline__ long long kv_elem(long long row, int n) const {
+    const int c = n - d, kv = c >= d, cc = c - kv * d, h = cc / head_dim;
+    return row + kv * kv_stride + (long long)h * tile_elems + (cc - h * head_dim);
+  }
   __device__ __forceinline__ void operator()(int, int m, int n, float acc) const {
-    T r = from_f<T>(acc + bias[n]);
+    const T r = from_f<T>(acc + bias[n]);
     if (n < d) { q[(long long)m * d + n] = r; return; }
-    const int b = m / n_nodes, node = m % n_nodes;
-    if (node >= nvalid[b]) return;
-    const int pos = ctx_len[b] + node;
-    const long long blk = kv_block_of(block_table, geom, b, pos, err);
-    if (blk < 0) return;
-    const int c = n - d, kv = c / d, cc = c % d;
-    pool[geom.elem(blk, kv, cc / geom.head_dim, pos % kKvBlock) + cc % geom.head_dim] = r;
+    const long long row = kv_row[m];
+    if (row >= 0) pool[kv_elem(row, n)] = r;
+  }
+  __device__ __forceinline__ void vec4(int, int m, int n, float4 a) const {
+    const float4 b = *reinterpret_cast<const float4*>(bias + n);
+    if (n < d) { store4<T>(q + (long long)m * d + n, a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); return; }
+    const long long row = kv_row[m];
+    if (row >= 0) store4<T>(pool + kv_elem(row, n), a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
   }
 };
 
@@ -42,6 +59,13 @@ struct EpiResidual {
   int ld;
   __device__ __forceinline__ void operator()(int, int m, int n, float acc) const {
     x[(long long)m * ld + n] += acc + bias[n];
+  }
+  __device__ __forceinline__ void vec4(int, int m, int n, float4 a) const {
+    const float4 b = *reinterpret_cast<const float4*>(bias + n);
+    float4* p = reinterpret_cast<float4*>(x + (long long)m * ld + n);
+    float4 v = *p;
+    v.x += a.x + b.x; v.y += a.y + b.y; v.z += a.z + b.z; v.w += a.w + b.w;
+    *p = v;
   }
 };
 
@@ -54,6 +78,11 @@ struct EpiRelu {
   __device__ __forceinline__ void operator()(int, int m, int n, float acc) const {
     out[(long long)m * ld + n] = from_f<T>(fmaxf(acc + bias[n], 0.f));
   }
+  __device__ __forceinline__ void vec4(int, int m, int n, float4 a) const {
+    const float4 b = *reinterpret_cast<const float4*>(bias + n);
+    store4<T>(out + (long long)m * ld + n, fmaxf(a.x + b.x, 0.f), fmaxf(a.y + b.y, 0.f), fmaxf(a.z + b.z, 0.f),
+              fmaxf(a.w + b.w, 0.f));
+  }
 };
 
 // vocabulary heads: fp32 logits; z selects the draft head
@@ -63,6 +92,9 @@ struct EpiLogits {
   long long z_stride;
   __device__ __forceinline__ void operator()(int z, int m, int n, float acc) const {
     out[z * z_stride + (long long)m * ld + n] = acc;
+  }
+  __device__ __forceinline__ void vec4(int z, int m, int n, float4 a) const {
+    *reinterpret_cast<float4*>(out + z * z_stride + (long long)m * ld + n) = a;
   }
 };
 
@@ -92,6 +124,9 @@ struct EpiDraftHiddenFlat {
     const float t = acc + bias[n];
     const float s = t / (1.0f + expf(-t));
     out[((long long)head * batch + m) * d + col] = from_f<T>(to_f<T>(h[(long long)m * d + col]) + s);
+  }
+  __device__ __forceinline__ void vec4(int z, int m, int n, float4 a) const {
+    (*this)(z, m, n, a.x); (*this)(z, m, n + 1, a.y); (*this)(z, m, n + 2, a.z); (*this)(z, m, n + 3, a.w);
   }
 };
 

@@ -153,13 +153,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
 #pragma unroll
       for (int peer = 0; peer < 8; ++peer)
         if (peer < ksplit) { acc.x += part[peer].x; acc.y += part[peer].y; acc.z += part[peer].z; acc.w += part[peer].w; }
-      if (m0 + t < M) {
-        const int nn = n0 + n4;
-        if (nn + 0 < N) epi(zb, m0 + t, nn + 0, acc.x);
-        if (nn + 1 < N) epi(zb, m0 + t, nn + 1, acc.y);
-        if (nn + 2 < N) epi(zb, m0 + t, nn + 2, acc.z);
-        if (nn + 3 < N) epi(zb, m0 + t, nn + 3, acc.w);
-      }
+      if (m0 + t < M && n0 + n4 < N) epi.vec4(zb, m0 + t, n0 + n4, acc);     // N is a multiple of 4
     }
     cluster_sync_all();                                  // peers may still be reading this CTA's tile
   }

@@ -96,6 +96,7 @@ struct WorkspaceLayout {
   int64_t tree_parent, tree_depth, tree_rank, tree_anc;       // [B*64] (anc: uint64)
   int64_t chain_parent, chain_depth, chain_rank, chain_anc;   // [64]
   int64_t tokens, stage_tokens;          // int32 [M]
+  int64_t kv_row;                        // int64 [M]: element offset of the row's K slot (head 0) in a layer's pool, -1: none
   int64_t topk;                          // int32 [B][heads][k]
   int64_t x;                             // fp32 [M][d]
   int64_t a, q, o, hfinal;               // T [M][d]
@@ -123,6 +124,7 @@ inline WorkspaceLayout workspace_layout(const vadusa_config* c) {
   w.chain_parent = take(64 * 4); w.chain_depth = take(64 * 4); w.chain_rank = take(64 * 4);
   w.chain_anc = take(64 * 8);
   w.tokens = take(M * 4); w.stage_tokens = take(M * 4);
+  w.kv_row = take(M * 8);
   w.topk = take(B * hd * c->draft_topk * 4);
   w.x = take(M * d * 4);
   w.a = take(M * d * es); w.q = take(M * d * es); w.o = take(M * d * es); w.hfinal = take(M * d * es);
