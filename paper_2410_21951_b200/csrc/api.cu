@@ -336,7 +336,7 @@ vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeVi
                               (g.layer_stride * (long long)sizeof(bf16)));
       cudaLaunchConfig_t lc = {};
       lc.gridDim = dim3(c.n_heads, ctx->batch, splits);
-      lc.blockDim = dim3(128);
+      lc.blockDim = dim3(kAttThreads);
       lc.dynamicSmemBytes = kAttSmemBytes;
       lc.stream = ctx->stream;
       cudaLaunchAttribute at[2];

@@ -3,23 +3,32 @@
 // the tree slots ctx_len[b] + m whose bit m is set in anc[n] (paper Sec. II-A, tree attention).
 //
 // One CTA per (head, sequence, KV split); the splits of one (head, sequence) form a cluster.
-// Per 64-key page:  TMA brings the page's K and V tiles (8 KB each, 128-byte swizzle);
-//   S = Q K^T      tcgen05.mma, A = Q tile (rows 64..127 zero), B = K tile, D in TMEM cols 0..63
-//   softmax        one thread per node row reads its 64 scores from TMEM, keeps the running
-//                  max / sum, and writes the weights back to TMEM as two bf16 halves
-//                  (p = hi + lo, 16 significant bits) over the score columns
-//   O_tile = P V   tcgen05.mma with A from TMEM (hi then lo), B = V tile (MN-major), D in cols 64..127
-//   the row's thread folds O_tile into its fp32 register accumulator while the next page runs.
-// Splits are merged over distributed shared memory in a fixed order.
-// Warps: 0-1 softmax rows, warp 2 lane 0 TMA producer, warp 3 TMEM owner and MMA issuer.
+// The 64 query rows are stored twice in the 128-row Q operand, so the scores of row r appear in
+// TMEM lanes r and r + 64: warps 0-1 (lanes 0..63) work on keys 0..31 of every 64-key page,
+// warps 2-3 (lanes 64..127) on keys 32..63.  Per page:
+//   S = Q K^T      tcgen05.mma, A = Q tile, B = K tile, D in TMEM columns 0..63
+//   softmax        each thread reads its 32 scores, the two threads of a row agree on the
+//                  scaling maximum through shared memory, and the weights go back to TMEM as
+//                  two bf16 halves (p = hi + lo, 16 significant bits) over the score columns,
+//                  zero in the other thread's key range
+//   O += P V       tcgen05.mma with A from TMEM (hi then lo), B = V tile (MN-major), accumulating
+//                  in TMEM columns 64..127; lanes r and r + 64 hold the two key-halves' sums
+// The scaling maximum of a row only moves when the page maximum exceeds it by more than 2^6
+// (p <= 64 is harmless in fp32 / bf16); then the row's accumulator is rescaled in TMEM.
+// At the end rows r and r + 64 are added; splits are merged over distributed shared memory in
+// a fixed order.  Warps: 0-3 softmax, warp 4 lane 0 TMA producer, warp 5 TMEM owner / MMA issuer.
 #pragma once
 #include "tc.cuh"
 
 namespace vadusa {
 
-constexpr int kAttStages = 3;
+constexpr int kAttStages = 2;
+constexpr int kAttThreads = 192;
 constexpr int kAttTileBytes = 64 * 64 * 2;                                   // one K or V page tile
-constexpr int kAttSmemBytes = 2 * kAttTileBytes /*Q, 128 rows*/ + kAttStages * 2 * kAttTileBytes + 1024 + 256;
+constexpr int kAttRingBytes = kAttStages * 2 * kAttTileBytes;                // 32 KB; also holds the 64x64 fp32 output exchange
+constexpr int kAttSmemBytes = 2 * kAttTileBytes /*Q, 128 rows*/ + kAttRingBytes + 1024 /*max exchange, block ids*/ +
+                              1024 /*alignment*/ + 256 /*barriers*/;
+constexpr float kAttRescaleStep = 6.0f;                                      // log2 units
 
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
   asm volatile(
@@ -34,6 +43,7 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // D[tmem] (+)= A[tmem] * B[smem] for one K step of 16 elements (A: lane = row, 8 columns of bf16 pairs).
 __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, bool accumulate) {
@@ -46,10 +56,11 @@ __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, u
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
 }
 
-__global__ void __launch_bounds__(128) tree_attention_tc_kernel(
+__global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
     const __grid_constant__ CUtensorMap tmQ,    // q [1][batch * n_nodes][d_model], box 64 x 64
     const __grid_constant__ CUtensorMap tmKV,   // pool [layers][blocks * 2 * heads * 64][64], box 64 x 64
     int layer, const int32_t* __restrict__ block_table, const int32_t* __restrict__ ctx_len,
@@ -61,10 +72,11 @@ __global__ void __launch_bounds__(128) tree_attention_tc_kernel(
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t q_addr = base, ring = base + 2 * kAttTileBytes;
   uint8_t* ring_ptr = base_ptr + 2 * kAttTileBytes;
-  const uint32_t bars = ring + S * 2 * kAttTileBytes;
+  float* xmax = reinterpret_cast<float*>(ring_ptr + kAttRingBytes);          // [2][128] scaling maxima exchange
+  const uint32_t bars = ring + kAttRingBytes + 1024;
   const uint32_t full0 = bars, empty0 = bars + 8 * S, bar_q = bars + 16 * S, bar_s = bar_q + 8, bar_p = bar_q + 16,
                  bar_o = bar_q + 24, holder = bar_q + 32;
-  volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(ring_ptr + S * 2 * kAttTileBytes + 16 * S + 32);
+  volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(ring_ptr + kAttRingBytes + 1024 + 16 * S + 32);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int h = blockIdx.x, b = blockIdx.y, split = blockIdx.z;
@@ -72,17 +84,12 @@ __global__ void __launch_bounds__(128) tree_attention_tc_kernel(
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-    mbar_init(bar_q, 1); mbar_init(bar_s, 1); mbar_init(bar_p, 64); mbar_init(bar_o, 1);
+    mbar_init(bar_q, 1); mbar_init(bar_s, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
     mbar_fence_init();
     tma_prefetch_desc(&tmQ);
     tma_prefetch_desc(&tmKV);
   }
-  {  // rows 64..127 of the Q operand are zero
-    uint4* z = reinterpret_cast<uint4*>(base_ptr + kAttTileBytes);
-    for (int i = tid; i < kAttTileBytes / 16; i += 128) z[i] = make_uint4(0, 0, 0, 0);
-    fence_proxy_async_smem();
-  }
-  if (warp == 3) { tmem_alloc(holder, 128); tmem_relinquish(); }
+  if (warp == 5) { tmem_alloc(holder, 128); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -96,133 +103,187 @@ __global__ void __launch_bounds__(128) tree_attention_tc_kernel(
   const int p0 = split * per, p1 = min(npages, p0 + per);
   const int ntiles = max(0, p1 - p0);
 
-  float o_acc[64];
-  float m_run = -INFINITY, l_run = 0.f;
+  float m_use = -INFINITY, l_run = 0.f;       // softmax threads: scaling maximum (log2 units) and partial sum
 
-  if (warp == 2 && lane == 0) {
-    // ---- TMA producer
-    if (ntiles > 0) {
-      mbar_expect_tx(bar_q, kAttTileBytes);
+  if (warp == 4) {
+    // ---- TMA producer (lane 0); the block ids of this CTA's pages are fetched by the whole warp first
+    long long blk_mine[2] = {0, 0};
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      const int i = lane + 32 * r;
+      if (i < ntiles) {
+        const long long v = kv_block_of(block_table, geom, b, (p0 + i) * kKvBlock, err);
+        blk_mine[r] = v < 0 ? 0 : v;          // flagged; stay inside the pool
+      }
+    }
+    if (lane == 0 && ntiles > 0) {
+      mbar_expect_tx(bar_q, 2 * kAttTileBytes);
       tma_load_3d(q_addr, &tmQ, bar_q, h * 64, b * N, 0);
+      tma_load_3d(q_addr + kAttTileBytes, &tmQ, bar_q, h * 64, b * N, 0);      // the same rows again: lanes 64..127
     }
+    bool ok = true;
     for (int i = 0; i < ntiles; ++i) {
-      const int s = i % S;
-      if (i >= S && !mbar_wait(empty0 + 8 * s, ((i / S) - 1) & 1, err)) break;
-      long long blk = kv_block_of(block_table, geom, b, (p0 + i) * kKvBlock, err);
-      if (blk < 0) blk = 0;                   // flagged; stay inside the pool
-      const int row = (int)((blk * 2 * geom.n_heads + h) * kKvBlock);
-      mbar_expect_tx(full0 + 8 * s, 2 * kAttTileBytes);
-      tma_load_3d(ring + s * 2 * kAttTileBytes, &tmKV, full0 + 8 * s, 0, row, layer);
-      tma_load_3d(ring + s * 2 * kAttTileBytes + kAttTileBytes, &tmKV, full0 + 8 * s, 0, row + geom.n_heads * kKvBlock, layer);
+      long long blk;
+      if (i < 64) {
+        blk = __shfl_sync(0xffffffffu, (i < 32) ? blk_mine[0] : blk_mine[1], i & 31);
+      } else {
+        blk = kv_block_of(block_table, geom, b, (p0 + i) * kKvBlock, err);
+        if (blk < 0) blk = 0;
+      }
+      if (lane == 0 && ok) {
+        const int s = i % S;
+        if (i >= S && !mbar_wait(empty0 + 8 * s, ((i / S) - 1) & 1, err)) {
+          ok = false;                         // timed out (recorded): stop issuing, keep the warp converged
+        } else {
+          const int row = (int)((blk * 2 * geom.n_heads + h) * kKvBlock);
+          mbar_expect_tx(full0 + 8 * s, 2 * kAttTileBytes);
+          tma_load_3d(ring + s * 2 * kAttTileBytes, &tmKV, full0 + 8 * s, 0, row, layer);
+          tma_load_3d(ring + s * 2 * kAttTileBytes + kAttTileBytes, &tmKV, full0 + 8 * s, 0, row + geom.n_heads * kKvBlock, layer);
+        }
+      }
     }
-  } else if (warp == 3 && lane == 0) {
-    // ---- MMA issuer
-    constexpr uint32_t idesc_qk = umma_idesc_bf16(128, 64);
-    constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 64) | (1u << 16);       // B (V tile) is MN-major
-    bool ok = ntiles == 0 || mbar_wait(bar_q, 0, err);
-    for (int i = 0; i < ntiles && ok; ++i) {
-      const int s = i % S;
-      if (!mbar_wait(full0 + 8 * s, (i / S) & 1, err)) break;
-      tc_fence_after();
-      const uint32_t ka = ring + s * 2 * kAttTileBytes, va = ka + kAttTileBytes;
+  } else if (warp == 5) {
+    // ---- MMA issuer (lane 0)
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = umma_idesc_bf16(128, 64);
+      constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 64) | (1u << 16);     // B (V tile) is MN-major
+      bool ok = ntiles == 0 || mbar_wait(bar_q, 0, err);
+      for (int i = 0; i < ntiles && ok; ++i) {
+        const int s = i % S;
+        if (!mbar_wait(full0 + 8 * s, (i / S) & 1, err)) break;
+        tc_fence_after();
+        const uint32_t ka = ring + s * 2 * kAttTileBytes, va = ka + kAttTileBytes;
 #pragma unroll
-      for (int k = 0; k < 4; ++k)
-        umma_bf16(tmem, umma_desc_k_sw128(q_addr + 32 * k), umma_desc_k_sw128(ka + 32 * k), idesc_qk, k != 0);
-      umma_commit(bar_s);
-      if (!mbar_wait(bar_p, i & 1, err)) break;
-      tc_fence_after();
+        for (int k = 0; k < 4; ++k)
+          umma_bf16(tmem, umma_desc_k_sw128(q_addr + 32 * k), umma_desc_k_sw128(ka + 32 * k), idesc_qk, k != 0);
+        umma_commit(bar_s);
+        if (!mbar_wait(bar_p, i & 1, err)) break;
+        tc_fence_after();
 #pragma unroll
-      for (int k = 0; k < 4; ++k)            // 16 keys per step: 8 TMEM columns of A, 16 rows (2048 bytes) of V
-        umma_bf16_ts(tmem + 64, tmem + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, k != 0);
+        for (int k = 0; k < 4; ++k)          // 16 keys per step: 8 TMEM columns of A, 16 rows (2048 bytes) of V
+          umma_bf16_ts(tmem + 64, tmem + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, (i | k) != 0);
 #pragma unroll
-      for (int k = 0; k < 4; ++k)
-        umma_bf16_ts(tmem + 64, tmem + 32 + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, true);
-      umma_commit(empty0 + 8 * s);
-      umma_commit(bar_o);
+        for (int k = 0; k < 4; ++k)
+          umma_bf16_ts(tmem + 64, tmem + 32 + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, true);
+        umma_commit(empty0 + 8 * s);
+        umma_commit(bar_o);
+      }
     }
-  } else if (warp < 2) {
-    // ---- softmax: thread tid owns node row tid (TMEM lane tid)
-#pragma unroll
-    for (int e = 0; e < 64; ++e) o_acc[e] = 0.f;
-    const unsigned long long amask = tid < nv ? tree.anc[tree.off(b) + tid] : 0ull;
+  } else {
+    // ---- softmax: thread tid owns TMEM lane tid = query row (tid & 63), keys 32*half .. 32*half+31 of each page
+    const int row = tid & 63, half = tid >> 6;
+    const unsigned long long amask = row < nv ? tree.anc[tree.off(b) + row] : 0ull;
     const uint32_t trow = tmem + ((uint32_t)(32 * warp) << 16);
-    float corr_prev = 0.f;
     for (int i = 0; i < ntiles; ++i) {
       if (!mbar_wait(bar_s, i & 1, err)) break;
       tc_fence_after();
-      float sc[64];
-      tmem_ld32(trow, sc);
-      tmem_ld32(trow + 32, sc + 32);
-      if (i > 0) {                            // fold the previous page's P V (complete: issued before this S)
-        float ot[32];
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          tmem_ld32(trow + 64 + 32 * half, ot);
-#pragma unroll
-          for (int e = 0; e < 32; ++e) o_acc[32 * half + e] = fmaf(o_acc[32 * half + e], corr_prev, ot[e]);
-        }
-      }
-      const int key0 = (p0 + i) * kKvBlock;
+      float sc[32];
+      tmem_ld32(trow + 32 * half, sc);
+      const int key0 = (p0 + i) * kKvBlock + 32 * half;
       float mx = -INFINITY;
-      if (key0 + kKvBlock <= ctx) {           // whole page inside the context: every key visible
+      if (key0 + 32 <= ctx) {                 // all 32 keys inside the context: every key visible
 #pragma unroll
-        for (int j = 0; j < 64; ++j) { sc[j] *= scale_log2e; mx = fmaxf(mx, sc[j]); }
+        for (int j = 0; j < 32; ++j) { sc[j] *= scale_log2e; mx = fmaxf(mx, sc[j]); }
       } else {
 #pragma unroll
-        for (int j = 0; j < 64; ++j) {
+        for (int j = 0; j < 32; ++j) {
           const int p = key0 + j;
           const bool vis = p < ctx || (p < total && ((amask >> ((p - ctx) & 63)) & 1ull));
           sc[j] = vis ? sc[j] * scale_log2e : -INFINITY;
           mx = fmaxf(mx, sc[j]);
         }
-        if (key0 + kKvBlock > total) {        // rows of V past the tree may hold anything: zero them
-          const int valid = total - key0;
-          if (tid >= valid) {
-            uint4* vr = reinterpret_cast<uint4*>(ring_ptr + (i % S) * 2 * kAttTileBytes + kAttTileBytes + tid * 128);
+      }
+      if ((p0 + i + 1) * kKvBlock > total && tid < 64) {   // rows of V past the tree may hold anything: zero them
+        const int valid = total - (p0 + i) * kKvBlock;
+        if (tid >= valid) {
+          uint4* vr = reinterpret_cast<uint4*>(ring_ptr + (i % S) * 2 * kAttTileBytes + kAttTileBytes + tid * 128);
 #pragma unroll
-            for (int c = 0; c < 8; ++c) vr[c] = make_uint4(0, 0, 0, 0);
-          }
-          fence_proxy_async_smem();
+          for (int c = 0; c < 8; ++c) vr[c] = make_uint4(0, 0, 0, 0);
+        }
+        fence_proxy_async_smem();
+      }
+      // the two threads of a row agree on the page maximum
+      xmax[(i & 1) * 128 + tid] = mx;
+      softmax_bar_sync();
+      mx = fmaxf(mx, xmax[(i & 1) * 128 + (tid ^ 64)]);
+      // move the scaling maximum only when the page maximum exceeds it by more than the step
+      float factor = 1.f;
+      if (mx > m_use + kAttRescaleStep || m_use == -INFINITY) {
+        factor = (m_use == -INFINITY) ? 0.f : exp2f(m_use - mx);
+        if (mx > -INFINITY) m_use = mx;
+      }
+      if (i > 0 && __any_sync(0xffffffffu, factor != 1.f)) {
+        // rescale this row's accumulator (the previous page's P V has completed: it was issued before this S)
+        float ot[32];
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          tmem_ld32(trow + 64 + 32 * hh, ot);
+          uint32_t ob[32];
+#pragma unroll
+          for (int e = 0; e < 32; ++e) ob[e] = __float_as_uint(ot[e] * factor);
+          tmem_st32(trow + 64 + 32 * hh, ob);
         }
       }
-      const float m_new = fmaxf(m_run, mx);
-      corr_prev = (m_run == -INFINITY) ? 0.f : exp2f(m_run - m_new);
+      l_run *= factor;
       float psum = 0.f;
+      uint32_t hv[16], lv[16];
+      const bool dead = m_use == -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const float pa = dead ? 0.f : exp2f(sc[2 * j] - m_use);
+        const float pb = dead ? 0.f : exp2f(sc[2 * j + 1] - m_use);
+        psum += pa + pb;
+        hv[j] = pack_bf16(pa, pb);
+        const float ha = __uint_as_float(hv[j] << 16), hb = __uint_as_float(hv[j] & 0xffff0000u);
+        lv[j] = pack_bf16(pa - ha, pb - hb);
+      }
+      // this thread's 32 keys sit in columns 16*half .. 16*half+15 of each 32-column group; zero elsewhere
       uint32_t hi[32], lo[32];
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const float pa = (m_new == -INFINITY) ? 0.f : exp2f(sc[2 * j] - m_new);
-        const float pb = (m_new == -INFINITY) ? 0.f : exp2f(sc[2 * j + 1] - m_new);
-        psum += pa + pb;
-        const bf16 ha = __float2bfloat16_rn(pa), hb = __float2bfloat16_rn(pb);
-        hi[j] = (uint32_t)__bfloat16_as_ushort(ha) | ((uint32_t)__bfloat16_as_ushort(hb) << 16);
-        lo[j] = pack_bf16(pa - __bfloat162float(ha), pb - __bfloat162float(hb));
+      for (int j = 0; j < 16; ++j) {
+        hi[j] = half == 0 ? hv[j] : 0u; hi[16 + j] = half == 1 ? hv[j] : 0u;
+        lo[j] = half == 0 ? lv[j] : 0u; lo[16 + j] = half == 1 ? lv[j] : 0u;
       }
-      l_run = l_run * corr_prev + psum;
-      m_run = m_new;
+      l_run += psum;
       tmem_st32(trow, hi);
       tmem_st32(trow + 32, lo);
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(bar_p);
     }
-    if (ntiles > 0 && mbar_wait(bar_o, (ntiles - 1) & 1, err)) {
-      tc_fence_after();
-      float ot[32];
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        tmem_ld32(trow + 64 + 32 * half, ot);
-#pragma unroll
-        for (int e = 0; e < 32; ++e) o_acc[32 * half + e] = fmaf(o_acc[32 * half + e], corr_prev, ot[e]);
-      }
-    }
+    if (ntiles > 0) { mbar_wait(bar_o, (ntiles - 1) & 1, err); tc_fence_after(); }
   }
   __syncwarp();
   grid_dep_launch();
+  __syncthreads();                            // the ring is idle from here on (every MMA has completed)
 
-  // ---- output
+  // ---- output: rows r and r + 64 are the two key-halves of node r
+  float* Ox = reinterpret_cast<float*>(ring_ptr);          // [64][64] fp32 exchange, skewed columns
+  float* lx = xmax;                                        // [128] partial sums; [128..255] scaling maxima
+  float o_acc[64];
+  if (warp < 4) {
+    const uint32_t trow = tmem + ((uint32_t)(32 * warp) << 16);
+    if (ntiles > 0) {
+      tmem_ld32(trow + 64, o_acc);
+      tmem_ld32(trow + 96, o_acc + 32);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 64; ++e) o_acc[e] = 0.f;
+    }
+    lx[tid] = l_run;
+    if (tid >= 64) {
+#pragma unroll
+      for (int e = 0; e < 64; ++e) Ox[(tid - 64) * 64 + ((e + tid) & 63)] = o_acc[e];
+    }
+  }
+  __syncthreads();
+  if (tid < 64) {
+#pragma unroll
+    for (int e = 0; e < 64; ++e) o_acc[e] += Ox[tid * 64 + ((e + tid) & 63)];
+    l_run += lx[tid + 64];
+  }
   if (splits == 1) {
-    if (warp < 2 && tid < N) {
+    if (tid < 64 && tid < N) {
       const float inv = (tid < nv && l_run > 0.f) ? 1.f / l_run : 0.f;
       uint4* dst = reinterpret_cast<uint4*>(out + ((long long)b * N + tid) * d_model + h * 64);
 #pragma unroll
@@ -236,46 +297,47 @@ __global__ void __launch_bounds__(128) tree_attention_tc_kernel(
       }
     }
   } else {
-    // partial results to shared memory: O[64 nodes][64] fp32, then m[64], l[64] (the ring is idle)
+    // this split's result to shared memory (O [64][64], then l and m per row), then merge over the cluster
     __syncthreads();
-    float* Op = reinterpret_cast<float*>(ring_ptr);
-    float* mp = Op + 64 * 64;
-    float* lp = mp + 64;
-    if (warp < 2) {
+    float* mp = xmax + 128;
+    if (tid < 64) {
 #pragma unroll
-      for (int e = 0; e < 64; ++e) Op[tid * 64 + ((e + tid) & 63)] = o_acc[e];   // skewed: conflict-free
-      mp[tid] = m_run;
-      lp[tid] = l_run;
+      for (int e = 0; e < 64; ++e) Ox[tid * 64 + ((e + tid) & 63)] = o_acc[e];
+      lx[tid] = l_run;
+      mp[tid] = m_use;
     }
     cluster_sync_all();
+    const uint32_t ox_addr = ring, lx_addr = ring + kAttRingBytes, mp_addr = lx_addr + 128 * 4;
     const int per_n = 64 / splits;
-    const int e = tid & 63;
-    for (int n = split * per_n + (tid >> 6); n < (split + 1) * per_n; n += 2) {
-      float mm[8], ll[8], oo[8];
-      float M = -INFINITY;
+    if (tid < 128) {
+      const int e = tid & 63;
+      for (int n = split * per_n + (tid >> 6); n < (split + 1) * per_n; n += 2) {
+        float mm[8], ll[8], oo[8];
+        float M = -INFINITY;
 #pragma unroll
-      for (int p = 0; p < 8; ++p)
-        if (p < splits) {
-          mm[p] = ld_peer_f32(ring + (uint32_t)(64 * 64 + n) * 4u, p);
-          ll[p] = ld_peer_f32(ring + (uint32_t)(64 * 64 + 64 + n) * 4u, p);
-          oo[p] = ld_peer_f32(ring + (uint32_t)(n * 64 + ((e + n) & 63)) * 4u, p);
-          M = fmaxf(M, mm[p]);
-        }
-      float L = 0.f, o = 0.f;
+        for (int p = 0; p < 8; ++p)
+          if (p < splits) {
+            mm[p] = ld_peer_f32(mp_addr + (uint32_t)n * 4u, p);
+            ll[p] = ld_peer_f32(lx_addr + (uint32_t)n * 4u, p);
+            oo[p] = ld_peer_f32(ox_addr + (uint32_t)(n * 64 + ((e + n) & 63)) * 4u, p);
+            M = fmaxf(M, mm[p]);
+          }
+        float L = 0.f, o = 0.f;
 #pragma unroll
-      for (int p = 0; p < 8; ++p)
-        if (p < splits) {
-          const float w = (mm[p] == -INFINITY) ? 0.f : exp2f(mm[p] - M);
-          L = fmaf(ll[p], w, L);
-          o = fmaf(oo[p], w, o);
-        }
-      if (n < N) out[((long long)b * N + n) * d_model + h * 64 + e] = __float2bfloat16_rn((n < nv && L > 0.f) ? o / L : 0.f);
+        for (int p = 0; p < 8; ++p)
+          if (p < splits) {
+            const float w = (mm[p] == -INFINITY) ? 0.f : exp2f(mm[p] - M);
+            L = fmaf(ll[p], w, L);
+            o = fmaf(oo[p], w, o);
+          }
+        if (n < N) out[((long long)b * N + n) * d_model + h * 64 + e] = __float2bfloat16_rn((n < nv && L > 0.f) ? o / L : 0.f);
+      }
     }
     cluster_sync_all();
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 3) tmem_dealloc(tmem, 128);
+  if (warp == 5) tmem_dealloc(tmem, 128);
 }
 
 }  // namespace vadusa
