@@ -41,6 +41,8 @@ struct vadusa_ctx {
   int n_nodes = 0;            // current tree size (0: none set)
   int tree_per_seq = 0;
   int max_rank_used = 0;
+  int tree_max_depth = 0;
+  long long ctx_bound = 0;    // host-side upper bound of the longest context (grows by the longest path per commit)
   const int32_t* block_table = nullptr;
   bool have_draft = false, have_verify = false;
   int64_t launches = 0;
@@ -305,6 +307,15 @@ vadusa_status product(vadusa_ctx* ctx, int cls, const T* X, const T* W, int w_ro
   return gemm<T>(ctx, cls, X, W, M, N, K, batches, x_z, w_z, epi);
 }
 
+// KV splits of the tensor-core attention: enough CTAs for about two per SM even at batch 1.
+// (Ragged batches are balanced by visiting the sequences longest first, see seq_order_kernel.)
+int attention_splits(const vadusa_ctx* ctx, int n_nodes) {
+  int splits = 1;
+  while (splits < 8 && ctx->cfg.n_heads * ctx->batch * splits * 2 <= 296) splits *= 2;
+  (void)n_nodes;
+  return splits;
+}
+
 template <typename T>
 vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeView& tv, T* out) {
   const vadusa_config& c = ctx->cfg;
@@ -324,8 +335,7 @@ vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeVi
   if constexpr (std::is_same<T, bf16>::value) {
     if (dh == 64) {
       // tensor-core kernel; KV splits so that about two CTAs per SM exist even at batch 1
-      int splits = 1;
-      while (splits < 8 && c.n_heads * ctx->batch * splits * 2 <= 296) splits *= 2;
+      const int splits = attention_splits(ctx, tv.n_nodes);
       const CUtensorMap *mq, *mkv;
       const int M = ctx->batch * tv.n_nodes;
       if (vadusa_status s = tensor_map(ctx, q, M, c.d_model, 64, 1, 0, &mq)) return s;
@@ -348,7 +358,8 @@ vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeVi
       PROF(ctx, K_ATTENTION);
       CU(cudaLaunchKernelEx(&lc, tree_attention_tc_kernel, *mq, *mkv, layer, ctx->block_table,
                             (const int32_t*)wsptr<int32_t>(ctx, ctx->ws.ctx_len),
-                            (const int32_t*)wsptr<int32_t>(ctx, ctx->ws.nvalid), tv, g, c.d_model,
+                            (const int32_t*)wsptr<int32_t>(ctx, ctx->ws.nvalid),
+                            (const int32_t*)(ctx->batch > 1 ? wsptr<int32_t>(ctx, ctx->ws.seq_order) : nullptr), tv, g, c.d_model,
                             scale * 1.4426950408889634f, splits, reinterpret_cast<bf16*>(out), err_word(ctx)));
       LAUNCH_CHECK();
       return VADUSA_OK;
@@ -397,6 +408,11 @@ vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* overri
       c.vocab, c.n_phonemes, c.max_pos, d, wsptr<int32_t>(ctx, ctx->ws.tokens), x, ctx->block_table, g,
       wsptr<long long>(ctx, ctx->ws.kv_row), err_word(ctx));
   LAUNCH_CHECK();
+  if (B > 1) {
+    PROF(ctx, K_MISC);
+    seq_order_kernel<<<1, 256, 0, ctx->stream>>>(ctx_len, nvalid, B, wsptr<int32_t>(ctx, ctx->ws.seq_order));
+    LAUNCH_CHECK();
+  }
   for (int l = 0; l < c.n_layers; ++l) {
     const LayerW& w = ctx->layers[l];
     T* pool = reinterpret_cast<T*>(c.kv_pool) + (long long)l * g.layer_stride;
@@ -503,6 +519,7 @@ vadusa_status prefill(vadusa_ctx* ctx, const int32_t* h_tokens, const int32_t* h
     CU(cudaStreamSynchronize(ctx->stream));   // the staging vectors are reused by the next chunk
     vadusa_status s = forward<T>(ctx, tv, d_stage, nullptr);
     if (s) return s;
+    ctx->ctx_bound += (longest - s0) < N ? (longest - s0) : N;
     prefill_advance_kernel<T><<<B, 256, 0, ctx->stream>>>(st, N, wsptr<T>(ctx, ctx->ws.hfinal), c.d_model,
                                                           wsptr<float>(ctx, ctx->ws.logits), vp,
                                                           wsptr<T>(ctx, ctx->ws.hstar),
@@ -725,7 +742,7 @@ vadusa_status vadusa_set_tree(vadusa_ctx* ctx, int32_t n_nodes, const int32_t* h
   }
   std::vector<int32_t> depth((size_t)copies * n_nodes);
   std::vector<unsigned long long> anc((size_t)copies * n_nodes);
-  int max_rank = 0;
+  int max_rank = 0, max_depth = 0;
   for (int s = 0; s < copies; ++s) {
     const int32_t* par = h_parent + (size_t)s * n_nodes;
     const int32_t* rnk = h_rank + (size_t)s * n_nodes;
@@ -751,6 +768,7 @@ vadusa_status vadusa_set_tree(vadusa_ctx* ctx, int32_t n_nodes, const int32_t* h
           return fail(ctx, VADUSA_EINVAL, "node %d: nodes of one depth must be in rank-path order", n);
       }
       max_rank = rnk[n] > max_rank ? rnk[n] : max_rank;
+      max_depth = dep[n] > max_depth ? dep[n] : max_depth;
     }
   }
   const size_t n4 = (size_t)copies * n_nodes * sizeof(int32_t);
@@ -762,6 +780,7 @@ vadusa_status vadusa_set_tree(vadusa_ctx* ctx, int32_t n_nodes, const int32_t* h
   ctx->n_nodes = n_nodes;
   ctx->tree_per_seq = per_sequence ? 1 : 0;
   ctx->max_rank_used = max_rank;
+  ctx->tree_max_depth = max_depth;
   ctx->have_draft = ctx->have_verify = false;
   if (ctx->batch > 0) return set_active(ctx, ctx->n_nodes);
   return VADUSA_OK;
@@ -778,10 +797,13 @@ vadusa_status vadusa_begin(vadusa_ctx* ctx, int32_t batch, const int32_t* block_
   ctx->have_draft = ctx->have_verify = false;
   CU(cudaMemsetAsync(ctx->wsp + ctx->ws.scalars, 0, 256, ctx->stream));
   CU(cudaMemsetAsync(ctx->wsp + ctx->ws.gen_count, 0, batch * 4, ctx->stream));
+  ctx->ctx_bound = 0;
   if (h_ctx_len) {
-    for (int b = 0; b < batch; ++b)
+    for (int b = 0; b < batch; ++b) {
       if (h_ctx_len[b] < 0 || h_ctx_len[b] > (int64_t)ctx->cfg.max_blocks_per_seq * 64)
         return fail(ctx, VADUSA_EINVAL, "context length of sequence %d out of range", b);
+      if (h_ctx_len[b] > ctx->ctx_bound) ctx->ctx_bound = h_ctx_len[b];
+    }
     CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.ctx_len, h_ctx_len, batch * 4, cudaMemcpyHostToDevice, ctx->stream));
     CU(cudaStreamSynchronize(ctx->stream));
   } else {
@@ -795,6 +817,7 @@ vadusa_status vadusa_prefill(vadusa_ctx* ctx, const int32_t* h_tokens, const int
   if (!h_tokens || !h_len || stride < 1) return fail(ctx, VADUSA_EINVAL, "prefill arguments are NULL or empty");
   vadusa_status s = DISPATCH(prefill<float>(ctx, h_tokens, h_len, stride), prefill<bf16>(ctx, h_tokens, h_len, stride));
   if (s) return s;
+
   ctx->have_draft = ctx->have_verify = false;
   return set_active(ctx, ctx->n_nodes);
 }
@@ -863,7 +886,8 @@ vadusa_status vadusa_verify_step(vadusa_ctx* ctx, const int32_t* tree_tokens_ove
   const vadusa_config& c = ctx->cfg;
   const int M = ctx->batch * tv.n_nodes;
   const std::string key = KeyBuilder("verify").add(tree_tokens_override).add(logits_out).add(attn_tap).add(hidden_out)
-                              .add(ctx->batch).add(ctx->n_nodes).add(ctx->tree_per_seq).add(ctx->block_table).k;
+                              .add(ctx->batch).add(ctx->n_nodes).add(ctx->tree_per_seq).add(ctx->block_table)
+                              .add(attention_splits(ctx, ctx->n_nodes)).k;
   vadusa_status s = run_graphed(ctx, key, [&]() -> vadusa_status {
     vadusa_status s = DISPATCH(forward<float>(ctx, tv, tree_tokens_override, reinterpret_cast<float*>(attn_tap)),
                                forward<bf16>(ctx, tv, tree_tokens_override, reinterpret_cast<bf16*>(attn_tap)));
@@ -896,6 +920,7 @@ vadusa_status vadusa_accept_and_commit(vadusa_ctx* ctx, const vadusa_sampling* s
                     accept_commit<bf16>(ctx, sp, forced_best_node, out, nullptr, 0, 0));
   });
   if (s) return s;
+  ctx->ctx_bound += ctx->tree_max_depth + 1;
   ctx->have_verify = ctx->have_draft = false;
   return VADUSA_OK;
 }
@@ -914,8 +939,6 @@ vadusa_status vadusa_generate(vadusa_ctx* ctx, const vadusa_sampling* sampling, 
   CU(cudaMemsetAsync(ctx->wsp + ctx->ws.gen_count, 0, ctx->batch * 4, ctx->stream));
   CU(cudaMemsetAsync(done_word(ctx), 0, 4, ctx->stream));
   if (vadusa_status s = set_active(ctx, ctx->n_nodes)) return s;
-  const std::string iter_key = KeyBuilder("iteration").add(sp).add(out_tokens).add(max_new_tokens).add(ctx->batch)
-                                   .add(ctx->n_nodes).add(ctx->block_table).k;
   ctx->h_pinned[0] = 0;
   bool poll_pending = false;
   int iters = 0;
@@ -925,6 +948,8 @@ vadusa_status vadusa_generate(vadusa_ctx* ctx, const vadusa_sampling* sampling, 
       poll_pending = false;
       if (ctx->h_pinned[0] >= ctx->batch) break;
     }
+    const std::string iter_key = KeyBuilder("iteration").add(sp).add(out_tokens).add(max_new_tokens).add(ctx->batch)
+                                     .add(ctx->n_nodes).add(ctx->block_table).add(attention_splits(ctx, ctx->n_nodes)).k;
     vadusa_status s = run_graphed(ctx, iter_key, [&]() -> vadusa_status {
       vadusa_status s = DISPATCH(draft<float>(ctx, sp), draft<bf16>(ctx, sp));
       if (s) return s;
@@ -934,6 +959,7 @@ vadusa_status vadusa_generate(vadusa_ctx* ctx, const vadusa_sampling* sampling, 
                       accept_commit<bf16>(ctx, sp, nullptr, none, out_tokens, max_new_tokens, max_new_tokens));
     });
     if (s) return s;
+    ctx->ctx_bound += ctx->tree_max_depth + 1;
     if (!poll_pending && (iters & 7) == 7) {
       CU(cudaMemcpyAsync(ctx->h_pinned, done_word(ctx), 4, cudaMemcpyDeviceToHost, ctx->stream));
       CU(cudaEventRecord(ctx->ev_poll, ctx->stream));

@@ -64,7 +64,8 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
     const __grid_constant__ CUtensorMap tmQ,    // q [1][batch * n_nodes][d_model], box 64 x 64
     const __grid_constant__ CUtensorMap tmKV,   // pool [layers][blocks * 2 * heads * 64][64], box 64 x 64
     int layer, const int32_t* __restrict__ block_table, const int32_t* __restrict__ ctx_len,
-    const int32_t* __restrict__ nvalid, TreeView tree, KvGeom geom, int d_model, float scale_log2e, int splits,
+    const int32_t* __restrict__ nvalid, const int32_t* __restrict__ order /*may be null*/, TreeView tree, KvGeom geom,
+    int d_model, float scale_log2e, int splits,
     bf16* __restrict__ out, uint32_t* err) {
   constexpr int S = kAttStages;
   extern __shared__ uint8_t smem_raw[];
@@ -79,7 +80,7 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
   volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(ring_ptr + kAttRingBytes + 1024 + 16 * S + 32);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int h = blockIdx.x, b = blockIdx.y, split = blockIdx.z;
+  const int h = blockIdx.x, split = blockIdx.z;
   const int N = tree.n_nodes;
 
   if (tid == 0) {
@@ -96,6 +97,7 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
   const uint32_t tmem = *holder_ptr;
 
   grid_dep_wait();                            // q, K/V rows, lengths come from upstream kernels
+  const int b = order ? order[blockIdx.y] : (int)blockIdx.y;     // longest sequences first
   const int nv = nvalid[b], ctx = ctx_len[b];
   const int total = ctx + nv;
   const int npages = nv > 0 ? (total + kKvBlock - 1) / kKvBlock : 0;
@@ -258,7 +260,7 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
   __syncthreads();                            // the ring is idle from here on (every MMA has completed)
 
   // ---- output: rows r and r + 64 are the two key-halves of node r
-  float* Ox = reinterpret_cast<float*>(ring_ptr);          // [64][64] fp32 exchange, skewed columns
+  float* Ox = reinterpret_cast<float*>(ring_ptr);          // [64][64] fp32 exchange, row r rotated by 4r columns
   float* lx = xmax;                                        // [128] partial sums; [128..255] scaling maxima
   float o_acc[64];
   if (warp < 4) {
@@ -273,13 +275,13 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
     lx[tid] = l_run;
     if (tid >= 64) {
 #pragma unroll
-      for (int e = 0; e < 64; ++e) Ox[(tid - 64) * 64 + ((e + tid) & 63)] = o_acc[e];
+      for (int e = 0; e < 64; ++e) Ox[(tid - 64) * 64 + ((e + 4 * tid) & 63)] = o_acc[e];
     }
   }
   __syncthreads();
   if (tid < 64) {
 #pragma unroll
-    for (int e = 0; e < 64; ++e) o_acc[e] += Ox[tid * 64 + ((e + tid) & 63)];
+    for (int e = 0; e < 64; ++e) o_acc[e] += Ox[tid * 64 + ((e + 4 * tid) & 63)];
     l_run += lx[tid + 64];
   }
   if (splits == 1) {
@@ -302,35 +304,46 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
     float* mp = xmax + 128;
     if (tid < 64) {
 #pragma unroll
-      for (int e = 0; e < 64; ++e) Ox[tid * 64 + ((e + tid) & 63)] = o_acc[e];
+      for (int e = 0; e < 64; ++e) Ox[tid * 64 + ((e + 4 * tid) & 63)] = o_acc[e];
       lx[tid] = l_run;
       mp[tid] = m_use;
     }
     cluster_sync_all();
     const uint32_t ox_addr = ring, lx_addr = ring + kAttRingBytes, mp_addr = lx_addr + 128 * 4;
+    // CTA `split` finishes nodes [split*per_n, (split+1)*per_n): 16 threads per node, four
+    // consecutive features each (16-byte loads from every peer, fixed peer order)
     const int per_n = 64 / splits;
     if (tid < 128) {
-      const int e = tid & 63;
-      for (int n = split * per_n + (tid >> 6); n < (split + 1) * per_n; n += 2) {
-        float mm[8], ll[8], oo[8];
+      const int e4 = (tid & 15) * 4;
+      for (int n = split * per_n + (tid >> 4); n < (split + 1) * per_n; n += 8) {
+        float mm[8], ll[8];
+        float4 oo[8];
         float M = -INFINITY;
+        const int c0 = (e4 + 4 * n) & 63;         // rows are rotated by 4n columns (bank spread, 16-byte aligned)
 #pragma unroll
         for (int p = 0; p < 8; ++p)
           if (p < splits) {
             mm[p] = ld_peer_f32(mp_addr + (uint32_t)n * 4u, p);
             ll[p] = ld_peer_f32(lx_addr + (uint32_t)n * 4u, p);
-            oo[p] = ld_peer_f32(ox_addr + (uint32_t)(n * 64 + ((e + n) & 63)) * 4u, p);
+            oo[p] = ld_peer_f32x4(ox_addr + (uint32_t)(n * 64 + c0) * 4u, p);
             M = fmaxf(M, mm[p]);
           }
-        float L = 0.f, o = 0.f;
+        float L = 0.f;
+        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int p = 0; p < 8; ++p)
           if (p < splits) {
             const float w = (mm[p] == -INFINITY) ? 0.f : exp2f(mm[p] - M);
             L = fmaf(ll[p], w, L);
-            o = fmaf(oo[p], w, o);
+            o.x = fmaf(oo[p].x, w, o.x); o.y = fmaf(oo[p].y, w, o.y); o.z = fmaf(oo[p].z, w, o.z); o.w = fmaf(oo[p].w, w, o.w);
           }
-        if (n < N) out[((long long)b * N + n) * d_model + h * 64 + e] = __float2bfloat16_rn((n < nv && L > 0.f) ? o / L : 0.f);
+        if (n < N) {
+          const float inv = (n < nv && L > 0.f) ? 1.f / L : 0.f;
+          uint2 v;
+          v.x = pack_bf16(o.x * inv, o.y * inv);
+          v.y = pack_bf16(o.z * inv, o.w * inv);
+          *reinterpret_cast<uint2*>(out + ((long long)b * N + n) * d_model + h * 64 + e4) = v;
+        }
       }
     }
     cluster_sync_all();

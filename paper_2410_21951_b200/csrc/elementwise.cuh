@@ -50,6 +50,22 @@ __global__ void tree_embed_kernel(TreeView tree, const int32_t* __restrict__ ove
   for (int i = threadIdx.x; i < d; i += blockDim.x) x[(long long)m * d + i] = to_f<T>(e[i]) + to_f<T>(p[i]);
 }
 
+// order[r] = the sequence with the r-th longest context (ties: lower index first); inactive
+// sequences last.  The attention grid visits sequences in this order, so the longest chains
+// start first and a ragged batch balances over the SMs.  One block.
+__global__ void seq_order_kernel(const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ nvalid, int batch,
+                                 int32_t* __restrict__ order) {
+  for (int b = threadIdx.x; b < batch; b += blockDim.x) {
+    const int lb = nvalid[b] > 0 ? ctx_len[b] : -1;
+    int rank = 0;
+    for (int o = 0; o < batch; ++o) {
+      const int lo = nvalid[o] > 0 ? ctx_len[o] : -1;
+      rank += (lo > lb || (lo == lb && o < b)) ? 1 : 0;
+    }
+    order[rank] = b;
+  }
+}
+
 // One block per row: y = (x - mean) / sqrt(var + eps) * g + b, rounded to T.  The row is read
 // once into registers (up to 8 values per thread, d <= 8 * blockDim.x).
 template <typename T>

@@ -93,6 +93,7 @@ struct WorkspaceLayout {
   int64_t scalars;                       // uint32 err, int32 done_count, padding
   int64_t ctx_len, nvalid, gen_count, commit_base, commit_len, best, root, saved_nvalid;   // int32 [B]
   int64_t commit_path;                   // int32 [B][16]
+  int64_t seq_order;                     // int32 [B]: sequences by descending context length
   int64_t tree_parent, tree_depth, tree_rank, tree_anc;       // [B*64] (anc: uint64)
   int64_t chain_parent, chain_depth, chain_rank, chain_anc;   // [64]
   int64_t tokens, stage_tokens;          // int32 [M]
@@ -119,6 +120,7 @@ inline WorkspaceLayout workspace_layout(const vadusa_config* c) {
   w.commit_base = take(B * 4); w.commit_len = take(B * 4); w.best = take(B * 4); w.root = take(B * 4);
   w.saved_nvalid = take(B * 4);
   w.commit_path = take(B * 16 * 4);
+  w.seq_order = take(B * 4);
   w.tree_parent = take(B * 64 * 4); w.tree_depth = take(B * 64 * 4); w.tree_rank = take(B * 64 * 4);
   w.tree_anc = take(B * 64 * 8);
   w.chain_parent = take(64 * 4); w.chain_depth = take(64 * 4); w.chain_rank = take(64 * 4);
