@@ -298,7 +298,7 @@ def run_c5(args):
     wl = W.workload("C5")
     sh = wl.shape
     weights = W.make_weights(sh, wl.seed())
-    B, N, K, Wm = wl.batch, wl.tree_nodes, args.steps, max(args.warmup, 3)
+    B, N, K, Wm = (args.batch or wl.batch), wl.tree_nodes, args.steps, max(args.warmup, 3)
     lens = W.ragged_lengths(B, wl.context_len[0], wl.context_len[1], wl.seed(900))
     table, total = W.shuffled_block_table([int(s) + N + 16 * (K + Wm + 60) + 8 for s in lens], 64, wl.seed(1))
     g = P.Vadusa(sh, weights, max_batch=B, max_tree_nodes=N, max_blocks_per_seq=table.shape[1], kv_num_blocks=total)
@@ -360,7 +360,7 @@ def run_c5(args):
     line = {"metric": "generated speech tokens/s", "value": tokens / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
             "steps": K, "warmup": Wm, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "C5: verify-step microbenchmark, 12L d1024 16H bf16, batch 64, KV lengths 256-3000, "
+            "config": {"workload": f"C5: verify-step microbenchmark, 12L d1024 16H bf16, batch {B}, KV lengths 256-3000, "
                                    "random 64-node topology per sequence, random K/V and tokens",
                        "step": "draft heads + verify pass over 4096 tree nodes + accept/commit",
                        "l2": "inputs larger than L2 (5 GB of K/V, 321 MB of weights per step)",
@@ -380,6 +380,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="C2", choices=["C2", "C5"],
                     help="C2: the headline step (default); C5: verify-step microbenchmark at batch 64")
+    ap.add_argument("--batch", type=int, default=0, help="C5 only: smaller batch (for profiler captures)")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=5)

@@ -253,6 +253,7 @@ vadusa_status launch_gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void
   static bool attr_done = false;
   if (!attr_done) {
     CU(cudaFuncSetAttribute(gemm_tc_kernel<TN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemMax));
+    CU(cudaFuncSetAttribute(gemm_tc_kernel<TN, Epi>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
     attr_done = true;
   }
   const int chunks = K / kGemmBK / ksplit;
@@ -537,6 +538,8 @@ vadusa_status set_kernel_attributes(vadusa_ctx* ctx) {
   CU(cudaFuncSetAttribute(tree_attention_simt_kernel<bf16, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(64)));
   CU(cudaFuncSetAttribute(tree_attention_simt_kernel<bf16, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(32)));
   CU(cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmemBytes));
+  // ask for the largest shared-memory carve-out so that several CTAs fit on an SM
+  CU(cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
   return VADUSA_OK;
 }
 
