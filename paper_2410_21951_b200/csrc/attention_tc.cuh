@@ -6,13 +6,14 @@
 // The 64 query rows are stored twice in the 128-row Q operand, so the scores of row r appear in
 // TMEM lanes r and r + 64: warps 0-1 (lanes 0..63) work on keys 0..31 of every 64-key page,
 // warps 2-3 (lanes 64..127) on keys 32..63.  Per page:
-//   S = Q K^T      tcgen05.mma, A = Q tile, B = K tile, D in TMEM columns 0..63
+//   S = Q K^T      tcgen05.mma, A = Q tile, B = K tile, D in one of two TMEM score buffers (columns
+//                  0..63 / 64..127), issued one page ahead so that it overlaps the previous softmax
 //   softmax        each thread reads its 32 scores, the two threads of a row agree on the
 //                  scaling maximum through shared memory, and the weights go back to TMEM as
 //                  two bf16 halves (p = hi + lo, 16 significant bits) over the score columns,
 //                  zero in the other thread's key range
 //   O += P V       tcgen05.mma with A from TMEM (hi then lo), B = V tile (MN-major), accumulating
-//                  in TMEM columns 64..127; lanes r and r + 64 hold the two key-halves' sums
+//                  in TMEM columns 128..191; lanes r and r + 64 hold the two key-halves' sums
 // The scaling maximum of a row only moves when the page maximum exceeds it by more than 2^6
 // (p <= 64 is harmless in fp32 / bf16); then the row's accumulator is rescaled in TMEM.
 // At the end rows r and r + 64 are added; splits are merged over distributed shared memory in
@@ -22,10 +23,10 @@
 
 namespace vadusa {
 
-constexpr int kAttStages = 2;
+constexpr int kAttStages = 4;
 constexpr int kAttThreads = 192;
 constexpr int kAttTileBytes = 64 * 64 * 2;                                   // one K or V page tile
-constexpr int kAttRingBytes = kAttStages * 2 * kAttTileBytes;                // 32 KB; also holds the 64x64 fp32 output exchange
+constexpr int kAttRingBytes = kAttStages * 2 * kAttTileBytes;                // 64 KB; also holds the 64x64 fp32 output exchange
 constexpr int kAttSmemBytes = 2 * kAttTileBytes /*Q, 128 rows*/ + kAttRingBytes + 1024 /*max exchange, block ids*/ +
                               1024 /*alignment*/ + 256 /*barriers*/;
 constexpr float kAttRescaleStep = 6.0f;                                      // log2 units
@@ -55,6 +56,12 @@ __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, u
       : "memory");
 }
 
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -75,9 +82,9 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
   uint8_t* ring_ptr = base_ptr + 2 * kAttTileBytes;
   float* xmax = reinterpret_cast<float*>(ring_ptr + kAttRingBytes);          // [2][128] scaling maxima exchange
   const uint32_t bars = ring + kAttRingBytes + 1024;
-  const uint32_t full0 = bars, empty0 = bars + 8 * S, bar_q = bars + 16 * S, bar_s = bar_q + 8, bar_p = bar_q + 16,
-                 bar_o = bar_q + 24, holder = bar_q + 32;
-  volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(ring_ptr + kAttRingBytes + 1024 + 16 * S + 32);
+  const uint32_t full0 = bars, empty0 = bars + 8 * S, bar_q = bars + 16 * S, bar_s0 = bar_q + 8, bar_p = bar_q + 24,
+                 bar_o = bar_q + 32, holder = bar_q + 40;      // bar_s0, bar_s0 + 8: one per score buffer
+  volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(ring_ptr + kAttRingBytes + 1024 + 16 * S + 40);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int h = blockIdx.x, split = blockIdx.z;
@@ -85,12 +92,12 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-    mbar_init(bar_q, 1); mbar_init(bar_s, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
+    mbar_init(bar_q, 1); mbar_init(bar_s0, 1); mbar_init(bar_s0 + 8, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
     mbar_fence_init();
     tma_prefetch_desc(&tmQ);
     tma_prefetch_desc(&tmKV);
   }
-  if (warp == 5) { tmem_alloc(holder, 128); tmem_relinquish(); }
+  if (warp == 5) { tmem_alloc(holder, 256); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -150,24 +157,31 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
       constexpr uint32_t idesc_qk = umma_idesc_bf16(128, 64);
       constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 64) | (1u << 16);     // B (V tile) is MN-major
       bool ok = ntiles == 0 || mbar_wait(bar_q, 0, err);
-      for (int i = 0; i < ntiles && ok; ++i) {
+      // S(i) = Q K(i)^T into score buffer i & 1
+      auto issue_scores = [&](int i) -> bool {
         const int s = i % S;
-        if (!mbar_wait(full0 + 8 * s, (i / S) & 1, err)) break;
+        if (!mbar_wait(full0 + 8 * s, (i / S) & 1, err)) return false;
         tc_fence_after();
-        const uint32_t ka = ring + s * 2 * kAttTileBytes, va = ka + kAttTileBytes;
+        const uint32_t ka = ring + s * 2 * kAttTileBytes;
 #pragma unroll
         for (int k = 0; k < 4; ++k)
-          umma_bf16(tmem, umma_desc_k_sw128(q_addr + 32 * k), umma_desc_k_sw128(ka + 32 * k), idesc_qk, k != 0);
-        umma_commit(bar_s);
+          umma_bf16(tmem + 64 * (i & 1), umma_desc_k_sw128(q_addr + 32 * k), umma_desc_k_sw128(ka + 32 * k), idesc_qk, k != 0);
+        umma_commit(bar_s0 + 8 * (i & 1));
+        return true;
+      };
+      if (ok && ntiles > 0) ok = issue_scores(0);
+      for (int i = 0; i < ntiles && ok; ++i) {
+        if (i + 1 < ntiles && !issue_scores(i + 1)) break;      // one page ahead of the softmax
         if (!mbar_wait(bar_p, i & 1, err)) break;
         tc_fence_after();
+        const uint32_t va = ring + (i % S) * 2 * kAttTileBytes + kAttTileBytes, pa = tmem + 64 * (i & 1);
 #pragma unroll
         for (int k = 0; k < 4; ++k)          // 16 keys per step: 8 TMEM columns of A, 16 rows (2048 bytes) of V
-          umma_bf16_ts(tmem + 64, tmem + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, (i | k) != 0);
+          umma_bf16_ts(tmem + 128, pa + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, (i | k) != 0);
 #pragma unroll
         for (int k = 0; k < 4; ++k)
-          umma_bf16_ts(tmem + 64, tmem + 32 + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, true);
-        umma_commit(empty0 + 8 * s);
+          umma_bf16_ts(tmem + 128, pa + 32 + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, true);
+        umma_commit(empty0 + 8 * (i % S));
         umma_commit(bar_o);
       }
     }
@@ -177,10 +191,11 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
     const unsigned long long amask = row < nv ? tree.anc[tree.off(b) + row] : 0ull;
     const uint32_t trow = tmem + ((uint32_t)(32 * warp) << 16);
     for (int i = 0; i < ntiles; ++i) {
-      if (!mbar_wait(bar_s, i & 1, err)) break;
+      if (!mbar_wait(bar_s0 + 8 * (i & 1), (i >> 1) & 1, err)) break;
       tc_fence_after();
+      const uint32_t tsp = trow + 64 * (i & 1);       // this page's score / weight buffer
       float sc[32];
-      tmem_ld32(trow + 32 * half, sc);
+      tmem_ld32(tsp + 32 * half, sc);
       const int key0 = (p0 + i) * kKvBlock + 32 * half;
       float mx = -INFINITY;
       if (key0 + 32 <= ctx) {                 // all 32 keys inside the context: every key visible
@@ -211,30 +226,32 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
       // move the scaling maximum only when the page maximum exceeds it by more than the step
       float factor = 1.f;
       if (mx > m_use + kAttRescaleStep || m_use == -INFINITY) {
-        factor = (m_use == -INFINITY) ? 0.f : exp2f(m_use - mx);
+        factor = (m_use == -INFINITY) ? 0.f : fast_exp2(m_use - mx);
         if (mx > -INFINITY) m_use = mx;
       }
       if (i > 0 && __any_sync(0xffffffffu, factor != 1.f)) {
-        // rescale this row's accumulator (the previous page's P V has completed: it was issued before this S)
+        // rescale this row's accumulator, once the previous page's P V has completed
+        if (!mbar_wait(bar_o, (i - 1) & 1, err)) break;
+        tc_fence_after();
         float ot[32];
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
-          tmem_ld32(trow + 64 + 32 * hh, ot);
+          tmem_ld32(trow + 128 + 32 * hh, ot);
           uint32_t ob[32];
 #pragma unroll
           for (int e = 0; e < 32; ++e) ob[e] = __float_as_uint(ot[e] * factor);
-          tmem_st32(trow + 64 + 32 * hh, ob);
+          tmem_st32(trow + 128 + 32 * hh, ob);
         }
       }
       l_run *= factor;
-      float psum = 0.f;
+      float psum4[4] = {0.f, 0.f, 0.f, 0.f};
       uint32_t hv[16], lv[16];
-      const bool dead = m_use == -INFINITY;
+      const float m_sub = (m_use == -INFINITY) ? 0.f : m_use;      // no visible key yet: every score is -inf, p = 0
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
-        const float pa = dead ? 0.f : exp2f(sc[2 * j] - m_use);
-        const float pb = dead ? 0.f : exp2f(sc[2 * j + 1] - m_use);
-        psum += pa + pb;
+        const float pa = fast_exp2(sc[2 * j] - m_sub);
+        const float pb = fast_exp2(sc[2 * j + 1] - m_sub);
+        psum4[j & 3] += pa + pb;
         hv[j] = pack_bf16(pa, pb);
         const float ha = __uint_as_float(hv[j] << 16), hb = __uint_as_float(hv[j] & 0xffff0000u);
         lv[j] = pack_bf16(pa - ha, pb - hb);
@@ -246,9 +263,9 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
         hi[j] = half == 0 ? hv[j] : 0u; hi[16 + j] = half == 1 ? hv[j] : 0u;
         lo[j] = half == 0 ? lv[j] : 0u; lo[16 + j] = half == 1 ? lv[j] : 0u;
       }
-      l_run += psum;
-      tmem_st32(trow, hi);
-      tmem_st32(trow + 32, lo);
+      l_run += (psum4[0] + psum4[1]) + (psum4[2] + psum4[3]);
+      tmem_st32(tsp, hi);
+      tmem_st32(tsp + 32, lo);
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(bar_p);
@@ -266,8 +283,8 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
   if (warp < 4) {
     const uint32_t trow = tmem + ((uint32_t)(32 * warp) << 16);
     if (ntiles > 0) {
-      tmem_ld32(trow + 64, o_acc);
-      tmem_ld32(trow + 96, o_acc + 32);
+      tmem_ld32(trow + 128, o_acc);
+      tmem_ld32(trow + 160, o_acc + 32);
     } else {
 #pragma unroll
       for (int e = 0; e < 64; ++e) o_acc[e] = 0.f;
@@ -350,7 +367,7 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) tmem_dealloc(tmem, 128);
+  if (warp == 5) tmem_dealloc(tmem, 256);
 }
 
 }  // namespace vadusa
