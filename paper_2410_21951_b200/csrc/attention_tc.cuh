@@ -42,6 +42,14 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
         "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
 }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
@@ -200,13 +208,13 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
       float mx = -INFINITY;
       if (key0 + 32 <= ctx) {                 // all 32 keys inside the context: every key visible
 #pragma unroll
-        for (int j = 0; j < 32; ++j) { sc[j] *= scale_log2e; mx = fmaxf(mx, sc[j]); }
+        for (int j = 0; j < 32; ++j) mx = fmaxf(mx, sc[j]);
       } else {
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           const int p = key0 + j;
           const bool vis = p < ctx || (p < total && ((amask >> ((p - ctx) & 63)) & 1ull));
-          sc[j] = vis ? sc[j] * scale_log2e : -INFINITY;
+          sc[j] = vis ? sc[j] : -INFINITY;
           mx = fmaxf(mx, sc[j]);
         }
       }
@@ -222,7 +230,7 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
       // the two threads of a row agree on the page maximum
       xmax[(i & 1) * 128 + tid] = mx;
       softmax_bar_sync();
-      mx = fmaxf(mx, xmax[(i & 1) * 128 + (tid ^ 64)]);
+      mx = fmaxf(mx, xmax[(i & 1) * 128 + (tid ^ 64)]) * scale_log2e;     // raw scores; the (positive) scale moves into the exponent
       // move the scaling maximum only when the page maximum exceeds it by more than the step
       float factor = 1.f;
       if (mx > m_use + kAttRescaleStep || m_use == -INFINITY) {
@@ -249,23 +257,24 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
       const float m_sub = (m_use == -INFINITY) ? 0.f : m_use;      // no visible key yet: every score is -inf, p = 0
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
-        const float pa = fast_exp2(sc[2 * j] - m_sub);
-        const float pb = fast_exp2(sc[2 * j + 1] - m_sub);
+        const float pa = fast_exp2(fmaf(sc[2 * j], scale_log2e, -m_sub));
+        const float pb = fast_exp2(fmaf(sc[2 * j + 1], scale_log2e, -m_sub));
         psum4[j & 3] += pa + pb;
         hv[j] = pack_bf16(pa, pb);
         const float ha = __uint_as_float(hv[j] << 16), hb = __uint_as_float(hv[j] & 0xffff0000u);
         lv[j] = pack_bf16(pa - ha, pb - hb);
       }
-      // this thread's 32 keys sit in columns 16*half .. 16*half+15 of each 32-column group; zero elsewhere
-      uint32_t hi[32], lo[32];
-#pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        hi[j] = half == 0 ? hv[j] : 0u; hi[16 + j] = half == 1 ? hv[j] : 0u;
-        lo[j] = half == 0 ? lv[j] : 0u; lo[16 + j] = half == 1 ? lv[j] : 0u;
-      }
       l_run += (psum4[0] + psum4[1]) + (psum4[2] + psum4[3]);
-      tmem_st32(tsp, hi);
-      tmem_st32(tsp + 32, lo);
+      // this thread's 32 keys sit in columns 16*half .. 16*half+15 of each 32-column group; zero elsewhere
+      {
+        uint32_t zero[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) zero[j] = 0u;
+        tmem_st16(tsp + 16 * half, hv);
+        tmem_st16(tsp + 16 * (1 - half), zero);
+        tmem_st16(tsp + 32 + 16 * half, lv);
+        tmem_st16(tsp + 32 + 16 * (1 - half), zero);
+      }
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(bar_p);
