@@ -50,6 +50,24 @@ struct EpiQKV {
     const long long row = kv_row[m];
     if (row >= 0) store4<T>(pool + kv_elem(row, n), a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
   }
+  // CH consecutive tokens m .. m+count-1 of one feature n (all loads first, then the stores)
+  template <int CH>
+  __device__ __forceinline__ void col(int, int m, int n, const float* v, int count) const {
+    const float b = bias[n];
+    if (n < d) {
+#pragma unroll
+      for (int j = 0; j < CH; ++j)
+        if (j < count) q[(long long)(m + j) * d + n] = from_f<T>(v[j] + b);
+      return;
+    }
+    long long rows[CH];
+#pragma unroll
+    for (int j = 0; j < CH; ++j) rows[j] = j < count ? kv_row[m + j] : -1;
+    const long long off = kv_elem(0, n);
+#pragma unroll
+    for (int j = 0; j < CH; ++j)
+      if (rows[j] >= 0) pool[rows[j] + off] = from_f<T>(v[j] + b);
+  }
 };
 
 // output projection / second feed-forward matrix: x += acc + bias (fp32 residual stream)
@@ -67,6 +85,16 @@ struct EpiResidual {
     v.x += a.x + b.x; v.y += a.y + b.y; v.z += a.z + b.z; v.w += a.w + b.w;
     *p = v;
   }
+  template <int CH>
+  __device__ __forceinline__ void col(int, int m, int n, const float* v, int count) const {
+    const float b = bias[n];
+    float xv[CH];
+#pragma unroll
+    for (int j = 0; j < CH; ++j) xv[j] = j < count ? x[(long long)(m + j) * ld + n] : 0.f;
+#pragma unroll
+    for (int j = 0; j < CH; ++j)
+      if (j < count) x[(long long)(m + j) * ld + n] = xv[j] + (v[j] + b);
+  }
 };
 
 // first feed-forward matrix: relu(acc + bias) rounded to T
@@ -83,6 +111,13 @@ struct EpiRelu {
     store4<T>(out + (long long)m * ld + n, fmaxf(a.x + b.x, 0.f), fmaxf(a.y + b.y, 0.f), fmaxf(a.z + b.z, 0.f),
               fmaxf(a.w + b.w, 0.f));
   }
+  template <int CH>
+  __device__ __forceinline__ void col(int, int m, int n, const float* v, int count) const {
+    const float b = bias[n];
+#pragma unroll
+    for (int j = 0; j < CH; ++j)
+      if (j < count) out[(long long)(m + j) * ld + n] = from_f<T>(fmaxf(v[j] + b, 0.f));
+  }
 };
 
 // vocabulary heads: fp32 logits; z selects the draft head
@@ -95,6 +130,12 @@ struct EpiLogits {
   }
   __device__ __forceinline__ void vec4(int z, int m, int n, float4 a) const {
     *reinterpret_cast<float4*>(out + z * z_stride + (long long)m * ld + n) = a;
+  }
+  template <int CH>
+  __device__ __forceinline__ void col(int z, int m, int n, const float* v, int count) const {
+#pragma unroll
+    for (int j = 0; j < CH; ++j)
+      if (j < count) out[z * z_stride + (long long)(m + j) * ld + n] = v[j];
   }
 };
 
@@ -127,6 +168,12 @@ struct EpiDraftHiddenFlat {
   }
   __device__ __forceinline__ void vec4(int z, int m, int n, float4 a) const {
     (*this)(z, m, n, a.x); (*this)(z, m, n + 1, a.y); (*this)(z, m, n + 2, a.z); (*this)(z, m, n + 3, a.w);
+  }
+  template <int CH>
+  __device__ __forceinline__ void col(int z, int m, int n, const float* v, int count) const {
+#pragma unroll
+    for (int j = 0; j < CH; ++j)
+      if (j < count) (*this)(z, m + j, n, v[j]);
   }
 };
 

@@ -26,7 +26,9 @@ constexpr int kGemmSmemBudget = 196 * 1024;
 
 template <int TN> struct GemmTcCfg {
   static constexpr int kStageBytes = kGemmRowsW * kGemmBK * 2 + TN * kGemmBK * 2;
-  static constexpr int kStagesMax = kGemmSmemBudget / kStageBytes;
+  // wide token tiles (tensor-bound shapes): half the budget per CTA, so that two CTAs share an SM and one's
+  // epilogue overlaps the other's main loop; narrow tiles (weight streaming): the whole budget, up to 8 stages
+  static constexpr int kStagesMax = (TN >= 128 ? kGemmSmemBudget / 2 : kGemmSmemBudget) / kStageBytes;
   static constexpr int kStages = kStagesMax > 8 ? 8 : kStagesMax;
   static constexpr int kTmemCols = TN < 32 ? 32 : TN;
   // Shared memory needed for `chunks` K chunks per CTA: no more stages than chunks (so that
@@ -38,7 +40,8 @@ template <int TN> struct GemmTcCfg {
     return ring < part ? part : ring;
   }
   static int smem_for(int chunks, int ksplit) { return ring_for(chunks, ksplit) + 1024 /*alignment*/ + 256 /*barriers*/; }
-  static constexpr int kSmemMax = kStages * kStageBytes + 1024 + 256;
+  static constexpr int kPartBytes = TN * kGemmRowsW * 4;
+  static constexpr int kSmemMax = (kStages * kStageBytes > kPartBytes ? kStages * kStageBytes : kPartBytes) + 1024 + 256;
 };
 
 template <int TN, typename Epi>
@@ -121,11 +124,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
     for (int c0 = 0; c0 < TN; c0 += CH) {
       float v[CH];
       if (CH == 32) tmem_ld32(trow + c0, v); else tmem_ld16(trow + c0, v);
-      if (n < N) {
-#pragma unroll
-        for (int j = 0; j < CH; ++j)
-          if (m0 + c0 + j < M) epi(zb, m0 + c0 + j, n, v[j]);
-      }
+      if (n < N && m0 + c0 < M) epi.template col<CH>(zb, m0 + c0, n, v, M - (m0 + c0));
     }
   } else {
     // park the partial tile as P[token][feature] (the ring is idle: all MMAs have completed)
