@@ -283,7 +283,11 @@ vadusa_status launch_gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void
 template <typename Epi>
 vadusa_status gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void* W, int w_rows, int M, int N, int K,
                       int batches, long long x_z, long long w_z, const Epi& epi) {
-  const int tn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 1024 ? 128 : 256;
+  // token tile: as narrow as the token count allows for weight streaming; 256 for the tensor-bound shapes
+  // when that still gives every SM a CTA pair, else 128
+  const int ntiles_n = (N + kGemmRowsW - 1) / kGemmRowsW;
+  int tn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 1024 ? 128 : 256;
+  if (tn == 256 && ntiles_n * ((M + 255) / 256) * batches < 200) tn = 128;
   const int tiles = ((N + kGemmRowsW - 1) / kGemmRowsW) * ((M + tn - 1) / tn) * batches;
   const int chunks = K / kGemmBK;
   int ksplit = 1;
