@@ -136,11 +136,33 @@ def run_reference(args):
     line = {"impl": "reference", "metric": "generated speech tokens/s", "value": val, "unit": "tokens/s",
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": f"{WORKLOAD}: 12L d1024 16H FFN4096 vocab1025, batch 1, 64-node tree, tau 3, T 1.0"},
+            "config": workload_config(),
             "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
+
+
+def workload_config(extra=None):
+    """The `config` object both arms print."""
+    c = {"workload": f"{WORKLOAD}: 12L d1024 16H FFN4096 vocab1025 bf16, batch 1 per GPU, 64-node tree "
+                     f"(top-10/5/3/2), tau 3, T 1.0, 325-token prefix, random-init weights",
+         "step": "one draft+verify+accept/commit iteration"}
+    if extra:
+        c.update(extra)
+    return c
+
+
+def aggregate(dist, device, ms, e2e_s, tokens, e2e_tokens, launches):
+    """Whole-job numbers of a weak-scaling run: every rank decodes its own sequences, so times
+    are the maximum over ranks and counts the sum.  Works on any backend (NCCL on GPUs; gloo in
+    the CPU tests)."""
+    import torch
+    t = torch.tensor([ms, e2e_s], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    c = torch.tensor([tokens, e2e_tokens, launches], device=device, dtype=torch.float64)
+    dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    return float(t[0]), float(t[1]), int(c[0]), int(c[1]), int(c[2])
 
 
 # ------------------------------------------------------------------------------ our arm
@@ -233,12 +255,7 @@ def run_ours(args):
 
     # ---- aggregate over ranks
     if world > 1:
-        t = torch.tensor([ms, e2e_s], device=g.dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        c = torch.tensor([tokens, e2e_tokens, launches], device=g.dev, dtype=torch.float64)
-        dist.all_reduce(c, op=dist.ReduceOp.SUM)
-        ms, e2e_s = float(t[0]), float(t[1])
-        tokens, e2e_tokens, launches = int(c[0]), int(c[1]), int(c[2])
+        ms, e2e_s, tokens, e2e_tokens, launches = aggregate(dist, g.dev, ms, e2e_s, tokens, e2e_tokens, launches)
 
     if rank == 0:
         peak, peak_kind = _peaks()
@@ -264,11 +281,9 @@ def run_ours(args):
             "metric": "generated speech tokens/s", "value": tokens / (ms * 1e-3), "unit": "tokens/s",
             "n_gpus": world, "steps": K, "warmup": Wm, "ms_per_step": ms / K, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": f"{WORKLOAD}: 12L d1024 16H FFN4096 vocab1025 bf16, batch 1 per GPU, 64-node tree "
-                                   f"(top-10/5/3/2), tau 3, T 1.0, 325-token prefix, random-init weights",
-                       "step": "one draft+verify+accept/commit iteration", "mean_accepted_tokens": tokens / (K * world),
-                       "l2": "inputs larger than L2 (321 MB of weights streamed per step)",
-                       "verify_step_us": ms / K * 1e3},
+            "config": workload_config({"mean_accepted_tokens": tokens / (K * world),
+                                       "l2": "inputs larger than L2 (321 MB of weights streamed per step)",
+                                       "verify_step_us": ms / K * 1e3}),
             "roofline": {"bound": "hbm", "kernel": "projection GEMMs (qkv, out, ffn1, ffn2, lm head)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": f"{peak_kind} copy bandwidth", "traffic": None,
