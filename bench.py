@@ -239,6 +239,33 @@ def run_ours(args):
     steps(n_prof)
     prof = g.profile_end()
 
+    # ---- the same step at a planted acceptance: random-init draft heads are accepted at chance (about 1
+    # token per step), so a labelled second run forces the winning node (test hook) to mimic the mean
+    # acceptance the paper reports for its best setting (3.87 tokens per step, Table 1)
+    fresh()
+    lens_cycle = [4, 4, 4, 3, 4, 4, 4, 4]                          # mean 3.875
+    forced = {L: torch.tensor([int(np.nonzero(tpl.depth == L - 1)[0][0])], dtype=torch.int32, device=g.dev)
+              for L in set(lens_cycle)}
+
+    def planted_steps(n):
+        for i in range(n):
+            g.draft(sp)
+            g.verify_step()
+            g.accept_and_commit(sp, forced_best=forced[lens_cycle[i % len(lens_cycle)]])
+
+    n_pl = min(K, 160)
+    planted_steps(16)
+    pl0 = int(g.lengths()[0])
+    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    p0.record()
+    planted_steps(n_pl)
+    p1.record()
+    barrier()
+    pl_ms = p0.elapsed_time(p1)
+    pl_tokens = int(g.lengths()[0]) - pl0
+    g.check()
+
     # ---- end to end through the host-buffer entry: prefix from host memory, tokens back to host
     h_out = np.zeros((1, gen_cap), dtype=np.int32)
     h_len = np.zeros(1, dtype=np.int32)
@@ -283,7 +310,12 @@ def run_ours(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": workload_config({"mean_accepted_tokens": tokens / (K * world),
                                        "l2": "inputs larger than L2 (321 MB of weights streamed per step)",
-                                       "verify_step_us": ms / K * 1e3}),
+                                       "verify_step_us": ms / K * 1e3,
+                                       "planted_acceptance": {
+                                           "what": "same step with the winning node forced (test hook) so that the mean accepted "
+                                                   "length is the paper's 3.87 (Table 1); this rank only",
+                                           "mean_accepted_tokens": pl_tokens / n_pl, "tokens_per_s": pl_tokens / (pl_ms * 1e-3),
+                                           "ms_per_step": pl_ms / n_pl, "steps": n_pl}}),
             "roofline": {"bound": "hbm", "kernel": "projection GEMMs (qkv, out, ffn1, ffn2, lm head)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": f"{peak_kind} copy bandwidth", "traffic": None,
@@ -391,10 +423,75 @@ def run_c5(args):
     g.close()
 
 
+def run_batch(args):
+    """BASELINE configs 3 (batch 16, vocab 2049, 42-node tree, tau 5, T 0.8, 500 tokens) and 4 (batch 32,
+    contexts 1000-4000 in a paged cache, 64-node tree, tau in {1,3,5}, 256 iterations): prefill through the
+    library, then timed draft+verify+accept/commit steps.  One JSON line per tolerance value."""
+    import torch
+    import workloads as W
+    import paper_2410_21951_b200 as P
+    wl = W.workload(args.workload)
+    sh = wl.shape
+    weights = W.make_weights(sh, wl.seed())
+    tpl = W.static_template(wl.tree_nodes, wl.tree_caps)
+    B = wl.batch
+    prefixes = [W.prefix_for(wl, b) for b in range(B)]
+    toks = [np.concatenate([ph.astype(np.int32) + sh.vocab, pr.astype(np.int32)]) for ph, pr in prefixes]
+    iters = wl.iterations if wl.iterations else wl.gen_tokens
+    if args.steps != 400:
+        iters = args.steps
+    taus = wl.tau_sweep if wl.tau_sweep else (wl.tau,)
+    need = [len(t) + (iters + 8) * (tpl.max_depth + 1) + wl.tree_nodes + 64 for t in toks]
+    table, total = W.shuffled_block_table(need, 64, wl.seed(77), spare_pages=2)
+    g = P.Vadusa(sh, weights, max_batch=B, max_tree_nodes=wl.tree_nodes, max_blocks_per_seq=table.shape[1], kv_num_blocks=total)
+    torch.cuda.set_stream(g.stream)
+    g.set_tree(tpl.parent, tpl.rank)
+    bt = torch.from_numpy(table).to(g.dev)
+    mat = np.zeros((B, max(len(t) for t in toks)), dtype=np.int32)
+    for b, t in enumerate(toks):
+        mat[b, :len(t)] = t
+    lens = np.array([len(t) for t in toks], dtype=np.int32)
+    for tau in taus:
+        sp = P.Sampling.make(tau=tau, temperature=wl.temperature if wl.temperature else 1.0, seed=wl.seed())
+        g.begin(bt)
+        t0 = time.perf_counter()
+        g.prefill(mat, lens)
+        torch.cuda.synchronize()
+        prefill_s = time.perf_counter() - t0
+
+        def steps(n):
+            for _ in range(n):
+                g.draft(sp)
+                g.verify_step()
+                g.accept_and_commit(sp)
+
+        steps(3)
+        len0 = g.lengths().astype(np.int64)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        steps(iters)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        tokens = int((g.lengths().astype(np.int64) - len0).sum())
+        g.check()
+        print(json.dumps({"metric": "generated speech tokens/s", "value": tokens / (ms * 1e-3), "unit": "tokens/s",
+                          "n_gpus": 1, "steps": iters, "warmup": 3, "ms_per_step": ms / iters, "higher_is_better": True,
+                          "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                          "config": {"workload": f"{args.workload}: 12L d1024 16H vocab {sh.vocab} bf16, batch {B}, "
+                                                 f"{wl.tree_nodes}-node tree, tau {tau}, T {sp.temperature:g}, "
+                                                 f"contexts {int(lens.min())}-{int(lens.max())} tokens before decoding",
+                                     "mean_accepted_tokens": tokens / (iters * B), "verify_step_us": ms / iters * 1e3,
+                                     "prefill_s_untimed": round(prefill_s, 3)}}))
+    g.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--workload", default="C2", choices=["C2", "C5"],
-                    help="C2: the headline step (default); C5: verify-step microbenchmark at batch 64")
+    ap.add_argument("--workload", default="C2", choices=["C2", "C3", "C4", "C5"],
+                    help="C2: the headline step (default); C3, C4: the batched configurations; C5: verify-step "
+                         "microbenchmark at batch 64")
     ap.add_argument("--batch", type=int, default=0, help="C5 only: smaller batch (for profiler captures)")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
@@ -405,6 +502,8 @@ def main():
         args.steps = 20 if args.impl == "reference" else 400
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload in ("C3", "C4"):
+        run_batch(args)
     elif args.workload == "C5":
         if args.steps == 400:
             args.steps = 20
