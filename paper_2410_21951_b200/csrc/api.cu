@@ -274,7 +274,7 @@ vadusa_status launch_gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void
   lc.attrs = at; lc.numAttrs = 2;
   PROF(ctx, cls);
   CU(cudaLaunchKernelEx(&lc, gemm_tc_kernel<TN, Epi>, *mw, *mx, M, N, chunks, ksplit, Cfg::stages_for(chunks),
-                        Cfg::ring_for(chunks, ksplit), epi, err_word(ctx)));
+                        Cfg::ring_for(chunks, ksplit), epi, wsptr<float>(ctx, ctx->ws.gemm_part), err_word(ctx)));
   LAUNCH_CHECK();
   return VADUSA_OK;
 }
@@ -291,7 +291,9 @@ vadusa_status gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void* W, in
   const int tiles = ((N + kGemmRowsW - 1) / kGemmRowsW) * ((M + tn - 1) / tn) * batches;
   const int chunks = K / kGemmBK;
   int ksplit = 1;
-  while (ksplit < 8 && tiles * ksplit < 148 && chunks % (ksplit * 2) == 0 && ksplit * 2 <= tn) ksplit *= 2;
+  while (ksplit < 8 && tiles * ksplit < 148 && chunks % (ksplit * 2) == 0 && ksplit * 2 <= tn &&
+         (long long)tiles * ksplit * 2 * tn * kGemmRowsW * 4 <= kGemmPartBytes)
+    ksplit *= 2;
   switch (tn) {
     case 16: return launch_gemm_tc<16>(ctx, cls, X, W, w_rows, M, N, K, batches, x_z, w_z, ksplit, epi);
     case 32: return launch_gemm_tc<32>(ctx, cls, X, W, w_rows, M, N, K, batches, x_z, w_z, ksplit, epi);

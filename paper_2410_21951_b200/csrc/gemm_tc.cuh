@@ -8,8 +8,9 @@
 //
 // Work split: grid.x = feature tiles of 128, grid.y = token tiles of TN, grid.z = batch *
 // ksplit.  With ksplit > 1 the CTAs of one cluster (1,1,ksplit) each take a K slice, park
-// their partial tile in shared memory, and reduce it over distributed shared memory in a
-// fixed order (deterministic), each CTA finishing TN/ksplit tokens of the tile.
+// their partial tile in an exchange area in global memory (it stays in L2, which moves these
+// tiles faster than distributed shared memory did), meet at a cluster barrier, and add the
+// slices in a fixed order (deterministic), each CTA finishing TN/ksplit tokens of the tile.
 //
 // Warp roles (128 threads): warp 0 lane 0 issues TMA loads into a ring of stages, warp 1
 // owns the TMEM allocation and its lane 0 issues the MMAs, all four warps run the epilogue.
@@ -32,23 +33,18 @@ template <int TN> struct GemmTcCfg {
   static constexpr int kStages = kStagesMax > 8 ? 8 : kStagesMax;
   static constexpr int kTmemCols = TN < 32 ? 32 : TN;
   // Shared memory needed for `chunks` K chunks per CTA: no more stages than chunks (so that
-  // several CTAs fit on an SM), but room for the split-K partial tile TN x 128 fp32.
+  // several CTAs fit on an SM).
   static int stages_for(int chunks) { return chunks < kStages ? chunks : kStages; }
-  static int ring_for(int chunks, int ksplit) {
-    int ring = stages_for(chunks) * kStageBytes;
-    const int part = ksplit > 1 ? TN * kGemmRowsW * 4 : 0;
-    return ring < part ? part : ring;
-  }
+  static int ring_for(int chunks, int) { return stages_for(chunks) * kStageBytes; }
   static int smem_for(int chunks, int ksplit) { return ring_for(chunks, ksplit) + 1024 /*alignment*/ + 256 /*barriers*/; }
-  static constexpr int kPartBytes = TN * kGemmRowsW * 4;
-  static constexpr int kSmemMax = (kStages * kStageBytes > kPartBytes ? kStages * kStageBytes : kPartBytes) + 1024 + 256;
+  static constexpr int kSmemMax = kStages * kStageBytes + 1024 + 256;
 };
 
 template <int TN, typename Epi>
 __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW,
                                                       const __grid_constant__ CUtensorMap tmX, int M, int N,
                                                       int chunks_per_split, int ksplit, int S, int ring_bytes,
-                                                      Epi epi, uint32_t* err) {
+                                                      Epi epi, float* __restrict__ part /*split-K exchange*/, uint32_t* err) {
   using Cfg = GemmTcCfg<TN>;
   constexpr uint32_t kWBytes = kGemmRowsW * kGemmBK * 2, kXBytes = TN * kGemmBK * 2;
   extern __shared__ uint8_t smem_raw[];
@@ -127,8 +123,10 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
       if (n < N && m0 + c0 < M) epi.template col<CH>(zb, m0 + c0, n, v, M - (m0 + c0));
     }
   } else {
-    // park the partial tile as P[token][feature] (the ring is idle: all MMAs have completed)
-    float* P = reinterpret_cast<float*>(ring_ptr);
+    // park the partial tile as P[token][feature] in the exchange area of this (tile, slice); the slices of
+    // a tile are summed in a fixed order, CTA ks finishing tokens [ks*per, (ks+1)*per)
+    const long long tile_id = ((long long)blockIdx.x * gridDim.y + blockIdx.y) * gridDim.z + (long long)zb * ksplit;
+    float* P = part + (tile_id + ks) * (TN * kGemmRowsW);
     constexpr int CH = TN < 32 ? 16 : 32;
 #pragma unroll 1
     for (int c0 = 0; c0 < TN; c0 += CH) {
@@ -137,24 +135,21 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
 #pragma unroll
       for (int j = 0; j < CH; ++j) P[(c0 + j) * kGemmRowsW + threadIdx.x] = v[j];
     }
-    cluster_sync_all();
-    // CTA ks finishes tokens [ks*per, (ks+1)*per): a thread sums four consecutive features of
-    // one token over the peers (16-byte loads, fixed peer order), warp w takes every 4th token.
+    cluster_sync_all();                                  // release / acquire: the peers' tiles are visible
     const int per = TN / ksplit;
     const int n4 = (threadIdx.x & 31) * 4;
     for (int t = ks * per + warp; t < (ks + 1) * per; t += 4) {
-      const uint32_t a = base + (uint32_t)(t * kGemmRowsW + n4) * 4u;
+      const float* a = part + tile_id * (TN * kGemmRowsW) + t * kGemmRowsW + n4;
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      float4 part[8];
+      float4 pv[8];
 #pragma unroll
       for (int peer = 0; peer < 8; ++peer)
-        if (peer < ksplit) part[peer] = ld_peer_f32x4(a, peer);
+        if (peer < ksplit) pv[peer] = __ldcg(reinterpret_cast<const float4*>(a + (long long)peer * (TN * kGemmRowsW)));
 #pragma unroll
       for (int peer = 0; peer < 8; ++peer)
-        if (peer < ksplit) { acc.x += part[peer].x; acc.y += part[peer].y; acc.z += part[peer].z; acc.w += part[peer].w; }
+        if (peer < ksplit) { acc.x += pv[peer].x; acc.y += pv[peer].y; acc.z += pv[peer].z; acc.w += pv[peer].w; }
       if (m0 + t < M && n0 + n4 < N) epi.vec4(zb, m0 + t, n0 + n4, acc);     // N is a multiple of 4
     }
-    cluster_sync_all();                                  // peers may still be reading this CTA's tile
   }
   tc_fence_before();
   __syncthreads();

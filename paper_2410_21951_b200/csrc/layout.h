@@ -11,6 +11,7 @@
 
 namespace vadusa {
 
+constexpr int64_t kGemmPartBytes = 32ll << 20;   // split-K exchange area (a launch needs tiles * ksplit * TN * 128 * 4 bytes)
 constexpr int kGenHostCap = 4096;     // most tokens per sequence vadusa_generate_host can return
 
 inline int64_t align_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
@@ -105,6 +106,7 @@ struct WorkspaceLayout {
   int64_t logits;                        // fp32 [M][vpad]
   int64_t hstar, logits_star;            // T [B][d], fp32 [B][vpad]
   int64_t z, dlogits;                    // T [heads][B][d], fp32 [heads][B][vpad]
+  int64_t gemm_part;                     // fp32 split-K exchange of the tensor-core products (kGemmPartBytes)
   int64_t gen_out, gen_len;              // int32 [B][kGenHostCap], int32 [B] (vadusa_generate_host staging)
   int64_t total;
 };
@@ -134,6 +136,7 @@ inline WorkspaceLayout workspace_layout(const vadusa_config* c) {
   w.logits = take(M * vp * 4);
   w.hstar = take(B * d * es); w.logits_star = take(B * vp * 4);
   w.z = take(hd * B * d * es); w.dlogits = take(hd * B * vp * 4);
+  w.gemm_part = take(kGemmPartBytes);
   w.gen_out = take(B * kGenHostCap * 4); w.gen_len = take(B * 4);
   w.total = off;
   return w;
