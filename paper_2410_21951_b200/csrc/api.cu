@@ -367,7 +367,8 @@ vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeVi
                             (const int32_t*)wsptr<int32_t>(ctx, ctx->ws.ctx_len),
                             (const int32_t*)wsptr<int32_t>(ctx, ctx->ws.nvalid),
                             (const int32_t*)(ctx->batch > 1 ? wsptr<int32_t>(ctx, ctx->ws.seq_order) : nullptr), tv, g, c.d_model,
-                            scale * 1.4426950408889634f, splits, reinterpret_cast<bf16*>(out), err_word(ctx)));
+                            scale * 1.4426950408889634f, splits, reinterpret_cast<bf16*>(out),
+                            wsptr<float>(ctx, ctx->ws.att_xch), err_word(ctx)));
       LAUNCH_CHECK();
       return VADUSA_OK;
     }

@@ -16,8 +16,8 @@
 //                  in TMEM columns 128..191; lanes r and r + 64 hold the two key-halves' sums
 // The scaling maximum of a row only moves when the page maximum exceeds it by more than 2^6
 // (p <= 64 is harmless in fp32 / bf16); then the row's accumulator is rescaled in TMEM.
-// At the end rows r and r + 64 are added; splits are merged over distributed shared memory in
-// a fixed order.  Warps: 0-3 softmax, warp 4 lane 0 TMA producer, warp 5 TMEM owner / MMA issuer.
+// At the end rows r and r + 64 are added; splits are merged through an exchange area in global
+// memory (L2) in a fixed order.  Warps: 0-3 softmax, warp 4 lane 0 TMA producer, warp 5 TMEM owner / MMA issuer.
 #pragma once
 #include "tc.cuh"
 
@@ -81,7 +81,7 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
     int layer, const int32_t* __restrict__ block_table, const int32_t* __restrict__ ctx_len,
     const int32_t* __restrict__ nvalid, const int32_t* __restrict__ order /*may be null*/, TreeView tree, KvGeom geom,
     int d_model, float scale_log2e, int splits,
-    bf16* __restrict__ out, uint32_t* err) {
+    bf16* __restrict__ out, float* __restrict__ xch /*split exchange area*/, uint32_t* err) {
   constexpr int S = kAttStages;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -325,19 +325,22 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
       }
     }
   } else {
-    // this split's result to shared memory (O [64][64], then l and m per row), then merge over the cluster
-    __syncthreads();
-    float* mp = xmax + 128;
+    // this split's result goes to its slot of the exchange area in global memory (it stays in L2):
+    // O [64 nodes][64] fp32, then the row sums l[64] and scaling maxima m[64]; the splits of one (head,
+    // sequence) meet at a cluster barrier and are merged in a fixed order
+    constexpr int kSlot = 64 * 64 + 128;
+    float* mine = xch + ((long long)(blockIdx.y * gridDim.x + blockIdx.x) * splits + split) * kSlot;
     if (tid < 64) {
+      float4* dst = reinterpret_cast<float4*>(mine + tid * 64);
 #pragma unroll
-      for (int e = 0; e < 64; ++e) Ox[tid * 64 + ((e + 4 * tid) & 63)] = o_acc[e];
-      lx[tid] = l_run;
-      mp[tid] = m_use;
+      for (int c = 0; c < 16; ++c) dst[c] = make_float4(o_acc[4 * c], o_acc[4 * c + 1], o_acc[4 * c + 2], o_acc[4 * c + 3]);
+      mine[64 * 64 + tid] = l_run;
+      mine[64 * 64 + 64 + tid] = m_use;
     }
-    cluster_sync_all();
-    const uint32_t ox_addr = ring, lx_addr = ring + kAttRingBytes, mp_addr = lx_addr + 128 * 4;
-    // CTA `split` finishes nodes [split*per_n, (split+1)*per_n): 16 threads per node, four
-    // consecutive features each (16-byte loads from every peer, fixed peer order)
+    cluster_sync_all();                        // release / acquire: the peers' slots are visible
+    // CTA `split` finishes nodes [split*per_n, (split+1)*per_n): 16 threads per node, four consecutive
+    // features each
+    const float* first = xch + (long long)(blockIdx.y * gridDim.x + blockIdx.x) * splits * kSlot;
     const int per_n = 64 / splits;
     if (tid < 128) {
       const int e4 = (tid & 15) * 4;
@@ -345,13 +348,13 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
         float mm[8], ll[8];
         float4 oo[8];
         float M = -INFINITY;
-        const int c0 = (e4 + 4 * n) & 63;         // rows are rotated by 4n columns (bank spread, 16-byte aligned)
 #pragma unroll
         for (int p = 0; p < 8; ++p)
           if (p < splits) {
-            mm[p] = ld_peer_f32(mp_addr + (uint32_t)n * 4u, p);
-            ll[p] = ld_peer_f32(lx_addr + (uint32_t)n * 4u, p);
-            oo[p] = ld_peer_f32x4(ox_addr + (uint32_t)(n * 64 + c0) * 4u, p);
+            const float* sl = first + (long long)p * kSlot;
+            mm[p] = __ldcg(sl + 64 * 64 + 64 + n);
+            ll[p] = __ldcg(sl + 64 * 64 + n);
+            oo[p] = __ldcg(reinterpret_cast<const float4*>(sl + n * 64 + e4));
             M = fmaxf(M, mm[p]);
           }
         float L = 0.f;
@@ -372,7 +375,6 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
         }
       }
     }
-    cluster_sync_all();
   }
   tc_fence_before();
   __syncthreads();

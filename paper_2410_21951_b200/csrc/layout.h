@@ -106,6 +106,7 @@ struct WorkspaceLayout {
   int64_t logits;                        // fp32 [M][vpad]
   int64_t hstar, logits_star;            // T [B][d], fp32 [B][vpad]
   int64_t z, dlogits;                    // T [heads][B][d], fp32 [heads][B][vpad]
+  int64_t att_xch;                       // fp32 split-KV exchange of the attention kernel: 296 slots of 64*64+128 floats
   int64_t gemm_part;                     // fp32 split-K exchange of the tensor-core products (kGemmPartBytes)
   int64_t gen_out, gen_len;              // int32 [B][kGenHostCap], int32 [B] (vadusa_generate_host staging)
   int64_t total;
@@ -136,6 +137,7 @@ inline WorkspaceLayout workspace_layout(const vadusa_config* c) {
   w.logits = take(M * vp * 4);
   w.hstar = take(B * d * es); w.logits_star = take(B * vp * 4);
   w.z = take(hd * B * d * es); w.dlogits = take(hd * B * vp * 4);
+  w.att_xch = take(296ll * (64 * 64 + 128) * 4);
   w.gemm_part = take(kGemmPartBytes);
   w.gen_out = take(B * kGenHostCap * 4); w.gen_len = take(B * 4);
   w.total = off;
