@@ -246,21 +246,25 @@ vadusa_status tensor_map(vadusa_ctx* ctx, const void* ptr, int rows, int K, int 
   return VADUSA_OK;
 }
 
-template <int TN, typename Epi>
+// X == nullptr with ln != nullptr: the LayerNorm-fused variant (the operand is made in the kernel).
+template <int TN, typename Epi, bool LN = false>
 vadusa_status launch_gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void* W, int w_rows, int M, int N, int K,
-                             int batches, long long x_z, long long w_z, int ksplit, const Epi& epi) {
+                             int batches, long long x_z, long long w_z, int ksplit, const Epi& epi,
+                             const LnFuse* ln = nullptr) {
   using Cfg = GemmTcCfg<TN>;
   static bool attr_done = false;
   if (!attr_done) {
-    CU(cudaFuncSetAttribute(gemm_tc_kernel<TN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemMax));
-    CU(cudaFuncSetAttribute(gemm_tc_kernel<TN, Epi>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+    CU(cudaFuncSetAttribute(gemm_tc_kernel<TN, Epi, LN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemMax));
+    CU(cudaFuncSetAttribute(gemm_tc_kernel<TN, Epi, LN>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+    CU(cudaFuncSetAttribute(gemm_tc_kernel<TN, Epi, LN>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
     attr_done = true;
   }
   const int chunks = K / kGemmBK / ksplit;
   const int smem = Cfg::smem_for(chunks, ksplit);
   const CUtensorMap *mw, *mx;
   if (vadusa_status s = tensor_map(ctx, W, w_rows, K, kGemmRowsW, batches, w_z, &mw)) return s;
-  if (vadusa_status s = tensor_map(ctx, X, M, K, TN, batches, x_z, &mx)) return s;
+  if (LN) mx = mw;                                       // unused by the kernel
+  else if (vadusa_status s = tensor_map(ctx, X, M, K, TN, batches, x_z, &mx)) return s;
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3((N + kGemmRowsW - 1) / kGemmRowsW, (M + TN - 1) / TN, batches * ksplit);
   lc.blockDim = dim3(128);
@@ -273,10 +277,48 @@ vadusa_status launch_gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void
   at[1].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = at; lc.numAttrs = 2;
   PROF(ctx, cls);
-  CU(cudaLaunchKernelEx(&lc, gemm_tc_kernel<TN, Epi>, *mw, *mx, M, N, chunks, ksplit, Cfg::stages_for(chunks),
-                        Cfg::ring_for(chunks, ksplit), epi, wsptr<float>(ctx, ctx->ws.gemm_part), err_word(ctx)));
+  CU(cudaLaunchKernelEx(&lc, gemm_tc_kernel<TN, Epi, LN>, *mw, *mx, M, N, chunks, ksplit, Cfg::stages_for(chunks),
+                        Cfg::ring_for(chunks, ksplit), epi, wsptr<float>(ctx, ctx->ws.gemm_part), err_word(ctx),
+                        ln ? *ln : LnFuse{}));
   LAUNCH_CHECK();
   return VADUSA_OK;
+}
+
+// K split of a product with `tiles` output tiles of tn tokens: about one CTA per SM streams weights.
+static int gemm_ksplit(int tiles, int chunks, int tn) {
+  int ksplit = 1;
+  while (ksplit < kGemmMaxSplit && tiles * ksplit < 148 && chunks % (ksplit * 2) == 0 && ksplit * 2 <= tn &&
+         (long long)tiles * ksplit * 2 * tn * kGemmRowsW * 4 <= kGemmPartBytes)
+    ksplit *= 2;
+  return ksplit;
+}
+
+// Does a residual product of N = d_model features over K inputs leave LayerNorm statistics for M
+// tokens?  (Its split-K epilogue does; the fused consumer handles at most 64 tokens and 8 groups.)
+static bool residual_leaves_stats(int M, int d, int K) {
+  if (M > 64 || d % 128 || d / 128 > 8 || K % kGemmBK) return false;
+  const int tn = M <= 16 ? 16 : M <= 32 ? 32 : 64;
+  return gemm_ksplit(d / kGemmRowsW, K / kGemmBK, tn) >= 2;
+}
+
+// LayerNorm(x) * W^T with the normalisation done inside the product kernel from the statistics the
+// producer of x left; applies when the tokens fit one tile of at most 64 and the K slices of the
+// cluster are 128 columns.  Returns false (nothing launched) when the shape does not qualify.
+template <typename Epi>
+bool gemm_tc_ln(vadusa_ctx* ctx, int cls, const float* x, const float* g, const float* b, const void* W, int w_rows,
+                int M, int N, int K, const Epi& epi, vadusa_status* st) {
+  if (M > 64 || K % 128 || K / 128 > 8) return false;
+  const int tn = M <= 16 ? 16 : M <= 32 ? 32 : 64;
+  const int tiles = (N + kGemmRowsW - 1) / kGemmRowsW, chunks = K / kGemmBK;
+  const int ksplit = gemm_ksplit(tiles, chunks, tn);
+  if (chunks / ksplit != 2) return false;
+  const LnFuse ln{x, g, b, wsptr<float2>(ctx, ctx->ws.ln_stats), K, ctx->cfg.ln_eps};
+  switch (tn) {
+    case 16: *st = launch_gemm_tc<16, Epi, true>(ctx, cls, nullptr, W, w_rows, M, N, K, 1, 0, 0, ksplit, epi, &ln); break;
+    case 32: *st = launch_gemm_tc<32, Epi, true>(ctx, cls, nullptr, W, w_rows, M, N, K, 1, 0, 0, ksplit, epi, &ln); break;
+    default: *st = launch_gemm_tc<64, Epi, true>(ctx, cls, nullptr, W, w_rows, M, N, K, 1, 0, 0, ksplit, epi, &ln); break;
+  }
+  return true;
 }
 
 // Tile width by token count; K split so that about one CTA per SM streams weights.
@@ -289,11 +331,7 @@ vadusa_status gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void* W, in
   int tn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 1024 ? 128 : 256;
   if (tn == 256 && ntiles_n * ((M + 255) / 256) * batches < 200) tn = 128;
   const int tiles = ((N + kGemmRowsW - 1) / kGemmRowsW) * ((M + tn - 1) / tn) * batches;
-  const int chunks = K / kGemmBK;
-  int ksplit = 1;
-  while (ksplit < 8 && tiles * ksplit < 148 && chunks % (ksplit * 2) == 0 && ksplit * 2 <= tn &&
-         (long long)tiles * ksplit * 2 * tn * kGemmRowsW * 4 <= kGemmPartBytes)
-    ksplit *= 2;
+  const int ksplit = gemm_ksplit(tiles, K / kGemmBK, tn);
   switch (tn) {
     case 16: return launch_gemm_tc<16>(ctx, cls, X, W, w_rows, M, N, K, batches, x_z, w_z, ksplit, epi);
     case 32: return launch_gemm_tc<32>(ctx, cls, X, W, w_rows, M, N, K, batches, x_z, w_z, ksplit, epi);
@@ -312,6 +350,14 @@ vadusa_status product(vadusa_ctx* ctx, int cls, const T* X, const T* W, int w_ro
     if (K % kGemmBK == 0) return gemm_tc(ctx, cls, X, W, w_rows, M, N, K, batches, x_z, w_z, epi);
   }
   return gemm<T>(ctx, cls, X, W, M, N, K, batches, x_z, w_z, epi);
+}
+
+// LayerNorm followed by a product, in one kernel where the shape allows (bf16 models, few tokens).
+template <typename T, typename Epi>
+bool ln_product(vadusa_ctx* ctx, int cls, const float* x, const float* g, const float* b, const T* W, int w_rows, int M,
+                int N, int K, const Epi& epi, vadusa_status* st) {
+  if constexpr (std::is_same<T, bf16>::value) return gemm_tc_ln(ctx, cls, x, g, b, W, w_rows, M, N, K, epi, st);
+  return false;
 }
 
 // KV splits of the tensor-core attention: enough CTAs for about two per SM even at batch 1.
@@ -421,29 +467,52 @@ vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* overri
     seq_order_kernel<<<1, 256, 0, ctx->stream>>>(ctx_len, nvalid, B, wsptr<int32_t>(ctx, ctx->ws.seq_order));
     LAUNCH_CHECK();
   }
+  // residual products that can leave LayerNorm statistics for the product after them (bf16 models, few tokens)
+  const bool tc = std::is_same<T, bf16>::value;
+  const bool stats_out = tc && residual_leaves_stats(M, d, d), stats_ffn = tc && residual_leaves_stats(M, d, f);
+  float2* stats = wsptr<float2>(ctx, ctx->ws.ln_stats);
+  bool have_stats = false;
   for (int l = 0; l < c.n_layers; ++l) {
     const LayerW& w = ctx->layers[l];
     T* pool = reinterpret_cast<T*>(c.kv_pool) + (long long)l * g.layer_stride;
-    vadusa_status s = layernorm<T>(ctx, x, w.ln1_g, w.ln1_b, a, M);
-    if (s) return s;
+    vadusa_status s = VADUSA_OK;
+    // (layer 0 reads the embedding kernel's x, which comes without statistics)
     EpiQKV<T> eq{w.bqkv, q, pool, wsptr<long long>(ctx, ctx->ws.kv_row), (long long)c.n_heads * kKvBlock * g.head_dim,
                  kKvBlock * g.head_dim, g.head_dim, d};
-    s = product<T>(ctx, K_GEMM_QKV, a, as<T>(w.wqkv), 3 * d, M, 3 * d, d, 1, 0, 0, eq);
+    if (!(have_stats && ln_product<T>(ctx, K_GEMM_QKV, x, w.ln1_g, w.ln1_b, as<T>(w.wqkv), 3 * d, M, 3 * d, d, eq, &s))) {
+      s = layernorm<T>(ctx, x, w.ln1_g, w.ln1_b, a, M);
+      if (s) return s;
+      s = product<T>(ctx, K_GEMM_QKV, a, as<T>(w.wqkv), 3 * d, M, 3 * d, d, 1, 0, 0, eq);
+    }
     if (s) return s;
     s = attention<T>(ctx, q, pool, tv, o);
     if (s) return s;
     if (attn_tap)
       CU(cudaMemcpyAsync(attn_tap + (long long)l * M * d, o, (size_t)M * d * sizeof(T), cudaMemcpyDeviceToDevice, ctx->stream));
-    EpiResidual eo{w.bo, x, d};
-    s = product<T>(ctx, K_GEMM_OUT, o, as<T>(w.wo), d, M, d, d, 1, 0, 0, eo);
-    if (s) return s;
-    s = layernorm<T>(ctx, x, w.ln2_g, w.ln2_b, a, M);
+    if (stats_out) {
+      EpiResidualStats eo{w.bo, x, d, stats};
+      s = product<T>(ctx, K_GEMM_OUT, o, as<T>(w.wo), d, M, d, d, 1, 0, 0, eo);
+      have_stats = true;
+    } else {
+      EpiResidual eo{w.bo, x, d};
+      s = product<T>(ctx, K_GEMM_OUT, o, as<T>(w.wo), d, M, d, d, 1, 0, 0, eo);
+    }
     if (s) return s;
     EpiRelu<T> e1{w.b1, mid, f};
-    s = product<T>(ctx, K_GEMM_FFN1, a, as<T>(w.w1), f, M, f, d, 1, 0, 0, e1);
+    if (!(have_stats && ln_product<T>(ctx, K_GEMM_FFN1, x, w.ln2_g, w.ln2_b, as<T>(w.w1), f, M, f, d, e1, &s))) {
+      s = layernorm<T>(ctx, x, w.ln2_g, w.ln2_b, a, M);
+      if (s) return s;
+      s = product<T>(ctx, K_GEMM_FFN1, a, as<T>(w.w1), f, M, f, d, 1, 0, 0, e1);
+    }
     if (s) return s;
-    EpiResidual e2{w.b2, x, d};
-    s = product<T>(ctx, K_GEMM_FFN2, mid, as<T>(w.w2), d, M, d, f, 1, 0, 0, e2);
+    if (stats_ffn) {
+      EpiResidualStats e2{w.b2, x, d, stats};
+      s = product<T>(ctx, K_GEMM_FFN2, mid, as<T>(w.w2), d, M, d, f, 1, 0, 0, e2);
+    } else {
+      EpiResidual e2{w.b2, x, d};
+      s = product<T>(ctx, K_GEMM_FFN2, mid, as<T>(w.w2), d, M, d, f, 1, 0, 0, e2);
+    }
+    have_stats = stats_ffn;
     if (s) return s;
   }
   if (vadusa_status s = layernorm<T>(ctx, x, ctx->lnf_g, ctx->lnf_b, hfinal, M)) return s;

@@ -97,6 +97,39 @@ struct EpiResidual {
   }
 };
 
+// EpiResidual that also leaves, per row and group of 128 features, the mean and the sum of squared
+// deviations of the updated residual stream (the LayerNorm-fused product reads them).  vec4 must be
+// called by all 32 lanes of a warp with the same row m and n = (a multiple of 128) + 4 * lane.
+struct EpiResidualStats {
+  const float* bias;
+  float* x;
+  int ld;
+  float2* stats;          // [rows][ld / 128]
+  __device__ __forceinline__ void operator()(int, int m, int n, float acc) const {
+    x[(long long)m * ld + n] += acc + bias[n];
+  }
+  __device__ __forceinline__ void vec4(int, int m, int n, float4 a) const {
+    const float4 b = *reinterpret_cast<const float4*>(bias + n);
+    float4* p = reinterpret_cast<float4*>(x + (long long)m * ld + n);
+    float4 v = *p;
+    v.x += a.x + b.x; v.y += a.y + b.y; v.z += a.z + b.z; v.w += a.w + b.w;
+    *p = v;
+    float s = (v.x + v.y) + (v.z + v.w);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    const float mu = s * (1.0f / 128.0f);
+    const float d0 = v.x - mu, d1 = v.y - mu, d2 = v.z - mu, d3 = v.w - mu;
+    float q = (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+    if ((threadIdx.x & 31) == 0) stats[(long long)m * (ld >> 7) + (n >> 7)] = make_float2(mu, q);
+  }
+  template <int CH>
+  __device__ __forceinline__ void col(int z, int m, int n, const float* v, int count) const {
+    EpiResidual{bias, x, ld}.template col<CH>(z, m, n, v, count);     // no statistics on this path
+  }
+};
+
 // first feed-forward matrix: relu(acc + bias) rounded to T
 template <typename T>
 struct EpiRelu {

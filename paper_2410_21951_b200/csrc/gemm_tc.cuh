@@ -16,6 +16,13 @@
 // owns the TMEM allocation and its lane 0 issues the MMAs, all four warps run the epilogue.
 // Weight tiles of the first stages are requested before griddepcontrol.wait, so under
 // programmatic dependent launch they stream while the producer of X is still running.
+//
+// LN variant (few tokens, one token tile, K slices of 128 columns): X is not read by TMA but
+// made in the kernel as LayerNorm(x) of the fp32 residual stream.  The kernel that last wrote
+// x (a residual product) left, per row and per group of 128 features, the mean and the sum of
+// squared deviations; they are combined exactly (Chan's formula for equal group sizes, fixed
+// order), and the normalised, scaled and shifted slice is written as bf16 straight into the
+// operand's swizzled shared-memory layout.
 #pragma once
 #include "tc.cuh"
 
@@ -24,6 +31,7 @@ namespace vadusa {
 constexpr int kGemmBK = 64;                 // K elements per stage (128 bytes per row: one swizzle row)
 constexpr int kGemmRowsW = 128;             // weight rows per tile
 constexpr int kGemmSmemBudget = 196 * 1024;
+constexpr int kGemmMaxSplit = 16;           // K slices per tile = cluster size (above 8: non-portable cluster size)
 
 template <int TN> struct GemmTcCfg {
   static constexpr int kStageBytes = kGemmRowsW * kGemmBK * 2 + TN * kGemmBK * 2;
@@ -40,11 +48,87 @@ template <int TN> struct GemmTcCfg {
   static constexpr int kSmemMax = kStages * kStageBytes + 1024 + 256;
 };
 
-template <int TN, typename Epi>
+// LayerNorm fused into the operand load (LN variant).
+struct LnFuse {
+  const float* x;        // [M][ld] fp32 rows to normalise
+  const float* g;        // [K] gain
+  const float* b;        // [K] shift
+  const float2* stats;   // [M][K/128] (mean, sum of squared deviations) of each group of 128 features
+  int ld;
+  float eps;
+};
+
+// All 128 threads; warp w owns rows [w*TN/4, (w+1)*TN/4) of the token tile.  The K slice is the
+// 128 columns starting at k0 (two operand tiles of 64 columns); lane l holds columns 4l .. 4l+3.
+// K / 128 <= 8 groups per row.
+template <int TN>
+__device__ __forceinline__ void ln_operand(const LnFuse& ln, int M, int K, int k0, uint32_t x_stage0, uint32_t stage_bytes) {
+  constexpr int RPW = TN / 4;                      // rows per warp (multiple of 4)
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nt = K >> 7;
+  // gain and shift are weights: fetched while the producer of x is still running
+  const float4 gg = __ldg(reinterpret_cast<const float4*>(ln.g + k0 + 4 * lane));
+  const float4 bb = __ldg(reinterpret_cast<const float4*>(ln.b + k0 + 4 * lane));
+  grid_dep_wait();
+  // every load that depends on the producer is issued before the first use: one round trip
+  float4 v[RPW];
+  float2 st[RPW / 4];
+  const int rr = lane >> 3, t = lane & 7;
+#pragma unroll
+  for (int it = 0; it < RPW / 4; ++it) {
+    const int row = warp * RPW + 4 * it + rr;
+    st[it] = (t < nt && row < M) ? __ldcg(ln.stats + (long long)row * nt + t) : make_float2(0.f, 0.f);
+  }
+#pragma unroll
+  for (int r = 0; r < RPW; ++r) {
+    const int row = warp * RPW + r;
+    v[r] = row < M ? __ldcg(reinterpret_cast<const float4*>(ln.x + (long long)row * ln.ld + k0 + 4 * lane))
+                   : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  // row statistics from the groups': lane = 8 * (row in a group of four rows) + feature group
+  float mean_g[RPW / 4], rstd_g[RPW / 4];
+  {
+#pragma unroll
+    for (int it = 0; it < RPW / 4; ++it) {
+      float m = st[it].x;
+#pragma unroll
+      for (int o = 4; o > 0; o >>= 1) m += __shfl_xor_sync(0xffffffffu, m, o);
+      m /= (float)nt;
+      const float dv = st[it].x - m;
+      float m2 = t < nt ? st[it].y + 128.0f * dv * dv : 0.f;
+#pragma unroll
+      for (int o = 4; o > 0; o >>= 1) m2 += __shfl_xor_sync(0xffffffffu, m2, o);
+      mean_g[it] = m;
+      rstd_g[it] = 1.0f / sqrtf(m2 / (float)K + ln.eps);
+    }
+  }
+  // normalise into the swizzled K-major operand tiles: column 4*lane is in tile lane/16, 16-byte unit
+  // (lane%16)/2 of the row (xor row%8), half lane&1
+  const uint32_t tile = x_stage0 + (uint32_t)(lane >> 4) * stage_bytes + (uint32_t)(lane & 1) * 8u;
+#pragma unroll
+  for (int r = 0; r < RPW; ++r) {
+    const int row = warp * RPW + r;
+    const float m = __shfl_sync(0xffffffffu, mean_g[r / 4], 8 * (r % 4));
+    const float rs = __shfl_sync(0xffffffffu, rstd_g[r / 4], 8 * (r % 4));
+    uint32_t lo = 0u, hi = 0u;
+    if (row < M) {
+      const __nv_bfloat162 p0 = __floats2bfloat162_rn((v[r].x - m) * rs * gg.x + bb.x, (v[r].y - m) * rs * gg.y + bb.y);
+      const __nv_bfloat162 p1 = __floats2bfloat162_rn((v[r].z - m) * rs * gg.z + bb.z, (v[r].w - m) * rs * gg.w + bb.w);
+      lo = *reinterpret_cast<const uint32_t*>(&p0);
+      hi = *reinterpret_cast<const uint32_t*>(&p1);
+    }
+    const uint32_t unit = (uint32_t)((lane & 15) >> 1) ^ (uint32_t)(row & 7);
+    asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(tile + (uint32_t)row * 128u + (unit << 4)), "r"(lo), "r"(hi));
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tensor-core reads
+}
+
+template <int TN, typename Epi, bool LN = false>
 __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW,
                                                       const __grid_constant__ CUtensorMap tmX, int M, int N,
                                                       int chunks_per_split, int ksplit, int S, int ring_bytes,
-                                                      Epi epi, float* __restrict__ part /*split-K exchange*/, uint32_t* err) {
+                                                      Epi epi, float* __restrict__ part /*split-K exchange*/, uint32_t* err,
+                                                      LnFuse ln = LnFuse{}) {
   using Cfg = GemmTcCfg<TN>;
   constexpr uint32_t kWBytes = kGemmRowsW * kGemmBK * 2, kXBytes = TN * kGemmBK * 2;
   extern __shared__ uint8_t smem_raw[];
@@ -71,25 +155,34 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *holder_ptr;
-
   if (warp == 0 && lane == 0) {
     // ---- TMA producer
     const int pre = nchunks < S ? nchunks : S;
     for (int i = 0; i < pre; ++i) {                      // weights do not depend on the upstream kernel
-      mbar_expect_tx(full0 + 8 * i, kWBytes + kXBytes);
+      mbar_expect_tx(full0 + 8 * i, LN ? kWBytes : kWBytes + kXBytes);
       tma_load_3d(base + i * Cfg::kStageBytes, &tmW, full0 + 8 * i, (chunk0 + i) * kGemmBK, n0, zb);
     }
-    grid_dep_wait();
-    for (int i = 0; i < pre; ++i)
-      tma_load_3d(base + i * Cfg::kStageBytes + kWBytes, &tmX, full0 + 8 * i, (chunk0 + i) * kGemmBK, m0, zb);
-    for (int i = pre; i < nchunks; ++i) {
-      const int s = i % S;
-      if (!mbar_wait(empty0 + 8 * s, ((i / S) - 1) & 1, err)) break;
-      mbar_expect_tx(full0 + 8 * s, kWBytes + kXBytes);
-      tma_load_3d(base + s * Cfg::kStageBytes, &tmW, full0 + 8 * s, (chunk0 + i) * kGemmBK, n0, zb);
-      tma_load_3d(base + s * Cfg::kStageBytes + kWBytes, &tmX, full0 + 8 * s, (chunk0 + i) * kGemmBK, m0, zb);
+    if constexpr (!LN) {
+      grid_dep_wait();
+      for (int i = 0; i < pre; ++i)
+        tma_load_3d(base + i * Cfg::kStageBytes + kWBytes, &tmX, full0 + 8 * i, (chunk0 + i) * kGemmBK, m0, zb);
+      for (int i = pre; i < nchunks; ++i) {
+        const int s = i % S;
+        if (!mbar_wait(empty0 + 8 * s, ((i / S) - 1) & 1, err)) break;
+        mbar_expect_tx(full0 + 8 * s, kWBytes + kXBytes);
+        tma_load_3d(base + s * Cfg::kStageBytes, &tmW, full0 + 8 * s, (chunk0 + i) * kGemmBK, n0, zb);
+        tma_load_3d(base + s * Cfg::kStageBytes + kWBytes, &tmX, full0 + 8 * s, (chunk0 + i) * kGemmBK, m0, zb);
+      }
     }
-  } else if (warp == 1 && lane == 0) {
+  }
+  if constexpr (LN) {
+    // every chunk of the slice has a stage of its own (nchunks <= S): all threads build the X tiles
+    __syncwarp();
+    if constexpr (TN <= 64)                          // (waits for the producer of x inside)
+      ln_operand<TN>(ln, M, nchunks * ksplit * kGemmBK, chunk0 * kGemmBK, base + kWBytes, Cfg::kStageBytes);
+    __syncthreads();
+  }
+  if (warp == 1 && lane == 0) {
     // ---- MMA issuer
     constexpr uint32_t idesc = umma_idesc_bf16(kGemmRowsW, TN < 16 ? 16 : TN);
     for (int i = 0; i < nchunks; ++i) {
@@ -141,12 +234,12 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
     for (int t = ks * per + warp; t < (ks + 1) * per; t += 4) {
       const float* a = part + tile_id * (TN * kGemmRowsW) + t * kGemmRowsW + n4;
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      float4 pv[8];
+      float4 pv[kGemmMaxSplit];
 #pragma unroll
-      for (int peer = 0; peer < 8; ++peer)
+      for (int peer = 0; peer < kGemmMaxSplit; ++peer)
         if (peer < ksplit) pv[peer] = __ldcg(reinterpret_cast<const float4*>(a + (long long)peer * (TN * kGemmRowsW)));
 #pragma unroll
-      for (int peer = 0; peer < 8; ++peer)
+      for (int peer = 0; peer < kGemmMaxSplit; ++peer)
         if (peer < ksplit) { acc.x += pv[peer].x; acc.y += pv[peer].y; acc.z += pv[peer].z; acc.w += pv[peer].w; }
       if (m0 + t < M && n0 + n4 < N) epi.vec4(zb, m0 + t, n0 + n4, acc);     // N is a multiple of 4
     }

@@ -11,6 +11,7 @@
 
 namespace vadusa {
 
+constexpr int64_t kLnStatsBytes = 64 * 8 * 8;     // [token <= 64][feature group <= 8] (mean, sum of squared deviations)
 constexpr int64_t kGemmPartBytes = 32ll << 20;   // split-K exchange area (a launch needs tiles * ksplit * TN * 128 * 4 bytes)
 constexpr int kGenHostCap = 4096;     // most tokens per sequence vadusa_generate_host can return
 
@@ -108,6 +109,7 @@ struct WorkspaceLayout {
   int64_t z, dlogits;                    // T [heads][B][d], fp32 [heads][B][vpad]
   int64_t att_xch;                       // fp32 split-KV exchange of the attention kernel: 296 slots of 64*64+128 floats
   int64_t gemm_part;                     // fp32 split-K exchange of the tensor-core products (kGemmPartBytes)
+  int64_t ln_stats;                      // per-group LayerNorm statistics for the fused products (kLnStatsBytes)
   int64_t gen_out, gen_len;              // int32 [B][kGenHostCap], int32 [B] (vadusa_generate_host staging)
   int64_t total;
 };
@@ -139,6 +141,7 @@ inline WorkspaceLayout workspace_layout(const vadusa_config* c) {
   w.z = take(hd * B * d * es); w.dlogits = take(hd * B * vp * 4);
   w.att_xch = take(296ll * (64 * 64 + 128) * 4);
   w.gemm_part = take(kGemmPartBytes);
+  w.ln_stats = take(kLnStatsBytes);
   w.gen_out = take(B * kGenHostCap * 4); w.gen_len = take(B * 4);
   w.total = off;
   return w;
