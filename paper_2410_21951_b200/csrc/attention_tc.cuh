@@ -210,11 +210,15 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
 #pragma unroll
         for (int j = 0; j < 32; ++j) mx = fmaxf(mx, sc[j]);
       } else {
+        // bit j of vis: key key0 + j is visible (context, or an ancestor-or-self tree node; the ancestor
+        // word has no bits at or above the node count).  Selects, not branches: the rows of a warp differ.
+        const int rel = key0 - ctx;           // > -32 here
+        uint32_t vis;
+        if (rel >= 0) vis = rel < 64 ? (uint32_t)(amask >> rel) : 0u;
+        else vis = ((1u << (-rel)) - 1u) | (uint32_t)(amask << (-rel));
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
-          const int p = key0 + j;
-          const bool vis = p < ctx || (p < total && ((amask >> ((p - ctx) & 63)) & 1ull));
-          sc[j] = vis ? sc[j] : -INFINITY;
+          sc[j] = ((vis >> j) & 1u) ? sc[j] : -INFINITY;
           mx = fmaxf(mx, sc[j]);
         }
       }
