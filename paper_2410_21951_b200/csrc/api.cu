@@ -309,9 +309,9 @@ bool gemm_tc_ln(vadusa_ctx* ctx, int cls, const float* x, const float* g, const 
                 int M, int N, int K, const Epi& epi, vadusa_status* st) {
   if (M > 64 || K % 128 || K / 128 > 8) return false;
   const int tn = M <= 16 ? 16 : M <= 32 ? 32 : 64;
-  const int tiles = (N + kGemmRowsW - 1) / kGemmRowsW, chunks = K / kGemmBK;
-  const int ksplit = gemm_ksplit(tiles, chunks, tn);
-  if (chunks / ksplit != 2) return false;
+  const int tiles = (N + kGemmRowsW - 1) / kGemmRowsW;
+  const int ksplit = K / 128;                            // one CTA of the cluster per group of 128 columns
+  if (ksplit < 2 || ksplit > tn || (long long)tiles * ksplit * tn * kGemmRowsW * 4 > kGemmPartBytes) return false;
   const LnFuse ln{x, g, b, wsptr<float2>(ctx, ctx->ws.ln_stats), K, ctx->cfg.ln_eps};
   switch (tn) {
     case 16: *st = launch_gemm_tc<16, Epi, true>(ctx, cls, nullptr, W, w_rows, M, N, K, 1, 0, 0, ksplit, epi, &ln); break;

@@ -133,16 +133,35 @@ __global__ void __launch_bounds__(256) draft_select_kernel(
     return;
   }
   const float* row = dlogits + ((long long)head * batch + b) * ld;
+  // the row is read once: each thread keeps its first kCache entries in registers (taken ones are
+  // struck out there); entries beyond kCache * blockDim.x are re-read and filtered by the last pick
+  constexpr int kCache = 8;
+  float cv[kCache];
+#pragma unroll
+  for (int c = 0; c < kCache; ++c) {
+    const int j = threadIdx.x + c * blockDim.x;
+    cv[c] = j < vocab ? masked_logit(row[j], j, sp) : -INFINITY;
+  }
+  const int cached = kCache * blockDim.x;
+  unsigned taken = 0u;
   Best bound{INFINITY, -1};
   for (int r = 0; r < k; ++r) {
     Best mine{0.f, -1};
-    for (int j = threadIdx.x; j < vocab; j += blockDim.x) {
+#pragma unroll
+    for (int c = 0; c < kCache; ++c) {
+      const int j = threadIdx.x + c * blockDim.x;
+      if (j < vocab && !((taken >> c) & 1u)) mine = better(mine, Best{cv[c], j});
+    }
+    for (int j = cached + threadIdx.x; j < vocab; j += blockDim.x) {
       const float v = masked_logit(row[j], j, sp);
       if (bound.i >= 0 && !precedes(bound.v, bound.i, v, j)) continue;
       mine = better(mine, Best{v, j});
     }
     const Best top = block_first(mine, bscratch);
     if (threadIdx.x == 0) topk[((long long)b * n_heads + head) * k + r] = top.i < 0 ? 0 : top.i;
+#pragma unroll
+    for (int c = 0; c < kCache; ++c)
+      if (top.i == threadIdx.x + c * blockDim.x) taken |= 1u << c;
     bound = top;
   }
 }

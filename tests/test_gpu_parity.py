@@ -73,6 +73,22 @@ def test_toy_lockstep_prefill_and_kv(dtype):
     g.check()
 
 
+@pytest.mark.parametrize("nodes", [10, 24, 48])
+def test_bf16_small_token_counts_take_the_layernorm_fused_products(nodes):
+    """d_model 256 (two groups of 128 features), one sequence: the token count selects the 16-, 32- and
+    64-wide tiles of the products that normalise their own operand from the producer's statistics;
+    prefill tails exercise short tiles as well."""
+    wl = W.toy_workload(dtype="bf16", d_model=256, n_heads=4, d_ffn=512, vocab=203, tree_nodes=nodes,
+                        tree_caps=(6, 3, 2), tau=3, temperature=1.0, batch=1, phoneme_len=(13, 13), prompt_len=70,
+                        index=14)
+    w, model, tpl, g, table = _setup(wl, 5, range(1))
+    states, _ = _prefill_both(wl, g, table, model, range(1), oracle_chunk=29)
+    so, sg = _sampling(wl)
+    rep = lockstep(g, table, model, states, tpl, so, sg, 5, "bf16", oracle_mode="memo", check_attn=True)
+    assert rep.iterations == 5 and rep.accept_checked + rep.accept_undecidable == 5
+    g.check()
+
+
 @pytest.mark.parametrize("dtype,tau,temperature,top_p,rule", [("fp32", 2, 0.9, 0.8, 0), ("fp32", 3, 1.0, 1.0, 1),
                                                                ("bf16", 5, 0.8, 1.0, 0), ("fp32", 1, 0.0, 1.0, 0)])
 def test_toy_planted_paths_are_accepted(dtype, tau, temperature, top_p, rule):
