@@ -232,16 +232,19 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
     const int per = TN / ksplit;
     const int n4 = (threadIdx.x & 31) * 4;
     for (int t = ks * per + warp; t < (ks + 1) * per; t += 4) {
-      const float* a = part + tile_id * (TN * kGemmRowsW) + t * kGemmRowsW + n4;
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      float4 pv[kGemmMaxSplit];
+      // (one block, so that the epilogue's own loads can be issued beside the peers')
+      if (m0 + t < M && n0 + n4 < N) {                                        // N is a multiple of 4
+        const float* a = part + tile_id * (TN * kGemmRowsW) + t * kGemmRowsW + n4;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 pv[kGemmMaxSplit];
 #pragma unroll
-      for (int peer = 0; peer < kGemmMaxSplit; ++peer)
-        if (peer < ksplit) pv[peer] = __ldcg(reinterpret_cast<const float4*>(a + (long long)peer * (TN * kGemmRowsW)));
+        for (int peer = 0; peer < kGemmMaxSplit; ++peer)
+          if (peer < ksplit) pv[peer] = __ldcg(reinterpret_cast<const float4*>(a + (long long)peer * (TN * kGemmRowsW)));
 #pragma unroll
-      for (int peer = 0; peer < kGemmMaxSplit; ++peer)
-        if (peer < ksplit) { acc.x += pv[peer].x; acc.y += pv[peer].y; acc.z += pv[peer].z; acc.w += pv[peer].w; }
-      if (m0 + t < M && n0 + n4 < N) epi.vec4(zb, m0 + t, n0 + n4, acc);     // N is a multiple of 4
+        for (int peer = 0; peer < kGemmMaxSplit; ++peer)
+          if (peer < ksplit) { acc.x += pv[peer].x; acc.y += pv[peer].y; acc.z += pv[peer].z; acc.w += pv[peer].w; }
+        epi.vec4(zb, m0 + t, n0 + n4, acc);
+      }
     }
   }
   tc_fence_before();
