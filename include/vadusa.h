@@ -50,7 +50,7 @@
 extern "C" {
 #endif
 
-#define VADUSA_ABI_VERSION 1u
+#define VADUSA_ABI_VERSION 2u
 #define VADUSA_MAX_TREE_NODES 64   /* one 64-bit ancestor word per node */
 #define VADUSA_MAX_DRAFT_TOPK 16
 #define VADUSA_MAX_DEPTH 15        /* a root path has at most 16 nodes */
@@ -81,6 +81,10 @@ typedef struct {
   int32_t max_tree_nodes;      /* <= VADUSA_MAX_TREE_NODES */
   int32_t kv_block;            /* tokens per KV block; must be 64 */
   int32_t max_blocks_per_seq;  /* row length of the block table */
+  int32_t prefill_rows;        /* chunks of max_tree_nodes prefix tokens that one prefill pass scores together
+                                  (sizes the activation buffers with max(max_batch, prefill_rows) rows of
+                                  max_tree_nodes tokens); 0 = max_batch; <= 4096 */
+  int32_t reserved0;           /* must be 0 */
   int64_t kv_num_blocks;       /* blocks per layer in the pool */
   float ln_eps;
   int32_t device;              /* CUDA device ordinal */
@@ -168,10 +172,15 @@ vadusa_status vadusa_begin(vadusa_ctx *ctx, int32_t batch, const int32_t *block_
                            const int32_t *h_ctx_len);
 
 /* Feeds the prefix [phonemes ; prompt speech tokens] of every sequence through the
- * model (paper Fig. 1a), in chunks, each chunk scored as a chain-shaped tree whose
- * nodes are all accepted.  h_tokens: host int32 [batch][stride], phoneme p written
- * as vocab + p; h_len: host int32 [batch].  Leaves the hidden state and base-head
- * logits of the last prefix token as the start of decoding. */
+ * model (paper Fig. 1a) behind whatever the cache already holds.  The prefixes are cut
+ * into chunks of max_tree_nodes tokens; a chunk is scored as a chain-shaped tree (all
+ * nodes accepted) whose context is everything before it, and up to max(max_batch,
+ * prefill_rows) chunks -- of one sequence or of several -- go through the model in one
+ * pass: every chunk's K/V rows are in the cache before the pass's attention reads
+ * them, so later chunks of a sequence see the earlier ones of the same pass.
+ * h_tokens: host int32 [batch][stride], phoneme p written as vocab + p; h_len: host
+ * int32 [batch].  Leaves the hidden state and base-head logits of the last prefix
+ * token as the start of decoding.  Synchronises the stream. */
 vadusa_status vadusa_prefill(vadusa_ctx *ctx, const int32_t *h_tokens, const int32_t *h_len, int32_t stride);
 
 /* Microbenchmark / test entry: sets the carried state directly.  hstar: [batch][d_model]

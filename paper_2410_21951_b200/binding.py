@@ -14,7 +14,7 @@ import numpy as np
 from . import build as _build
 
 MAX_PATH = 16          # VADUSA_MAX_DEPTH + 1
-ABI_VERSION = 1
+ABI_VERSION = 2
 
 STATUS = {0: "OK", 1: "EINVAL", 2: "ENOMEM", 3: "ECUDA", 4: "ECAPACITY", 5: "ESTATE", 6: "ETIMEOUT"}
 
@@ -31,6 +31,7 @@ class Config(C.Structure):
                 ("vocab", C.c_int32), ("n_phonemes", C.c_int32), ("max_pos", C.c_int32), ("dtype", C.c_int32),
                 ("n_draft_heads", C.c_int32), ("draft_topk", C.c_int32), ("max_batch", C.c_int32),
                 ("max_tree_nodes", C.c_int32), ("kv_block", C.c_int32), ("max_blocks_per_seq", C.c_int32),
+                ("prefill_rows", C.c_int32), ("reserved0", C.c_int32),
                 ("kv_num_blocks", C.c_int64), ("ln_eps", C.c_float), ("device", C.c_int32),
                 ("kv_pool", C.c_void_p), ("kv_pool_bytes", C.c_int64),
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_int64), ("stream", C.c_void_p)]
@@ -118,7 +119,7 @@ def lib() -> C.CDLL:
 
 
 def make_config(shape, max_batch: int, max_tree_nodes: int, max_blocks_per_seq: int, kv_num_blocks: int,
-                draft_topk: int = 10, device: int = 0) -> Config:
+                draft_topk: int = 10, device: int = 0, prefill_rows: int = 0) -> Config:
     """Config from a model shape (any object with the fields of workloads.ModelShape)."""
     c = Config()
     c.struct_size, c.abi_version = C.sizeof(Config), ABI_VERSION
@@ -129,6 +130,7 @@ def make_config(shape, max_batch: int, max_tree_nodes: int, max_blocks_per_seq: 
     c.max_batch, c.max_tree_nodes, c.kv_block = max_batch, max_tree_nodes, 64
     c.max_blocks_per_seq, c.kv_num_blocks = max_blocks_per_seq, kv_num_blocks
     c.ln_eps, c.device = shape.ln_eps, device
+    c.prefill_rows, c.reserved0 = prefill_rows, 0
     return c
 
 
@@ -193,7 +195,8 @@ class Vadusa:
 
     def __init__(self, shape, weights: Dict[str, np.ndarray], max_batch: int, max_tree_nodes: int,
                  max_blocks_per_seq: int, kv_num_blocks: int, draft_topk: int = 10, device: int = 0,
-                 stream=None):
+                 stream=None, prefill_rows: int = 16):
+        """prefill_rows: prefix chunks (of max_tree_nodes tokens) scored per prefill pass."""
         import torch
         self.torch = torch
         if not torch.cuda.is_available():
@@ -201,7 +204,8 @@ class Vadusa:
         self.L = lib()
         self.shape = shape
         self.dev = torch.device("cuda", device)
-        self.cfg = make_config(shape, max_batch, max_tree_nodes, max_blocks_per_seq, kv_num_blocks, draft_topk, device)
+        self.cfg = make_config(shape, max_batch, max_tree_nodes, max_blocks_per_seq, kv_num_blocks, draft_topk, device,
+                               prefill_rows)
         self.tdtype = torch.bfloat16 if self.cfg.dtype == 1 else torch.float32
         self.blob = torch.from_numpy(pack_weights(self.cfg, weights)).to(self.dev)
         self.kv_pool = torch.zeros(self.L.vadusa_kv_pool_bytes(C.byref(self.cfg)), dtype=torch.uint8, device=self.dev)

@@ -230,19 +230,26 @@ __global__ void __launch_bounds__(256) commit_kernel(
   }
 }
 
-// Prefill chunks are chains whose nodes are all kept and already sit in their final
-// slots: advance the context and carry the last node's state.  grid = batch.
+// Prefill bookkeeping.  gather: row r of the pass gets the block-table row of its sequence.
+__global__ void prefill_gather_kernel(const int32_t* __restrict__ block_table, const int32_t* __restrict__ seq_of,
+                                      int max_blocks, int32_t* __restrict__ out) {
+  const int r = blockIdx.x, b = seq_of[r];
+  for (int i = threadIdx.x; i < max_blocks; i += blockDim.x) out[(long long)r * max_blocks + i] = block_table[(long long)b * max_blocks + i];
+}
+
+// finish: the row holding the last chunk of sequence b carries that sequence's state forward: the
+// hidden state and base-head logits of its last token, and the new context length.  grid = rows.
 template <typename T>
-__global__ void prefill_advance_kernel(SeqState st, int n_nodes, const T* __restrict__ hfinal, int d_model,
-                                       const float* __restrict__ logits, int ld, T* __restrict__ hstar,
-                                       float* __restrict__ logits_star) {
-  const int b = blockIdx.x, nv = st.nvalid[b];
-  if (nv == 0) return;
-  const long long m = (long long)b * n_nodes + nv - 1;
+__global__ void prefill_finish_kernel(const int32_t* __restrict__ row_ctx, const int32_t* __restrict__ row_nvalid,
+                                      const int32_t* __restrict__ row_last, int n_nodes, const T* __restrict__ hfinal,
+                                      int d_model, const float* __restrict__ logits, int ld, T* __restrict__ hstar,
+                                      float* __restrict__ logits_star, int32_t* __restrict__ ctx_len) {
+  const int r = blockIdx.x, b = row_last[r], nv = row_nvalid[r];
+  if (b < 0 || nv == 0) return;
+  const long long m = (long long)r * n_nodes + nv - 1;
   for (int i = threadIdx.x; i < d_model; i += blockDim.x) hstar[(long long)b * d_model + i] = hfinal[m * d_model + i];
   for (int i = threadIdx.x; i < ld; i += blockDim.x) logits_star[(long long)b * ld + i] = logits[m * ld + i];
-  __syncthreads();
-  if (threadIdx.x == 0) st.ctx_len[b] += nv;
+  if (threadIdx.x == 0) ctx_len[b] = row_ctx[r] + nv;
 }
 
 }  // namespace vadusa

@@ -570,39 +570,75 @@ vadusa_status accept_commit(vadusa_ctx* ctx, const SamplingDev& sp, const int32_
   return VADUSA_OK;
 }
 
+// While alive, the model's passes see `rows` rows described by the given arrays instead of the batch.
+struct RowsView {
+  vadusa_ctx* c;
+  int batch; const int32_t* table; int64_t ctx_len, nvalid;
+  RowsView(vadusa_ctx* ctx, int rows, const int32_t* block_table, int64_t ctx_len_off, int64_t nvalid_off)
+      : c(ctx), batch(ctx->batch), table(ctx->block_table), ctx_len(ctx->ws.ctx_len), nvalid(ctx->ws.nvalid) {
+    ctx->batch = rows; ctx->block_table = block_table; ctx->ws.ctx_len = ctx_len_off; ctx->ws.nvalid = nvalid_off;
+  }
+  ~RowsView() { c->batch = batch; c->block_table = table; c->ws.ctx_len = ctx_len; c->ws.nvalid = nvalid; }
+};
+
 template <typename T>
 vadusa_status prefill(vadusa_ctx* ctx, const int32_t* h_tokens, const int32_t* h_len, int stride) {
   const vadusa_config& c = ctx->cfg;
-  const int B = ctx->batch, N = c.max_tree_nodes, vp = vpad(&c);
+  const int B = ctx->batch, N = c.max_tree_nodes, vp = vpad(&c), R = pass_rows(&c);
   int longest = 0;
   for (int b = 0; b < B; ++b) {
     if (h_len[b] < 1 || h_len[b] > stride) return fail(ctx, VADUSA_EINVAL, "prefix length of sequence %d out of range", b);
     longest = h_len[b] > longest ? h_len[b] : longest;
   }
-  int32_t* d_nvalid = wsptr<int32_t>(ctx, ctx->ws.nvalid);
-  int32_t* d_stage = wsptr<int32_t>(ctx, ctx->ws.stage_tokens);
-  std::vector<int32_t> stage((size_t)B * N), nv(B);
-  const TreeView tv = tree_of(ctx, true);
-  SeqState st = state_of(ctx, nullptr, 0, 0);
-  for (int s0 = 0; s0 < longest; s0 += N) {
-    for (int b = 0; b < B; ++b) {
-      int n = h_len[b] - s0;
-      n = n < 0 ? 0 : (n > N ? N : n);
-      nv[b] = n;
-      for (int i = 0; i < N; ++i) stage[(size_t)b * N + i] = i < n ? h_tokens[(size_t)b * stride + s0 + i] : 0;
+  // what the cache holds already
+  std::vector<int32_t> base(B);
+  CU(cudaMemcpyAsync(base.data(), ctx->wsp + ctx->ws.ctx_len, B * sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  // chunks in sequence order, so that a chunk never precedes an earlier chunk of its sequence
+  struct Chunk { int b, s0, n, last; };
+  std::vector<Chunk> chunks;
+  for (int b = 0; b < B; ++b)
+    for (int s0 = 0; s0 < h_len[b]; s0 += N) {
+      const int n = h_len[b] - s0 < N ? h_len[b] - s0 : N;
+      chunks.push_back({b, s0, n, s0 + n == h_len[b] ? b : -1});
     }
-    CU(cudaMemcpyAsync(d_nvalid, nv.data(), B * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream));
-    CU(cudaMemcpyAsync(d_stage, stage.data(), (size_t)B * N * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream));
-    CU(cudaStreamSynchronize(ctx->stream));   // the staging vectors are reused by the next chunk
-    vadusa_status s = forward<T>(ctx, tv, d_stage, nullptr);
-    if (s) return s;
-    ctx->ctx_bound += (longest - s0) < N ? (longest - s0) : N;
-    prefill_advance_kernel<T><<<B, 256, 0, ctx->stream>>>(st, N, wsptr<T>(ctx, ctx->ws.hfinal), c.d_model,
-                                                          wsptr<float>(ctx, ctx->ws.logits), vp,
-                                                          wsptr<T>(ctx, ctx->ws.hstar),
-                                                          wsptr<float>(ctx, ctx->ws.logits_star));
+  int32_t* d_stage = wsptr<int32_t>(ctx, ctx->ws.stage_tokens);
+  int32_t* d_ctx = wsptr<int32_t>(ctx, ctx->ws.pf_ctx_len);
+  int32_t* d_nv = wsptr<int32_t>(ctx, ctx->ws.pf_nvalid);
+  int32_t* d_seq = wsptr<int32_t>(ctx, ctx->ws.pf_seq);
+  int32_t* d_last = wsptr<int32_t>(ctx, ctx->ws.pf_last);
+  int32_t* d_table = wsptr<int32_t>(ctx, ctx->ws.pf_block_table);
+  int32_t* real_ctx_len = wsptr<int32_t>(ctx, ctx->ws.ctx_len);
+  const int32_t* real_table = ctx->block_table;
+  std::vector<int32_t> stage((size_t)R * N), v_ctx(R), v_nv(R), v_seq(R), v_last(R);
+  const TreeView tv = tree_of(ctx, true);
+  for (size_t c0 = 0; c0 < chunks.size(); c0 += R) {
+    const int rows = (int)(chunks.size() - c0 < (size_t)R ? chunks.size() - c0 : R);
+    for (int r = 0; r < rows; ++r) {
+      const Chunk& ch = chunks[c0 + r];
+      v_ctx[r] = base[ch.b] + ch.s0; v_nv[r] = ch.n; v_seq[r] = ch.b; v_last[r] = ch.last;
+      for (int i = 0; i < N; ++i) stage[(size_t)r * N + i] = i < ch.n ? h_tokens[(size_t)ch.b * stride + ch.s0 + i] : 0;
+    }
+    CU(cudaMemcpyAsync(d_ctx, v_ctx.data(), rows * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaMemcpyAsync(d_nv, v_nv.data(), rows * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaMemcpyAsync(d_seq, v_seq.data(), rows * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaMemcpyAsync(d_last, v_last.data(), rows * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaMemcpyAsync(d_stage, stage.data(), (size_t)rows * N * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));   // the staging vectors are reused by the next pass
+    prefill_gather_kernel<<<rows, 128, 0, ctx->stream>>>(real_table, d_seq, c.max_blocks_per_seq, d_table);
+    LAUNCH_CHECK();
+    {
+      RowsView view(ctx, rows, d_table, ctx->ws.pf_ctx_len, ctx->ws.pf_nvalid);
+      if (vadusa_status s = forward<T>(ctx, tv, d_stage, nullptr)) return s;
+    }
+    prefill_finish_kernel<T><<<rows, 256, 0, ctx->stream>>>(d_ctx, d_nv, d_last, N, wsptr<T>(ctx, ctx->ws.hfinal), c.d_model,
+                                                            wsptr<float>(ctx, ctx->ws.logits), vp,
+                                                            wsptr<T>(ctx, ctx->ws.hstar),
+                                                            wsptr<float>(ctx, ctx->ws.logits_star), real_ctx_len);
     LAUNCH_CHECK();
   }
+  ctx->ctx_bound += longest;
+  CU(cudaStreamSynchronize(ctx->stream));
   return VADUSA_OK;
 }
 

@@ -40,12 +40,16 @@ inline const char* check_config(const vadusa_config* c) {
   if (c->max_tree_nodes < 1 || c->max_tree_nodes > VADUSA_MAX_TREE_NODES) return "max_tree_nodes out of range";
   if (c->kv_block != 64) return "kv_block must be 64";
   if (c->max_blocks_per_seq < 1) return "max_blocks_per_seq must be positive";
+  if (c->prefill_rows < 0 || c->prefill_rows > 4096) return "prefill_rows out of range";
+  if (c->reserved0 != 0) return "reserved0 must be 0";
   if (c->kv_num_blocks < 1) return "kv_num_blocks must be positive";
   if (!(c->ln_eps > 0.f)) return "ln_eps must be positive";
   return nullptr;
 }
 
 inline int esize(const vadusa_config* c) { return c->dtype == 1 ? 2 : 4; }
+// Rows (sequences, or prefix chunks during prefill) of max_tree_nodes tokens that one pass through the model holds.
+inline int pass_rows(const vadusa_config* c) { return c->prefill_rows > c->max_batch ? c->prefill_rows : c->max_batch; }
 inline int vpad(const vadusa_config* c) { return (int)align_up(c->vocab, 128); }
 
 struct TensorDesc {
@@ -95,7 +99,7 @@ struct WorkspaceLayout {
   int64_t scalars;                       // uint32 err, int32 done_count, padding
   int64_t ctx_len, nvalid, gen_count, commit_base, commit_len, best, root, saved_nvalid;   // int32 [B]
   int64_t commit_path;                   // int32 [B][16]
-  int64_t seq_order;                     // int32 [B]: sequences by descending context length
+  int64_t seq_order;                     // int32 [R]: rows by descending context length
   int64_t tree_parent, tree_depth, tree_rank, tree_anc;       // [B*64] (anc: uint64)
   int64_t chain_parent, chain_depth, chain_rank, chain_anc;   // [64]
   int64_t tokens, stage_tokens;          // int32 [M]
@@ -111,13 +115,16 @@ struct WorkspaceLayout {
   int64_t gemm_part;                     // fp32 split-K exchange of the tensor-core products (kGemmPartBytes)
   int64_t ln_stats;                      // per-group LayerNorm statistics for the fused products (kLnStatsBytes)
   int64_t gen_out, gen_len;              // int32 [B][kGenHostCap], int32 [B] (vadusa_generate_host staging)
+  // prefill: one row per prefix chunk of a pass (R = pass_rows)
+  int64_t pf_ctx_len, pf_nvalid, pf_seq, pf_last;   // int32 [R]: tokens before the chunk, its length, its sequence, sequence if last chunk else -1
+  int64_t pf_block_table;                // int32 [R][max_blocks_per_seq]: the block-table row of the chunk's sequence
   int64_t total;
 };
 
 inline WorkspaceLayout workspace_layout(const vadusa_config* c) {
   WorkspaceLayout w;
   int64_t off = 0;
-  const int64_t B = c->max_batch, N = c->max_tree_nodes, M = B * N, d = c->d_model, f = c->d_ffn;
+  const int64_t B = c->max_batch, R = pass_rows(c), N = c->max_tree_nodes, M = R * N, d = c->d_model, f = c->d_ffn;
   const int64_t es = esize(c), vp = vpad(c), hd = c->n_draft_heads;
   auto take = [&](int64_t bytes) { int64_t o = off; off = align_up(off + bytes, 256); return o; };
   w.scalars = take(256);
@@ -125,7 +132,7 @@ inline WorkspaceLayout workspace_layout(const vadusa_config* c) {
   w.commit_base = take(B * 4); w.commit_len = take(B * 4); w.best = take(B * 4); w.root = take(B * 4);
   w.saved_nvalid = take(B * 4);
   w.commit_path = take(B * 16 * 4);
-  w.seq_order = take(B * 4);
+  w.seq_order = take(R * 4);
   w.tree_parent = take(B * 64 * 4); w.tree_depth = take(B * 64 * 4); w.tree_rank = take(B * 64 * 4);
   w.tree_anc = take(B * 64 * 8);
   w.chain_parent = take(64 * 4); w.chain_depth = take(64 * 4); w.chain_rank = take(64 * 4);
@@ -143,6 +150,8 @@ inline WorkspaceLayout workspace_layout(const vadusa_config* c) {
   w.gemm_part = take(kGemmPartBytes);
   w.ln_stats = take(kLnStatsBytes);
   w.gen_out = take(B * kGenHostCap * 4); w.gen_len = take(B * 4);
+  w.pf_ctx_len = take(R * 4); w.pf_nvalid = take(R * 4); w.pf_seq = take(R * 4); w.pf_last = take(R * 4);
+  w.pf_block_table = take(R * (int64_t)c->max_blocks_per_seq * 4);
   w.total = off;
   return w;
 }

@@ -73,6 +73,45 @@ def test_toy_lockstep_prefill_and_kv(dtype):
     g.check()
 
 
+@pytest.mark.parametrize("dtype,rows", [("fp32", 0), ("bf16", 5), ("bf16", 64)])
+def test_prefill_in_passes_of_many_chunks_and_behind_existing_context(dtype, rows):
+    """The prefix goes in as two calls (the second one behind what the first left in the cache), with
+    0 (= one chunk per sequence and pass), 5 and 64 chunks per pass: the K/V rows, lengths and the carried
+    state (through the next iteration's root and logits) equal the oracle's."""
+    import paper_2410_21951_b200 as P
+    wl = W.toy_workload(dtype=dtype, d_model=128, n_heads=2, d_ffn=256, vocab=203, tree_nodes=16, tree_caps=(6, 3, 2),
+                        tau=3, temperature=1.0, batch=3, phoneme_len=(20, 70), prompt_len=90, index=15)
+    w = W.make_weights(wl.shape, wl.seed())
+    model = O.Model.from_shape(wl.shape, w)
+    tpl = W.static_template(wl.tree_nodes, wl.tree_caps)
+    prefixes = [W.prefix_for(wl, b) for b in range(wl.batch)]
+    toks = [tokens_with_phonemes(wl.shape, ph, pr) for ph, pr in prefixes]
+    need = [len(t) + 3 * (tpl.max_depth + 1) + wl.tree_nodes for t in toks]
+    table, total = W.shuffled_block_table(need, 64, 21, spare_pages=3)
+    g = P.Vadusa(wl.shape, w, max_batch=wl.batch, max_tree_nodes=wl.tree_nodes, max_blocks_per_seq=table.shape[1],
+                 kv_num_blocks=total, prefill_rows=rows)
+    g.set_tree(tpl.parent, tpl.rank)
+    g.begin(table)
+    cut = [len(t) // 3 + b for b, t in enumerate(toks)]
+    for part in (0, 1):
+        seg = [t[:c] if part == 0 else t[c:] for t, c in zip(toks, cut)]
+        mat = np.zeros((wl.batch, max(len(x) for x in seg)), dtype=np.int32)
+        for b, x in enumerate(seg):
+            mat[b, :len(x)] = x
+        g.prefill(mat, [len(x) for x in seg])
+        want = cut if part == 0 else [len(t) for t in toks]
+        assert list(g.lengths()) == want
+    states = {b: O.prefill_blocked(model, prefixes[b][0], prefixes[b][1], seq=b, chunk=41) for b in range(wl.batch)}
+    for b, st in states.items():
+        K, V = read_kv(g, table, b, st.S)
+        assert np.abs(K - st.kv.K[:, :st.S]).max() <= TOL[dtype]
+        assert np.abs(V - st.kv.V[:, :st.S]).max() <= TOL[dtype]
+    so, sg = _sampling(wl)
+    rep = lockstep(g, table, model, states, tpl, so, sg, 3, dtype, oracle_mode="memo")
+    assert rep.iterations == 3
+    g.check()
+
+
 @pytest.mark.parametrize("nodes", [10, 24, 48])
 def test_bf16_small_token_counts_take_the_layernorm_fused_products(nodes):
     """d_model 256 (two groups of 128 features), one sequence: the token count selects the 16-, 32- and
