@@ -126,7 +126,10 @@ typedef struct {
   int32_t tau;           /* tolerance, >= 1 */
   float temperature;     /* 0 = greedy */
   float top_p;
-  int32_t eos_masked;    /* 1: the EOS logit counts as -inf everywhere (base and draft heads) */
+  int32_t eos_masked;    /* 1: the EOS logit counts as -inf everywhere (base and draft heads); generation ends by
+                            length.  0: EOS can be drawn and drafted; a sequence ends (becomes inactive) in the
+                            iteration that commits EOS, and the tokens behind EOS on the accepted path are
+                            dropped (tolerance 1 then stops exactly where plain decoding stops, Sec. II-A) */
   int32_t accept_rule;   /* 0: Algorithm 1 as above; 1: membership in the plain top-tau of the
                             unperturbed logits (the root is still sampled with noise) */
   uint64_t seed;

@@ -7,6 +7,12 @@ top-k tokens, every root-to-leaf branch is scored by its own sequential causal
 pass and checked with Algorithm 1, the longest (then leftmost) accepted branch
 is kept, and decoding continues from the base head's distribution at the last
 accepted token.
+
+End of sequence (the paper does not treat it; its tolerance-1 decoding is lossless,
+Sec. II-A, so nothing may follow a token at which plain decoding would have stopped):
+with `eos_masked` the EOS id can never be drawn or drafted and generation ends by
+length; without it, a sequence is finished as soon as EOS is committed, and the
+tokens behind EOS on the accepted path are dropped.
 """
 from __future__ import annotations
 
@@ -38,6 +44,7 @@ class State:
     h_star: np.ndarray            # final hidden state at the last committed token
     logits_star: np.ndarray       # base-head logits there (they predict position kv.n)
     seq: int = 0                  # sequence id, enters the noise only
+    finished: bool = False        # EOS has been committed (only when EOS is not masked)
 
     @property
     def S(self) -> int:
@@ -95,8 +102,12 @@ def ar_decode(model: Model, st: State, sp: Sampling, n_tokens: int) -> List[int]
     """Plain AR decoding from state `st` (which is advanced)."""
     out = []
     for _ in range(n_tokens):
+        if st.finished:
+            break
         pos = st.S
         tok = sample_next(model, st.logits_star, sp, st.seq, pos)
+        if not sp.eos_masked and tok == model.eos_id:
+            st.finished = True
         r = forward_token(model, st.kv, AUDIO, tok, pos)
         st.h_star, st.logits_star = r.h, r.logits
         st.tokens.append(tok); out.append(tok)
@@ -140,6 +151,7 @@ class IterationTrace:
     attn: Optional[List[np.ndarray]] = None     # per layer [N, d] (tree mode only)
     K: Optional[np.ndarray] = None              # [L, N, H, dh] rows of every node (tree/memo mode)
     V: Optional[np.ndarray] = None
+    finished: bool = False                      # EOS was committed in this iteration
 
 
 def _gap_top2(keys, nuc) -> float:
@@ -263,6 +275,12 @@ def vadusa_iteration(model: Model, st: State, template, sp: Sampling, mode: str 
     if forced_best is not None:
         path = template.node_path(int(forced_best))
         k_star = len(path) - 1
+    finished = False
+    if not sp.eos_masked:
+        for j, n in enumerate(path):
+            if int(toks[n]) == model.eos_id:          # the sequence ends here: drop what follows EOS
+                path, k_star, finished = path[: j + 1], j, True
+                break
     best = path[-1]
 
     edge_ok = np.zeros(N, dtype=bool); edge_ok[0] = True
@@ -280,18 +298,20 @@ def vadusa_iteration(model: Model, st: State, template, sp: Sampling, mode: str 
     st.kv.extend(node_K[:, path], node_V[:, path])
     st.tokens.extend(int(toks[n]) for n in path)
     st.h_star, st.logits_star = node_h[best].copy(), node_logits[best].copy()
+    st.finished = st.finished or finished
     return IterationTrace(S=S, root=root, topk=topk, tree_tokens=toks, node_logits=node_logits,
                           node_h=node_h, edge_ok=edge_ok, accept_len=k_star + 1, best_node=best,
                           path_nodes=list(path), path_tokens=[int(toks[n]) for n in path],
                           margin_root=_gap_top2(keys_s, nuc_s), margin_draft=margin_draft, draft_gaps=draft_gaps,
-                          margin_accept=margin_accept, attn=attn, K=node_K, V=node_V)
+                          margin_accept=margin_accept, attn=attn, K=node_K, V=node_V, finished=finished)
 
 
 def vadusa_generate(model: Model, st: State, template, sp: Sampling, n_tokens: int,
                     mode: str = "branch", max_iters: Optional[int] = None) -> List[IterationTrace]:
-    """Iterate until at least n_tokens have been generated (or max_iters)."""
+    """Iterate until at least n_tokens have been generated (or max_iters, or EOS committed)."""
     traces = []
     start = len(st.tokens)
-    while len(st.tokens) - start < n_tokens and (max_iters is None or len(traces) < max_iters):
+    while (len(st.tokens) - start < n_tokens and (max_iters is None or len(traces) < max_iters)
+           and not st.finished):
         traces.append(vadusa_iteration(model, st, template, sp, mode=mode))
     return traces

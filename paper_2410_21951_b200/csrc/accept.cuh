@@ -28,7 +28,8 @@ struct SeqState {             // device state of the batch (all [batch] unless n
   int target;                 // stop a sequence after this many tokens (0: never)
 };
 
-// One block per sequence.  Edges are tested depth by depth, only below accepted nodes:
+// One block per sequence.  A sequence whose path commits EOS (when EOS is not masked) or reaches the token
+// target becomes inactive (nvalid = 0).  Edges are tested depth by depth, only below accepted nodes:
 // for an accepted parent p the keys of its logits row are formed once in shared memory
 // (they predict absolute position ctx_len + depth(p) + 1), then each child token c is
 // accepted iff fewer than tau tokens precede it in key order (and it lies in the nucleus).
@@ -42,7 +43,7 @@ __global__ void __launch_bounds__(256) accept_kernel(
   __shared__ int s_parent[kMaxNodes], s_depth[kMaxNodes], s_tok[kMaxNodes];
   __shared__ int s_child[kMaxNodes], s_ok[kMaxNodes], s_nchild;
   __shared__ unsigned long long s_edges, s_acc;
-  __shared__ int s_path[kMaxPath], s_best, s_len;
+  __shared__ int s_path[kMaxPath], s_best, s_len, s_eos;
   __shared__ Best bscratch[32];
   __shared__ float fscratch[32];
 
@@ -140,6 +141,11 @@ __global__ void __launch_bounds__(256) accept_kernel(
     int len = min(s_depth[best] + 1, kMaxPath);
     int n = best;
     for (int j = len - 1; j >= 0; --j) { s_path[j] = n; n = s_parent[n]; }
+    // EOS not masked: the sequence ends with the first EOS on the path; what follows it is dropped
+    s_eos = 0;
+    if (!sp.eos_masked)
+      for (int j = 0; j < len; ++j)
+        if (s_tok[s_path[j]] == sp.eos_id) { len = j + 1; best = s_path[j]; s_eos = 1; break; }
     s_best = best; s_len = len;
   }
   __syncthreads();
@@ -171,7 +177,7 @@ __global__ void __launch_bounds__(256) accept_kernel(
     st.ctx_len[b] = S + len;
     const int g = st.gen_count[b] + len;
     st.gen_count[b] = g;
-    if (st.target > 0 && g >= st.target) { st.nvalid[b] = 0; atomicAdd(st.done_count, 1); }
+    if (s_eos || (st.target > 0 && g >= st.target)) { st.nvalid[b] = 0; atomicAdd(st.done_count, 1); }
     if (out.accept_len) out.accept_len[b] = len;
     if (out.edge_bits) out.edge_bits[b] = s_edges;
     if (out.next_root) out.next_root[b] = nroot;

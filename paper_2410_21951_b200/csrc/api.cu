@@ -425,8 +425,10 @@ vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeVi
 
 template <typename T>
 vadusa_status layernorm(vadusa_ctx* ctx, const float* x, const float* g, const float* b, T* y, int rows) {
+  const int d = ctx->cfg.d_model;
+  const bool by_warp = rows >= 64 && d % 128 == 0 && d <= 2048;   // many rows: one warp per row
   cudaLaunchConfig_t lc = {};
-  lc.gridDim = dim3(rows);
+  lc.gridDim = dim3(by_warp ? (rows + 7) / 8 : rows);
   lc.blockDim = dim3(256);
   lc.stream = ctx->stream;
   cudaLaunchAttribute at[1];
@@ -434,7 +436,8 @@ vadusa_status layernorm(vadusa_ctx* ctx, const float* x, const float* g, const f
   at[0].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = at; lc.numAttrs = 1;
   PROF(ctx, K_LAYERNORM);
-  CU(cudaLaunchKernelEx(&lc, layernorm_kernel<T>, x, g, b, y, rows, ctx->cfg.d_model, ctx->cfg.ln_eps));
+  if (by_warp) CU(cudaLaunchKernelEx(&lc, layernorm_rows_kernel<T>, x, g, b, y, rows, d, ctx->cfg.ln_eps));
+  else CU(cudaLaunchKernelEx(&lc, layernorm_kernel<T>, x, g, b, y, rows, d, ctx->cfg.ln_eps));
   LAUNCH_CHECK();
   return VADUSA_OK;
 }

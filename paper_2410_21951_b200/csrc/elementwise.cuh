@@ -103,4 +103,49 @@ __global__ void __launch_bounds__(256) layernorm_kernel(const float* __restrict_
   for (int i = threadIdx.x; i < d; i += blockDim.x) { yr[i] = from_f<T>((v[cnt] - mean) * rstd * g[i] + bta[i]); ++cnt; }
 }
 
+// The same LayerNorm with one warp per row, for rows whose length is a multiple of 128 (up to 2048): lane l
+// holds columns 128 j + 4 l .. + 3 of the row in registers (all loads issued at once), the two sums go through
+// warp shuffles, and the result is written four values at a time.  8 rows per block of 256 threads.
+template <typename T>
+__global__ void __launch_bounds__(256) layernorm_rows_kernel(const float* __restrict__ x, const float* __restrict__ g,
+                                                             const float* __restrict__ bta, T* __restrict__ y, int rows,
+                                                             int d, float eps) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  const int nj = d >> 7;
+  const float4* xr = reinterpret_cast<const float4*>(x + (long long)row * d);
+  float4 v[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j)
+    if (j < nj) v[j] = xr[32 * j + lane];
+  float s = 0.f;
+#pragma unroll
+  for (int j = 0; j < 16; ++j)
+    if (j < nj) s += (v[j].x + v[j].y) + (v[j].z + v[j].w);
+  s = warp_sum(s);
+  // the rows are in registers: the next kernel may start (all blocks of this grid fit on the GPU at once, so
+  // an earlier signal would let it take the SMs while the kernel before this one is still running)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const float mean = s / (float)d;
+  float q = 0.f;
+#pragma unroll
+  for (int j = 0; j < 16; ++j)
+    if (j < nj) {
+      const float a = v[j].x - mean, b = v[j].y - mean, c = v[j].z - mean, e = v[j].w - mean;
+      q += (a * a + b * b) + (c * c + e * e);
+    }
+  q = warp_sum(q);
+  const float rstd = 1.0f / sqrtf(q / (float)d + eps);
+  T* yr = y + (long long)row * d;
+#pragma unroll
+  for (int j = 0; j < 16; ++j)
+    if (j < nj) {
+      const int c0 = 128 * j + 4 * lane;
+      const float4 gg = *reinterpret_cast<const float4*>(g + c0), bb = *reinterpret_cast<const float4*>(bta + c0);
+      store4<T>(yr + c0, (v[j].x - mean) * rstd * gg.x + bb.x, (v[j].y - mean) * rstd * gg.y + bb.y,
+                (v[j].z - mean) * rstd * gg.z + bb.z, (v[j].w - mean) * rstd * gg.w + bb.w);
+    }
+}
+
 }  // namespace vadusa

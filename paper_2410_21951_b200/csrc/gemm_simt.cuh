@@ -10,18 +10,6 @@ namespace vadusa {
 // ---- epilogues: called with the fp32 accumulator, one element at a time (operator()) or
 // four consecutive features of one token at a time (vec4; n is a multiple of 4) ----------
 
-template <typename T> __device__ __forceinline__ void store4(T* p, float a, float b, float c, float d);
-template <> __device__ __forceinline__ void store4<float>(float* p, float a, float b, float c, float d) {
-  *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
-}
-template <> __device__ __forceinline__ void store4<bf16>(bf16* p, float a, float b, float c, float d) {
-  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
-  uint2 v;
-  v.x = *reinterpret_cast<uint32_t*>(&lo);
-  v.y = *reinterpret_cast<uint32_t*>(&hi);
-  *reinterpret_cast<uint2*>(p) = v;
-}
-
 // q/k/v projection (verify step, per layer): + bias, round to T; q goes to a dense buffer,
 // k and v go straight to the paged cache at the node's slot (kv_row[m], written by the
 // embedding kernel of the same pass; -1: the row is not scored).

@@ -153,6 +153,89 @@ def test_toy_planted_paths_are_accepted(dtype, tau, temperature, top_p, rule):
     g.check()
 
 
+def test_unmasked_eos_ends_a_sequence_and_drops_what_follows_it():
+    """EOS not masked: (1) EOS planted in the middle of a forced path: the path is cut behind it, the
+    sequence becomes inactive and later iterations leave it alone; (2) free-running generation of a
+    9-token vocabulary stops where the oracle's does, on seeds whose decisions are all decidable."""
+    import torch
+    import paper_2410_21951_b200 as P
+    wl = W.toy_workload(dtype="fp32", d_model=64, n_heads=2, d_ffn=128, vocab=9, tree_nodes=14, tree_caps=(3, 2, 2),
+                        batch=2, phoneme_len=(9, 9), prompt_len=40, index=17, gen_tokens=40)
+    w, model, tpl, g, table = _setup(wl, 45, range(2))
+    eos = wl.shape.vocab - 1
+    dev = g.dev
+    # (1) planted
+    states, _ = _prefill_both(wl, g, table, model, range(2))
+    so = O.Sampling(tau=1, temperature=0.0, eos_masked=False)
+    sg = P.Sampling.make(tau=1, temperature=0.0, eos_masked=0)
+    rank0 = [n for n in range(tpl.n_nodes) if all(r == 0 for r in tpl.rank_path(n))]
+    assert len(rank0) == 4
+    g.draft(sg)
+    ov = np.tile(np.arange(tpl.n_nodes, dtype=np.int32) % 7, (2, 1))
+    ov[0, rank0[1]] = eos                                   # sequence 0: EOS at depth 1 of the forced path
+    forced = np.array([rank0[3], rank0[2]], dtype=np.int32)
+    acc = torch.zeros(2, dtype=torch.int32, device=dev)
+    ptoks = torch.zeros(2, 16, dtype=torch.int32, device=dev)
+    g.verify_step(override=torch.from_numpy(ov).to(dev))
+    g.accept_and_commit(sg, forced_best=torch.from_numpy(forced).to(dev), accept_len=acc, path_tokens=ptoks)
+    for b in range(2):
+        tr = O.vadusa_iteration(model, states[b], tpl, so, mode="memo", tokens_override=ov[b], forced_best=int(forced[b]))
+        assert int(acc[b]) == tr.accept_len and list(ptoks[b, :tr.accept_len].cpu().numpy()) == tr.path_tokens
+    assert int(acc[0]) == 2 and int(acc[1]) == 3 and states[0].finished and not states[1].finished
+    lens = g.lengths().copy()
+    g.draft(sg); g.verify_step(); g.accept_and_commit(sg, accept_len=acc)
+    assert int(acc[0]) == 0 and g.lengths()[0] == lens[0] and g.lengths()[1] > lens[1]
+    # (2) free-running
+    checked = 0
+    for seed in range(8):
+        so = O.Sampling(tau=2, temperature=1.0, eos_masked=False, seed=seed)
+        sg = P.Sampling.make(tau=2, temperature=1.0, eos_masked=0, seed=seed)
+        states, _ = _prefill_both(wl, g, table, model, range(2))
+        traces = {b: O.vadusa_generate(model, states[b], tpl, so, 40, mode="memo") for b in range(2)}
+        margin = min(min(t.margin_root, t.margin_accept, float(t.margin_draft.min())) for ts in traces.values() for t in ts)
+        if margin <= MARGIN:
+            continue
+        out = torch.full((2, 40), -1, dtype=torch.int32, device=dev)
+        out_len = torch.zeros(2, dtype=torch.int32, device=dev)
+        g.generate(sg, 40, out, out_len)
+        for b in range(2):
+            want = states[b].tokens[:40]
+            n = int(out_len[b])
+            assert n == len(want) and list(out[b, :n].cpu().numpy()) == want
+            assert states[b].finished == (eos in want)
+        checked += 1
+    assert checked >= 2
+    g.check()
+
+
+def test_six_draft_heads_accept_up_to_seven_tokens():
+    """The paper's six-head ablation (Sec. III-A.3): depth-6 tree, planted continuation, paths of 7 tokens."""
+    from workloads.trees import _from_rank_paths
+    wl = W.toy_workload(dtype="fp32", d_model=64, n_heads=2, d_ffn=128, vocab=61, n_draft_heads=6, tree_nodes=20,
+                        tree_caps=(4, 3, 2, 2, 2, 2), batch=2, phoneme_len=(9, 9), prompt_len=60, index=16)
+    zero = tuple([0] * 6)
+    paths = [zero[:k] for k in range(7)] + [(1,), (2,), (3,), (0, 1), (0, 2), (1, 0), (0, 0, 1), (1, 0, 0), (0, 0, 0, 1),
+                                            (0, 0, 0, 0, 1), (0, 0, 0, 0, 0, 1), (0, 1, 0), (0, 1, 0, 0)]
+    tpl = _from_rank_paths(paths)
+    W.validate_template(tpl, wl.tree_caps)
+    assert tpl.n_nodes == 20 and tpl.max_depth == 6
+    w = W.make_weights(wl.shape, wl.seed())
+    model = O.Model.from_shape(wl.shape, w)
+    need = [sum(len(x) for x in W.prefix_for(wl, b)) + 6 * 7 + wl.tree_nodes for b in range(2)]
+    g, table = make_gpu(wl.shape, w, wl.batch, wl.tree_nodes, need, 11)
+    g.set_tree(tpl.parent, tpl.rank)
+    states, _ = _prefill_both(wl, g, table, model, range(2))
+    so, sg = _sampling(wl, seed=5, tau=2, temperature=0.9)
+    so1 = O.Sampling(tau=1, temperature=0.9, top_p=1.0, seed=5, accept_rule=0)
+    planted = {}
+    for b in range(2):
+        ph, pr = W.prefix_for(wl, b)
+        planted[b] = O.ar_decode(model, O.prefill(model, ph, pr, seq=b), so1, 50)
+    rep = lockstep(g, table, model, states, tpl, so, sg, 6, "fp32", oracle_mode="memo", planted=planted)
+    assert max(rep.accept_lens) == 7
+    g.check()
+
+
 def test_c1_generate_matches_oracle_and_plain_ar():
     """BASELINE config 1 end to end: free-running vadusa_generate (greedy, tolerance 1, 100
     tokens) equals the oracle's speculative decoding and plain AR decoding token for token

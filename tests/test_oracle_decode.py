@@ -56,6 +56,34 @@ def test_tolerance_one_equals_plain_ar(temperature, top_p, shape):
     assert all(1 <= t.accept_len <= tpl.max_depth + 1 for t in traces)
 
 
+def test_unmasked_eos_ends_the_sequence_exactly_where_plain_ar_ends_it():
+    """With EOS unmasked and tolerance 1 the speculative loop still equals plain decoding (Sec. II-A),
+    including where it stops; tokens that follow EOS on an accepted path are not committed."""
+    wl, m, ph, pr = _setup(vocab=9)                 # 8 speech ids + EOS: EOS turns up within a few tokens
+    tpl = W.static_template(10, (4, 3, 2))
+    stopped = 0
+    for seed in range(6):
+        sp = O.Sampling(tau=1, temperature=1.0, eos_masked=False, seed=seed)
+        st_ar = O.prefill(m, ph, pr)
+        want = O.ar_decode(m, st_ar, sp, 40)
+        st = O.prefill(m, ph, pr)
+        traces = O.vadusa_generate(m, st, tpl, sp, 40)
+        assert st.tokens[:len(want)] == want and st.finished == st_ar.finished
+        if st_ar.finished:
+            stopped += 1
+            assert want[-1] == m.eos_id and m.eos_id not in want[:-1]
+            assert st.tokens == want and traces[-1].finished and traces[-1].path_tokens[-1] == m.eos_id
+    assert stopped >= 3
+    # EOS planted in the middle of a fully accepted path: the rest of the path is dropped
+    sp = O.Sampling(tau=1, temperature=0.0, eos_masked=False)
+    st = O.prefill(m, ph, pr)
+    chain = W.chain_template(4)
+    toks = np.array([3, m.eos_id, 5, 6])
+    tr = O.vadusa_iteration(m, st, chain, sp, tokens_override=toks, forced_best=3)
+    assert tr.finished and tr.accept_len == 2 and tr.path_tokens == [3, m.eos_id] and tr.best_node == 1
+    assert st.finished and st.tokens[-2:] == [3, m.eos_id]
+
+
 def test_planted_continuation_is_fully_accepted_and_cache_equals_ar_cache():
     """If the tree holds the true continuation, all of it is accepted (tau = 1),
     and afterwards the cache holds exactly what plain AR decoding stores."""
