@@ -31,6 +31,22 @@ sys.path.insert(0, ROOT)
 WORKLOAD = "C2"
 
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the 49 projection launches of one C2 step, from the
+# ncu capture summarised in profiles/gemm_tc_kernel_c2.md; valid for the kernel sources with this hash only.
+_NCU_TRAFFIC = {"src_sha256_16": "794ea809c19e1067", "bytes_per_step": 327.74e6, "launches": 49}
+
+
+def _gemm_traffic():
+    import hashlib
+    h = hashlib.sha256()
+    try:
+        for f in ("gemm_tc.cuh", "tc.cuh"):
+            h.update(open(os.path.join(ROOT, "paper_2410_21951_b200", "csrc", f), "rb").read())
+    except OSError:
+        return None
+    return _NCU_TRAFFIC["bytes_per_step"] if h.hexdigest()[:16] == _NCU_TRAFFIC["src_sha256_16"] else None
+
+
 def _peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -318,7 +334,8 @@ def run_ours(args):
                                            "ms_per_step": pl_ms / n_pl, "steps": n_pl}}),
             "roofline": {"bound": "hbm", "kernel": "projection GEMMs (qkv, out, ffn1, ffn2, lm head)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_source": f"{peak_kind} copy bandwidth", "traffic": None,
+                         "peak_source": f"{peak_kind} copy bandwidth", "traffic": _gemm_traffic(),
+                         "traffic_unit": "DRAM bytes per step over the same launches (ncu; null if the kernel changed since)",
                          "method": "algorithmic weight bytes per step / (CUDA-event step time x projections' share of kernel time)",
                          "algorithmic_bytes_per_step": gemm_alg_per_step, "launches_per_step": sum(prof[k][0] for k in gemm_bytes if k in prof) // n_prof,
                          "kernel_time_shares": shares, "profiled_steps": n_prof,
