@@ -246,6 +246,28 @@ vadusa_status vadusa_get_lengths(vadusa_ctx *ctx, int32_t *h_ctx_len);  /* synch
 vadusa_status vadusa_check(vadusa_ctx *ctx);                            /* synchronises; device error word */
 int64_t vadusa_kernel_launches(const vadusa_ctx *ctx);                  /* total kernels enqueued so far */
 
+/* ---- sparse-tree construction (paper Sec. II-D) --------------------------------------
+ * The paper grows its sparse candidate tree greedily so as to maximise the expected accepted
+ * length within a fixed number of nodes, from acceptance probabilities measured with the
+ * full tree.
+ *
+ * vadusa_accept_stats: since the last reset, how often the acceptance test (Algorithm 1) was
+ * applied to a candidate of draft head j+1 with top-k rank r below an accepted parent
+ * (h_tested[j * VADUSA_MAX_DRAFT_TOPK + r]) and how often it passed (h_accepted[...]); host
+ * int64 arrays of VADUSA_MAX_DEPTH * VADUSA_MAX_DRAFT_TOPK entries.  Iterations with a forced
+ * winner are not counted.  Synchronises; reset != 0 clears the counters afterwards.
+ *
+ * vadusa_build_sparse_tree (host only, no GPU): h_prob[j * topk + r] = probability that the
+ * rank-r candidate of head j+1 is accepted given that its parent is (j < depth, r < topk).  A
+ * node's probability is the product along its root path; starting from the root, the candidate
+ * child with the highest probability is added n_nodes - 1 times (ties: shallower, then
+ * lexicographically smaller rank path).  Writes parent[] and rank[] in (depth, rank path)
+ * order, ready for vadusa_set_tree, and the expected accepted length 1 + sum of the node
+ * probabilities.  VADUSA_EINVAL if the capped tree has fewer than n_nodes nodes. */
+vadusa_status vadusa_accept_stats(vadusa_ctx *ctx, int64_t *h_tested, int64_t *h_accepted, int32_t reset);
+vadusa_status vadusa_build_sparse_tree(const double *h_prob, int32_t depth, int32_t topk, int32_t n_nodes,
+                                       int32_t *h_parent, int32_t *h_rank, double *h_expected_len);
+
 /* ---- measurement ------------------------------------------------------------------ */
 /* Between vadusa_profile_begin and vadusa_profile_end every kernel launch of the library
  * is bracketed by a pair of CUDA events on the context's stream.  vadusa_profile_end

@@ -3,8 +3,8 @@
 A plain, slow, obviously-correct restatement of what the paper's decoding
 procedure computes (Sec. II-A: draft heads and candidate tree; Sec. II-C and
 Algorithm 1: verification with the tolerance mechanism and the choice of the
-longest, then leftmost, accepted branch), on a plain pre-LN decoder-only
-transformer.  Floating point is float64 throughout; in "bf16" models the values
+longest, then leftmost, accepted branch; Sec. II-D: greedy sparse-tree
+construction), on a plain pre-LN decoder-only transformer.  Floating point is float64 throughout; in "bf16" models the values
 the model *stores* in bf16 are rounded at the stated points; the keys that
 decide integers are formed in float32.
 
@@ -24,5 +24,7 @@ from .verify import verify_branch, select_best, accept_from_edges, tree_edge_acc
 from .decode import (Sampling, ar_decode, prefill, prefill_blocked, State, vadusa_iteration,
                      vadusa_generate, build_tree_tokens, IterationTrace, sample_next, draws_at,
                      draft_topk)
+from .tree_build import (greedy_tree, best_tree_brute_force, expected_length, path_probability)
+from . import tree_build
 
 __all__ = [n for n in dir() if not n.startswith("_")]

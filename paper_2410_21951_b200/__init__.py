@@ -6,7 +6,7 @@ ABI, see include/vadusa.h); this package only marshals arguments.  There is no
 CPU path: without the compiled library, or without a B200, calls fail.
 """
 from .binding import (Config, Sampling, Stats, Vadusa, VadusaError, lib, load_library, pack_weights,
-                      tensor_infos, MAX_PATH, draft_topk_static)
+                      tensor_infos, MAX_PATH, draft_topk_static, build_sparse_tree)
 
 __all__ = ["Config", "Sampling", "Stats", "Vadusa", "VadusaError", "lib", "load_library", "pack_weights",
-           "tensor_infos", "MAX_PATH", "draft_topk_static"]
+           "tensor_infos", "MAX_PATH", "draft_topk_static", "build_sparse_tree"]

@@ -69,6 +69,7 @@ EXPORTS = ["vadusa_workspace_bytes", "vadusa_weights_bytes", "vadusa_kv_pool_byt
            "vadusa_begin", "vadusa_prefill", "vadusa_load_state", "vadusa_draft", "vadusa_verify_step",
            "vadusa_accept_and_commit", "vadusa_generate", "vadusa_generate_host", "vadusa_get_lengths",
            "vadusa_check", "vadusa_kernel_launches", "vadusa_profile_begin", "vadusa_profile_end",
+           "vadusa_accept_stats", "vadusa_build_sparse_tree",
            "vadusa_draft_topk_static", "vadusa_static_scratch_bytes", "vadusa_static_last_error"]
 
 _lib = None
@@ -103,6 +104,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "vadusa_draft_topk_static": (I32, [P, P, P, P, I32, I32, I32, I32, I32, I32, I32, P, P]),
         "vadusa_static_scratch_bytes": (I64, []),
         "vadusa_static_last_error": (C.c_char_p, []),
+        "vadusa_accept_stats": (I32, [P, P, P, I32]),
+        "vadusa_build_sparse_tree": (I32, [P, I32, I32, I32, P, P, P]),
         "vadusa_profile_begin": (I32, [P]),
         "vadusa_profile_end": (I32, [P, C.POINTER(KernelTime), I32, C.POINTER(I32)]),
     }
@@ -188,6 +191,22 @@ def draft_topk_static(draft_w, draft_b, draft_u, hstar, dtype: int, batch: int, 
                                     C.c_void_p(stream.cuda_stream) if stream is not None else None)
     if st:
         raise VadusaError(st, L.vadusa_static_last_error().decode())
+
+
+MAX_DEPTH, MAX_DRAFT_TOPK = 15, 16
+
+
+def build_sparse_tree(prob: np.ndarray, n_nodes: int):
+    """(parent, rank, expected accepted length) of the greedily grown tree; prob is [depth][topk].  Host only."""
+    prob = np.ascontiguousarray(prob, dtype=np.float64)
+    parent = np.zeros(n_nodes, dtype=np.int32)
+    rank = np.zeros(n_nodes, dtype=np.int32)
+    exp = C.c_double(0.0)
+    st = lib().vadusa_build_sparse_tree(prob.ctypes.data, prob.shape[0], prob.shape[1], n_nodes, parent.ctypes.data,
+                                        rank.ctypes.data, C.addressof(exp))
+    if st:
+        raise VadusaError(st, "vadusa_build_sparse_tree: bad arguments or fewer candidate nodes than asked for")
+    return parent, rank, exp.value
 
 
 class Vadusa:
@@ -350,6 +369,13 @@ class Vadusa:
 
     def check(self):
         self._ck(self.L.vadusa_check(self.ctx))
+
+    def accept_stats(self, reset: bool = False):
+        """(tested, accepted) int64 [MAX_DEPTH][MAX_DRAFT_TOPK]: acceptance tests by (draft head, rank)."""
+        t = np.zeros((MAX_DEPTH, MAX_DRAFT_TOPK), dtype=np.int64)
+        a = np.zeros((MAX_DEPTH, MAX_DRAFT_TOPK), dtype=np.int64)
+        self._ck(self.L.vadusa_accept_stats(self.ctx, self._h(t), self._h(a), int(reset)))
+        return t, a
 
     def kernel_launches(self) -> int:
         return int(self.L.vadusa_kernel_launches(self.ctx))

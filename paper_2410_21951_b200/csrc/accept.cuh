@@ -26,7 +26,9 @@ struct SeqState {             // device state of the batch (all [batch] unless n
   int32_t* done_count;        // scalar: sequences that reached the target
   int out_cap;
   int target;                 // stop a sequence after this many tokens (0: never)
+  unsigned long long* stats;  // [2][kStatDepth][kStatTopk]: acceptance tests applied / passed, by (draft head, rank)
 };
+
 
 // One block per sequence.  A sequence whose path commits EOS (when EOS is not masked) or reaches the token
 // target becomes inactive (nvalid = 0).  Edges are tested depth by depth, only below accepted nodes:
@@ -127,6 +129,13 @@ __global__ void __launch_bounds__(256) accept_kernel(
       if (tid == 0) {
         for (int i = 0; i < nchild; ++i)
           if (s_ok[i]) { s_edges |= 1ull << s_child[i]; s_acc |= 1ull << s_child[i]; }
+      }
+      if (tid < nchild && st.stats && d < kStatDepth) {
+        const int r = tree.rank[to + s_child[tid]];
+        if (r >= 0 && r < kStatTopk) {
+          atomicAdd(st.stats + d * kStatTopk + r, 1ull);
+          if (s_ok[tid]) atomicAdd(st.stats + (kStatDepth + d) * kStatTopk + r, 1ull);
+        }
       }
       __syncthreads();
     }

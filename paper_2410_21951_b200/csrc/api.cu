@@ -5,6 +5,7 @@
 
 #include <type_traits>
 
+#include <algorithm>
 #include <map>
 #include <new>
 #include <string>
@@ -183,8 +184,10 @@ SeqState state_of(vadusa_ctx* c, int32_t* out_tokens, int out_cap, int target) {
   s.done_count = done_word(c);
   s.out_cap = out_cap;
   s.target = target;
+  s.stats = wsptr<unsigned long long>(c, c->ws.acc_stats);
   return s;
 }
+static_assert(kStatDepth == VADUSA_MAX_DEPTH && kStatTopk == VADUSA_MAX_DRAFT_TOPK, "statistics table follows the C ABI's maxima");
 
 vadusa_status sampling_dev(vadusa_ctx* ctx, const vadusa_sampling* s, SamplingDev* o) {
   if (!s) return fail(ctx, VADUSA_EINVAL, "sampling is NULL");
@@ -821,6 +824,7 @@ vadusa_status vadusa_init(const vadusa_weights* weights, const vadusa_config* cf
   CU(cudaEventCreateWithFlags(&ctx->ev_poll, cudaEventDisableTiming));
   CU(cudaMallocHost(&ctx->h_pinned, 4 * sizeof(int32_t)));
   CU(cudaMemsetAsync(ctx->wsp, 0, ctx->ws.tokens, ctx->stream));     // scalars, per-sequence state, trees
+  CU(cudaMemsetAsync(ctx->wsp + ctx->ws.acc_stats, 0, 2ull * kStatDepth * kStatTopk * 8, ctx->stream));
   // chain-shaped tree used by prefill: node i is the child of node i-1
   int32_t par[64], dep[64], rnk[64];
   unsigned long long anc[64];
@@ -1138,6 +1142,67 @@ vadusa_status vadusa_get_lengths(vadusa_ctx* ctx, int32_t* h_ctx_len) {
 vadusa_status vadusa_check(vadusa_ctx* ctx) {
   if (!ctx || !ctx->wsp) return VADUSA_EINVAL;
   return device_errors(ctx);
+}
+
+vadusa_status vadusa_accept_stats(vadusa_ctx* ctx, int64_t* h_tested, int64_t* h_accepted, int32_t reset) {
+  if (!ctx) return VADUSA_EINVAL;
+  if (!ctx->wsp) return fail(ctx, VADUSA_ESTATE, "context is not initialised");
+  if (!h_tested || !h_accepted) return fail(ctx, VADUSA_EINVAL, "statistics arrays are NULL");
+  const size_t n = (size_t)kStatDepth * kStatTopk;
+  static_assert(sizeof(int64_t) == sizeof(unsigned long long), "counter width");
+  CU(cudaMemcpyAsync(h_tested, ctx->wsp + ctx->ws.acc_stats, n * 8, cudaMemcpyDeviceToHost, ctx->stream));
+  CU(cudaMemcpyAsync(h_accepted, ctx->wsp + ctx->ws.acc_stats + n * 8, n * 8, cudaMemcpyDeviceToHost, ctx->stream));
+  if (reset) CU(cudaMemsetAsync(ctx->wsp + ctx->ws.acc_stats, 0, 2 * n * 8, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  return VADUSA_OK;
+}
+
+vadusa_status vadusa_build_sparse_tree(const double* h_prob, int32_t depth, int32_t topk, int32_t n_nodes,
+                                       int32_t* h_parent, int32_t* h_rank, double* h_expected_len) {
+  if (!h_prob || !h_parent || !h_rank) return VADUSA_EINVAL;
+  if (depth < 1 || depth > VADUSA_MAX_DEPTH || topk < 1 || topk > VADUSA_MAX_DRAFT_TOPK) return VADUSA_EINVAL;
+  if (n_nodes < 1 || n_nodes > VADUSA_MAX_TREE_NODES) return VADUSA_EINVAL;
+  struct Node { std::vector<int> path; double p; };
+  auto before = [](const Node& a, const Node& b) {       // higher probability, then shallower, then smaller path
+    if (a.p != b.p) return a.p > b.p;
+    if (a.path.size() != b.path.size()) return a.path.size() < b.path.size();
+    return a.path < b.path;
+  };
+  std::vector<Node> tree(1, Node{{}, 1.0}), frontier;
+  auto grow = [&](const Node& parent) {
+    if ((int)parent.path.size() == depth) return;
+    for (int r = 0; r < topk; ++r) {
+      Node c{parent.path, parent.p * h_prob[(size_t)parent.path.size() * topk + r]};
+      c.path.push_back(r);
+      frontier.push_back(c);
+    }
+  };
+  grow(tree[0]);
+  double expected = 1.0;
+  while ((int)tree.size() < n_nodes) {
+    if (frontier.empty()) return VADUSA_EINVAL;
+    size_t best = 0;
+    for (size_t i = 1; i < frontier.size(); ++i)
+      if (before(frontier[i], frontier[best])) best = i;
+    const Node pick = frontier[best];
+    frontier.erase(frontier.begin() + (long)best);
+    expected += pick.p;
+    tree.push_back(pick);
+    grow(pick);
+  }
+  std::sort(tree.begin(), tree.end(), [](const Node& a, const Node& b) {
+    return a.path.size() != b.path.size() ? a.path.size() < b.path.size() : a.path < b.path;
+  });
+  std::map<std::vector<int>, int> index;
+  for (int i = 0; i < n_nodes; ++i) index[tree[i].path] = i;
+  for (int i = 0; i < n_nodes; ++i) {
+    if (tree[i].path.empty()) { h_parent[i] = -1; h_rank[i] = 0; continue; }
+    std::vector<int> up(tree[i].path.begin(), tree[i].path.end() - 1);
+    h_parent[i] = index[up];
+    h_rank[i] = tree[i].path.back();
+  }
+  if (h_expected_len) *h_expected_len = expected;
+  return VADUSA_OK;
 }
 
 int64_t vadusa_kernel_launches(const vadusa_ctx* ctx) { return ctx ? ctx->launches : 0; }

@@ -11,6 +11,8 @@ typedef __nv_bfloat16 bf16;
 constexpr int kKvBlock = 64;         // tokens per KV block
 constexpr int kMaxNodes = 64;        // one 64-bit ancestor word per node
 constexpr int kMaxPath = 16;         // longest root path
+constexpr int kStatDepth = 15;       // acceptance statistics: draft heads x top-k ranks (the C ABI's maxima)
+constexpr int kStatTopk = 16;
 constexpr int kMaxTopk = 16;
 
 // bits of the device error word

@@ -114,6 +114,7 @@ struct WorkspaceLayout {
   int64_t att_xch;                       // fp32 split-KV exchange of the attention kernel: 296 slots of 64*64+128 floats
   int64_t gemm_part;                     // fp32 split-K exchange of the tensor-core products (kGemmPartBytes)
   int64_t ln_stats;                      // per-group LayerNorm statistics for the fused products (kLnStatsBytes)
+  int64_t acc_stats;                     // uint64 [2][VADUSA_MAX_DEPTH][VADUSA_MAX_DRAFT_TOPK]: edges tested, edges accepted
   int64_t gen_out, gen_len;              // int32 [B][kGenHostCap], int32 [B] (vadusa_generate_host staging)
   // prefill: one row per prefix chunk of a pass (R = pass_rows)
   int64_t pf_ctx_len, pf_nvalid, pf_seq, pf_last;   // int32 [R]: tokens before the chunk, its length, its sequence, sequence if last chunk else -1
@@ -149,6 +150,7 @@ inline WorkspaceLayout workspace_layout(const vadusa_config* c) {
   w.att_xch = take(296ll * (64 * 64 + 128) * 4);
   w.gemm_part = take(kGemmPartBytes);
   w.ln_stats = take(kLnStatsBytes);
+  w.acc_stats = take(2ll * VADUSA_MAX_DEPTH * VADUSA_MAX_DRAFT_TOPK * 8);
   w.gen_out = take(B * kGenHostCap * 4); w.gen_len = take(B * 4);
   w.pf_ctx_len = take(R * 4); w.pf_nvalid = take(R * 4); w.pf_seq = take(R * 4); w.pf_last = take(R * 4);
   w.pf_block_table = take(R * (int64_t)c->max_blocks_per_seq * 4);

@@ -84,6 +84,9 @@ class LockstepReport:
     max_logit_err: float = 0.0
     max_attn_err: float = 0.0
     accept_lens: List[int] = field(default_factory=list)
+    # acceptance tests by (draft head, rank) on the compared iterations: applied / passed
+    tested: np.ndarray = field(default_factory=lambda: np.zeros((15, 16), dtype=np.int64))
+    accepted: np.ndarray = field(default_factory=lambda: np.zeros((15, 16), dtype=np.int64))
 
 
 def lockstep(g, table, model, states: Dict[int, "O.State"], template, sp_oracle, sp_gpu, n_iters: int,
@@ -181,6 +184,9 @@ def lockstep(g, table, model, states: Dict[int, "O.State"], template, sp_oracle,
                 acc = {0}
                 for n in range(1, N):
                     p = int(template.parent[n])
+                    if p in acc:
+                        rep.tested[int(template.depth[n]) - 1, int(template.rank[n])] += 1
+                        rep.accepted[int(template.depth[n]) - 1, int(template.rank[n])] += int(tr.edge_ok[n])
                     if p in acc and tr.edge_ok[n]:
                         acc.add(n); want |= 1 << n
                 assert int(eb[b]) == want, f"it {it} seq {b}: edge bits {int(eb[b]):x} != {want:x}"

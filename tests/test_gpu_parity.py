@@ -147,6 +147,10 @@ def test_toy_planted_paths_are_accepted(dtype, tau, temperature, top_p, rule):
     rep = lockstep(g, table, model, states, tpl, so, sg, 8, dtype, oracle_mode="memo", planted=planted)
     if rule == 0:            # under rule 1 the noisy truth need not be among the plain top-tau
         assert max(rep.accept_lens) == tpl.max_depth + 1
+    # the kernel's acceptance statistics (input of the sparse-tree construction, Sec. II-D) count the same tests
+    tested, accepted = g.accept_stats()
+    assert np.array_equal(tested, rep.tested) and np.array_equal(accepted, rep.accepted)
+    assert tested.sum() > 0 and (rule != 0 or accepted[1:].sum() > 0)
     if tau == 1:
         for b, st in states.items():
             assert st.tokens == planted[b][:len(st.tokens)]
