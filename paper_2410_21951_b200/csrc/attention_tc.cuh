@@ -8,15 +8,15 @@
 // warps 2-3 (lanes 64..127) on keys 32..63.  Per page:
 //   S = Q K^T      tcgen05.mma, A = Q tile, B = K tile, D in one of two TMEM score buffers (columns
 //                  0..63 / 64..127), issued one page ahead so that it overlaps the previous softmax
-//   softmax        each thread reads its 32 scores, the two threads of a row agree on the
-//                  scaling maximum through shared memory, and the weights go back to TMEM as
+//   softmax        each thread reads its 32 scores, keeps a scaling maximum of its own for its key
+//                  half of the row, and the weights go back to TMEM as
 //                  two bf16 halves (p = hi + lo, 16 significant bits) over the score columns,
 //                  zero in the other thread's key range
 //   O += P V       tcgen05.mma with A from TMEM (hi then lo), B = V tile (MN-major), accumulating
 //                  in TMEM columns 128..191; lanes r and r + 64 hold the two key-halves' sums
 // The scaling maximum of a row only moves when the page maximum exceeds it by more than 2^6
 // (p <= 64 is harmless in fp32 / bf16); then the row's accumulator is rescaled in TMEM.
-// At the end rows r and r + 64 are added; splits are merged through an exchange area in global
+// At the end rows r and r + 64 are brought to a common scale and added; splits are merged through an exchange area in global
 // memory (L2) in a fixed order.  Warps: 0-3 softmax, warp 4 lane 0 TMA producer, warp 5 TMEM owner / MMA issuer.
 #pragma once
 #include "tc.cuh"
@@ -52,7 +52,6 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // D[tmem] (+)= A[tmem] * B[smem] for one K step of 16 elements (A: lane = row, 8 columns of bf16 pairs).
 __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, bool accumulate) {
@@ -88,7 +87,7 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t q_addr = base, ring = base + 2 * kAttTileBytes;
   uint8_t* ring_ptr = base_ptr + 2 * kAttTileBytes;
-  float* xmax = reinterpret_cast<float*>(ring_ptr + kAttRingBytes);          // [2][128] scaling maxima exchange
+  float* lx = reinterpret_cast<float*>(ring_ptr + kAttRingBytes);            // end of the kernel: [128] partial sums, [128] scaling maxima
   const uint32_t bars = ring + kAttRingBytes + 1024;
   const uint32_t full0 = bars, empty0 = bars + 8 * S, bar_q = bars + 16 * S, bar_s0 = bar_q + 8, bar_p = bar_q + 24,
                  bar_o = bar_q + 32, holder = bar_q + 40;      // bar_s0, bar_s0 + 8: one per score buffer
@@ -205,11 +204,7 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
       float sc[32];
       tmem_ld32(tsp + 32 * half, sc);
       const int key0 = (p0 + i) * kKvBlock + 32 * half;
-      float mx = -INFINITY;
-      if (key0 + 32 <= ctx) {                 // all 32 keys inside the context: every key visible
-#pragma unroll
-        for (int j = 0; j < 32; ++j) mx = fmaxf(mx, sc[j]);
-      } else {
+      if (key0 + 32 > ctx) {
         // bit j of vis: key key0 + j is visible (context, or an ancestor-or-self tree node; the ancestor
         // word has no bits at or above the node count).  Selects, not branches: the rows of a warp differ.
         const int rel = key0 - ctx;           // > -32 here
@@ -217,11 +212,12 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
         if (rel >= 0) vis = rel < 64 ? (uint32_t)(amask >> rel) : 0u;
         else vis = ((1u << (-rel)) - 1u) | (uint32_t)(amask << (-rel));
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          sc[j] = ((vis >> j) & 1u) ? sc[j] : -INFINITY;
-          mx = fmaxf(mx, sc[j]);
-        }
-      }
+        for (int j = 0; j < 32; ++j) sc[j] = ((vis >> j) & 1u) ? sc[j] : -INFINITY;
+      }                                       // else: all 32 keys inside the context, every key visible
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+      for (int j = 0; j < 32; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
+      float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       if ((p0 + i + 1) * kKvBlock > total && tid < 64) {   // rows of V past the tree may hold anything: zero them
         const int valid = total - (p0 + i) * kKvBlock;
         if (tid >= valid) {
@@ -231,10 +227,9 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
         }
         fence_proxy_async_smem();
       }
-      // the two threads of a row agree on the page maximum
-      xmax[(i & 1) * 128 + tid] = mx;
-      softmax_bar_sync();
-      mx = fmaxf(mx, xmax[(i & 1) * 128 + (tid ^ 64)]) * scale_log2e;     // raw scores; the (positive) scale moves into the exponent
+      // each key half of a row keeps its own scaling maximum (the halves accumulate in separate TMEM lanes
+      // and are brought to a common scale once, at the end)
+      mx *= scale_log2e;                      // raw scores; the (positive) scale moves into the exponent
       // move the scaling maximum only when the page maximum exceeds it by more than the step
       float factor = 1.f;
       if (mx > m_use + kAttRescaleStep || m_use == -INFINITY) {
@@ -291,7 +286,6 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
 
   // ---- output: rows r and r + 64 are the two key-halves of node r
   float* Ox = reinterpret_cast<float*>(ring_ptr);          // [64][64] fp32 exchange, row r rotated by 4r columns
-  float* lx = xmax;                                        // [128] partial sums; [128..255] scaling maxima
   float o_acc[64];
   if (warp < 4) {
     const uint32_t trow = tmem + ((uint32_t)(32 * warp) << 16);
@@ -303,6 +297,7 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
       for (int e = 0; e < 64; ++e) o_acc[e] = 0.f;
     }
     lx[tid] = l_run;
+    lx[128 + tid] = m_use;
     if (tid >= 64) {
 #pragma unroll
       for (int e = 0; e < 64; ++e) Ox[(tid - 64) * 64 + ((e + 4 * tid) & 63)] = o_acc[e];
@@ -310,9 +305,13 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
   }
   __syncthreads();
   if (tid < 64) {
+    // the two key halves of the row on a common scale
+    const float m1 = lx[128 + tid + 64], mm = fmaxf(m_use, m1);
+    const float w0 = (m_use == -INFINITY) ? 0.f : fast_exp2(m_use - mm), w1 = (m1 == -INFINITY) ? 0.f : fast_exp2(m1 - mm);
 #pragma unroll
-    for (int e = 0; e < 64; ++e) o_acc[e] += Ox[tid * 64 + ((e + 4 * tid) & 63)];
-    l_run += lx[tid + 64];
+    for (int e = 0; e < 64; ++e) o_acc[e] = o_acc[e] * w0 + Ox[tid * 64 + ((e + 4 * tid) & 63)] * w1;
+    l_run = l_run * w0 + lx[tid + 64] * w1;
+    m_use = mm;
   }
   if (splits == 1) {
     if (tid < 64 && tid < N) {
