@@ -51,7 +51,7 @@ extern "C" {
 #endif
 
 #define VADUSA_ABI_VERSION 2u
-#define VADUSA_MAX_TREE_NODES 64   /* one 64-bit ancestor word per node */
+#define VADUSA_MAX_TREE_NODES 128  /* two 64-bit ancestor words per node (the paper's 64-, 96- and 128-node trees) */
 #define VADUSA_MAX_DRAFT_TOPK 16
 #define VADUSA_MAX_DEPTH 15        /* a root path has at most 16 nodes */
 
@@ -217,8 +217,9 @@ vadusa_status vadusa_verify_step(vadusa_ctx *ctx, const int32_t *tree_tokens_ove
  * forced_best_node: int32 [batch] overrides the winner (test hook; -1 entries keep the rule).
  * accept_len int32 [batch]; path_nodes, path_tokens int32 [batch][VADUSA_MAX_DEPTH+1]
  * (entries beyond accept_len are -1); kv_slots int64 [batch][VADUSA_MAX_DEPTH+1]:
- * block * kv_block + offset of every committed token; edge_bits uint64 [batch]: bit n set
- * iff edge parent(n)->n was tested and accepted (bit 0 always set); next_root int32 [batch]:
+ * block * kv_block + offset of every committed token; edge_bits uint64 [batch][W], W = 1 if
+ * the configuration's max_tree_nodes <= 64, else 2: bit n (of word n / 64) set iff edge
+ * parent(n)->n was tested and accepted (bit 0 always set); next_root int32 [batch]:
  * the base head's sample for the position after the winner. */
 vadusa_status vadusa_accept_and_commit(vadusa_ctx *ctx, const vadusa_sampling *sampling,
                                        const int32_t *forced_best_node, int32_t *accept_len,

@@ -10,7 +10,8 @@ struct AcceptOut {            // optional user-visible outputs (any may be null)
   int32_t* path_nodes;        // [batch][kMaxPath]
   int32_t* path_tokens;       // [batch][kMaxPath]
   long long* kv_slots;        // [batch][kMaxPath]
-  unsigned long long* edge_bits;  // [batch]
+  unsigned long long* edge_bits;  // [batch][edge_words]
+  long long edge_words;       // 1 (trees of up to 64 nodes) or 2 (a full word: the struct's bytes key the graph cache)
   int32_t* next_root;         // [batch]
 };
 
@@ -44,7 +45,7 @@ __global__ void __launch_bounds__(256) accept_kernel(
   float* probs = keys + ld;
   __shared__ int s_parent[kMaxNodes], s_depth[kMaxNodes], s_tok[kMaxNodes];
   __shared__ int s_child[kMaxNodes], s_ok[kMaxNodes], s_nchild;
-  __shared__ unsigned long long s_edges, s_acc;
+  __shared__ unsigned long long s_edges[2], s_acc[2];    // bits 0..63, 64..127
   __shared__ int s_path[kMaxPath], s_best, s_len, s_eos;
   __shared__ Best bscratch[32];
   __shared__ float fscratch[32];
@@ -55,7 +56,7 @@ __global__ void __launch_bounds__(256) accept_kernel(
     if (tid == 0) {
       st.commit_len[b] = 0;
       if (out.accept_len) out.accept_len[b] = 0;
-      if (out.edge_bits) out.edge_bits[b] = 0ull;
+      if (out.edge_bits) for (int w = 0; w < (int)out.edge_words; ++w) out.edge_bits[b * out.edge_words + w] = 0ull;
       if (out.next_root) out.next_root[b] = -1;
     }
     if (tid < kMaxPath) {
@@ -73,7 +74,7 @@ __global__ void __launch_bounds__(256) accept_kernel(
     s_depth[tid] = in ? tree.depth[to + tid] : -1;
     s_tok[tid] = in ? tokens[(long long)b * N + tid] : -1;
   }
-  if (tid == 0) { s_edges = 1ull; s_acc = 1ull; }
+  if (tid == 0) { s_edges[0] = 1ull; s_acc[0] = 1ull; s_edges[1] = 0ull; s_acc[1] = 0ull; }
   __syncthreads();
   int maxdepth = 0;
   for (int n = 0; n < nv; ++n) maxdepth = max(maxdepth, s_depth[n]);
@@ -82,7 +83,7 @@ __global__ void __launch_bounds__(256) accept_kernel(
 
   for (int d = 0; d < maxdepth && fb < 0; ++d) {
     for (int p = 0; p < nv; ++p) {
-      if (s_depth[p] != d || !((s_acc >> p) & 1ull)) continue;       // uniform: shared memory
+      if (s_depth[p] != d || !bit_at(s_acc[0], s_acc[1], p)) continue;  // uniform: shared memory
       __syncthreads();
       if (tid == 0) s_nchild = 0;
       __syncthreads();
@@ -128,7 +129,7 @@ __global__ void __launch_bounds__(256) accept_kernel(
       __syncthreads();
       if (tid == 0) {
         for (int i = 0; i < nchild; ++i)
-          if (s_ok[i]) { s_edges |= 1ull << s_child[i]; s_acc |= 1ull << s_child[i]; }
+          if (s_ok[i]) { const int c = s_child[i]; s_edges[c >> 6] |= 1ull << (c & 63); s_acc[c >> 6] |= 1ull << (c & 63); }
       }
       if (tid < nchild && st.stats && d < kStatDepth) {
         const int r = tree.rank[to + s_child[tid]];
@@ -146,7 +147,7 @@ __global__ void __launch_bounds__(256) accept_kernel(
     if (fb >= 0 && fb < nv) best = fb;
     else
       for (int n = 1; n < nv; ++n)
-        if (((s_acc >> n) & 1ull) && s_depth[n] > s_depth[best]) best = n;
+        if (bit_at(s_acc[0], s_acc[1], n) && s_depth[n] > s_depth[best]) best = n;
     int len = min(s_depth[best] + 1, kMaxPath);
     int n = best;
     for (int j = len - 1; j >= 0; --j) { s_path[j] = n; n = s_parent[n]; }
@@ -188,7 +189,7 @@ __global__ void __launch_bounds__(256) accept_kernel(
     st.gen_count[b] = g;
     if (s_eos || (st.target > 0 && g >= st.target)) { st.nvalid[b] = 0; atomicAdd(st.done_count, 1); }
     if (out.accept_len) out.accept_len[b] = len;
-    if (out.edge_bits) out.edge_bits[b] = s_edges;
+    if (out.edge_bits) for (int w = 0; w < (int)out.edge_words; ++w) out.edge_bits[b * out.edge_words + w] = s_edges[w];
     if (out.next_root) out.next_root[b] = nroot;
   }
 }

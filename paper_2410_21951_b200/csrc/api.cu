@@ -367,8 +367,8 @@ bool ln_product(vadusa_ctx* ctx, int cls, const float* x, const float* g, const 
 // (Ragged batches are balanced by visiting the sequences longest first, see seq_order_kernel.)
 int attention_splits(const vadusa_ctx* ctx, int n_nodes) {
   int splits = 1;
-  while (splits < 8 && ctx->cfg.n_heads * ctx->batch * splits * 2 <= 296) splits *= 2;
-  (void)n_nodes;
+  const int ntile = (n_nodes + 63) / 64;                 // CTAs per (head, sequence): one per 64 nodes
+  while (splits < 8 && ctx->cfg.n_heads * ctx->batch * ntile * splits * 2 <= 296) splits *= 2;
   return splits;
 }
 
@@ -378,7 +378,8 @@ vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeVi
   const int dh = c.d_model / c.n_heads;
   const KvGeom g = geom_of(ctx);
   const float scale = (float)(1.0 / sqrt((double)dh));
-  dim3 grid(c.n_heads, ctx->batch);
+  const int ntile = (tv.n_nodes + 63) / 64;
+  dim3 grid(c.n_heads, ctx->batch * ntile);
   const size_t smem = (size_t)(64 * dh * 3 + 64 + 64 * 64) * sizeof(float);   // = attention_smem(dh)
   auto go = [&](auto kern) -> vadusa_status {
     PROF(ctx, K_ATTENTION);
@@ -401,7 +402,7 @@ vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeVi
       const int layer = (int)((reinterpret_cast<const char*>(pool) - reinterpret_cast<const char*>(c.kv_pool)) /
                               (g.layer_stride * (long long)sizeof(bf16)));
       cudaLaunchConfig_t lc = {};
-      lc.gridDim = dim3(c.n_heads, ctx->batch, splits);
+      lc.gridDim = dim3(c.n_heads, ctx->batch * ntile, splits);
       lc.blockDim = dim3(kAttThreads);
       lc.dynamicSmemBytes = kAttSmemBytes;
       lc.stream = ctx->stream;
@@ -826,9 +827,12 @@ vadusa_status vadusa_init(const vadusa_weights* weights, const vadusa_config* cf
   CU(cudaMemsetAsync(ctx->wsp, 0, ctx->ws.tokens, ctx->stream));     // scalars, per-sequence state, trees
   CU(cudaMemsetAsync(ctx->wsp + ctx->ws.acc_stats, 0, 2ull * kStatDepth * kStatTopk * 8, ctx->stream));
   // chain-shaped tree used by prefill: node i is the child of node i-1
-  int32_t par[64], dep[64], rnk[64];
-  unsigned long long anc[64];
-  for (int i = 0; i < 64; ++i) { par[i] = i - 1; dep[i] = i; rnk[i] = 0; anc[i] = i == 63 ? ~0ull : ((1ull << (i + 1)) - 1); }
+  constexpr int T = VADUSA_MAX_TREE_NODES;
+  static_assert(T == kMaxNodes, "node limit of the kernels");
+  int32_t par[T], dep[T], rnk[T];
+  unsigned long long anc[2 * T];
+  auto low_bits = [](int n) { return n <= 0 ? 0ull : n >= 64 ? ~0ull : ((1ull << n) - 1); };   // n lowest bits set
+  for (int i = 0; i < T; ++i) { par[i] = i - 1; dep[i] = i; rnk[i] = 0; anc[2 * i] = low_bits(i + 1); anc[2 * i + 1] = low_bits(i + 1 - 64); }
   CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.chain_parent, par, sizeof(par), cudaMemcpyHostToDevice, ctx->stream));
   CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.chain_depth, dep, sizeof(dep), cudaMemcpyHostToDevice, ctx->stream));
   CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.chain_rank, rnk, sizeof(rnk), cudaMemcpyHostToDevice, ctx->stream));
@@ -863,19 +867,20 @@ vadusa_status vadusa_set_tree(vadusa_ctx* ctx, int32_t n_nodes, const int32_t* h
     copies = ctx->batch;
   }
   std::vector<int32_t> depth((size_t)copies * n_nodes);
-  std::vector<unsigned long long> anc((size_t)copies * n_nodes);
+  std::vector<unsigned long long> anc((size_t)copies * n_nodes * 2);
   int max_rank = 0, max_depth = 0;
   for (int s = 0; s < copies; ++s) {
     const int32_t* par = h_parent + (size_t)s * n_nodes;
     const int32_t* rnk = h_rank + (size_t)s * n_nodes;
     int32_t* dep = depth.data() + (size_t)s * n_nodes;
-    unsigned long long* an = anc.data() + (size_t)s * n_nodes;
+    unsigned long long* an = anc.data() + (size_t)s * n_nodes * 2;       // two words per node
     if (par[0] != -1) return fail(ctx, VADUSA_EINVAL, "node 0 must be the root (parent -1)");
-    dep[0] = 0; an[0] = 1ull;
+    dep[0] = 0; an[0] = 1ull; an[1] = 0ull;
     for (int n = 1; n < n_nodes; ++n) {
       if (par[n] < 0 || par[n] >= n) return fail(ctx, VADUSA_EINVAL, "node %d: parent %d must precede it", n, par[n]);
       dep[n] = dep[par[n]] + 1;
-      an[n] = an[par[n]] | (1ull << n);
+      an[2 * n] = an[2 * par[n]] | (n < 64 ? 1ull << n : 0ull);
+      an[2 * n + 1] = an[2 * par[n] + 1] | (n >= 64 ? 1ull << (n - 64) : 0ull);
       if (dep[n] > VADUSA_MAX_DEPTH) return fail(ctx, VADUSA_EINVAL, "node %d: deeper than %d", n, VADUSA_MAX_DEPTH);
       if (!per_sequence) {
         if (dep[n] > ctx->cfg.n_draft_heads) return fail(ctx, VADUSA_EINVAL, "node %d: depth %d exceeds the number of draft heads", n, dep[n]);
@@ -897,7 +902,7 @@ vadusa_status vadusa_set_tree(vadusa_ctx* ctx, int32_t n_nodes, const int32_t* h
   CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.tree_parent, h_parent, n4, cudaMemcpyHostToDevice, ctx->stream));
   CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.tree_rank, h_rank, n4, cudaMemcpyHostToDevice, ctx->stream));
   CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.tree_depth, depth.data(), n4, cudaMemcpyHostToDevice, ctx->stream));
-  CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.tree_anc, anc.data(), (size_t)copies * n_nodes * 8, cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.tree_anc, anc.data(), (size_t)copies * n_nodes * 16, cudaMemcpyHostToDevice, ctx->stream));
   CU(cudaStreamSynchronize(ctx->stream));
   ctx->n_nodes = n_nodes;
   ctx->tree_per_seq = per_sequence ? 1 : 0;
@@ -1034,7 +1039,7 @@ vadusa_status vadusa_accept_and_commit(vadusa_ctx* ctx, const vadusa_sampling* s
   SamplingDev sp;
   if (vadusa_status s = sampling_dev(ctx, sampling, &sp)) return s;
   AcceptOut out{accept_len, path_nodes, path_tokens, reinterpret_cast<long long*>(kv_slots),
-                reinterpret_cast<unsigned long long*>(edge_bits), next_root};
+                reinterpret_cast<unsigned long long*>(edge_bits), ctx->cfg.max_tree_nodes > 64 ? 2 : 1, next_root};
   const std::string key = KeyBuilder("accept").add(sp).add(forced_best_node).add(out).add(ctx->batch).add(ctx->n_nodes)
                               .add(ctx->tree_per_seq).add(ctx->block_table).k;
   vadusa_status s = run_graphed(ctx, key, [&]() -> vadusa_status {
@@ -1057,7 +1062,7 @@ vadusa_status vadusa_generate(vadusa_ctx* ctx, const vadusa_sampling* sampling, 
   const int64_t launches0 = ctx->launches;
   const int limit = max_iters > 0 ? max_iters : max_new_tokens;
   const TreeView tv = tree_of(ctx, false);
-  AcceptOut none{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  AcceptOut none{nullptr, nullptr, nullptr, nullptr, nullptr, 1, nullptr};
   CU(cudaMemsetAsync(ctx->wsp + ctx->ws.gen_count, 0, ctx->batch * 4, ctx->stream));
   CU(cudaMemsetAsync(done_word(ctx), 0, 4, ctx->stream));
   if (vadusa_status s = set_active(ctx, ctx->n_nodes)) return s;

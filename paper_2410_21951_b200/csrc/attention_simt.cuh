@@ -19,22 +19,23 @@ __global__ void __launch_bounds__(256) tree_attention_simt_kernel(
   float* Ks = Qs + 64 * DH;               // [64][DH+1]
   float* Vs = Ks + 64 * (DH + 1);         // [64][DH]
   float* Ps = Vs + 64 * DH;               // [64][64]
-  const int h = blockIdx.x, b = blockIdx.y;
-  const int N = tree.n_nodes, nv = nvalid[b], S = ctx_len[b];
+  const int N = tree.n_nodes, ntile = (N + 63) >> 6;
+  const int h = blockIdx.x, b = (int)blockIdx.y / ntile, nb = 64 * ((int)blockIdx.y % ntile);   // nodes nb .. nb+63
+  const int nv = nvalid[b], S = ctx_len[b];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const unsigned long long* anc = tree.anc + tree.off(b);
 
   for (int i = threadIdx.x; i < 64 * DH; i += 256) {
     const int n = i / DH, e = i % DH;
-    Qs[i] = (n < N) ? to_f<T>(q[((long long)b * N + n) * d_model + h * DH + e]) : 0.f;
+    Qs[i] = (nb + n < N) ? to_f<T>(q[((long long)b * N + nb + n) * d_model + h * DH + e]) : 0.f;
   }
   float O[8][R], mrun[8], lrun[8];
-  unsigned long long amask[8];
+  unsigned long long alo[8], ahi[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     mrun[i] = -INFINITY; lrun[i] = 0.f;
     const int n = warp + 8 * i;
-    amask[i] = (n < nv) ? anc[n] : 0ull;
+    alo[i] = ahi[i] = 0ull;
+    if (nb + n < nv) tree.anc_of(b, nb + n, alo[i], ahi[i]);
 #pragma unroll
     for (int c = 0; c < R; ++c) O[i][c] = 0.f;
   }
@@ -55,14 +56,14 @@ __global__ void __launch_bounds__(256) tree_attention_simt_kernel(
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int n = warp + 8 * i;
-      if (n >= nv) continue;
+      if (nb + n >= nv) continue;
       float s[2];
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         const int j = lane + 32 * c, p = t0 + j;
         float a = 0.f;
         for (int e = 0; e < DH; ++e) a = fmaf(Qs[n * DH + e], Ks[j * (DH + 1) + e], a);
-        const bool vis = p < S || (p < total && ((amask[i] >> (p - S)) & 1ull));
+        const bool vis = p < S || (p < total && bit_at(alo[i], ahi[i], p - S));
         s[c] = vis ? a * scale : -INFINITY;
       }
       const float mnew = fmaxf(mrun[i], warp_max(fmaxf(s[0], s[1])));
@@ -86,11 +87,11 @@ __global__ void __launch_bounds__(256) tree_attention_simt_kernel(
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const int n = warp + 8 * i;
-    if (n >= N) continue;
+    if (nb + n >= N) continue;
 #pragma unroll
     for (int c = 0; c < R; ++c) {
-      const float v = (n < nv && lrun[i] > 0.f) ? O[i][c] / lrun[i] : 0.f;
-      out[((long long)b * N + n) * d_model + h * DH + lane + 32 * c] = from_f<T>(v);
+      const float v = (nb + n < nv && lrun[i] > 0.f) ? O[i][c] / lrun[i] : 0.f;
+      out[((long long)b * N + nb + n) * d_model + h * DH + lane + 32 * c] = from_f<T>(v);
     }
   }
 }

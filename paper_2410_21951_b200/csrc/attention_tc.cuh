@@ -2,7 +2,8 @@
 // (head_dim 64).  Node n of sequence b attends to every cached position < ctx_len[b] and to
 // the tree slots ctx_len[b] + m whose bit m is set in anc[n] (paper Sec. II-A, tree attention).
 //
-// One CTA per (head, sequence, KV split); the splits of one (head, sequence) form a cluster.
+// One CTA per (head, sequence, tile of 64 nodes, KV split); the splits of one (head, sequence, tile) form a
+// cluster.  Trees of up to 128 nodes carry two 64-bit ancestor words per node.
 // The 64 query rows are stored twice in the 128-row Q operand, so the scores of row r appear in
 // TMEM lanes r and r + 64: warps 0-1 (lanes 0..63) work on keys 0..31 of every 64-key page,
 // warps 2-3 (lanes 64..127) on keys 32..63.  Per page:
@@ -111,7 +112,9 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
   const uint32_t tmem = *holder_ptr;
 
   grid_dep_wait();                            // q, K/V rows, lengths come from upstream kernels
-  const int b = order ? order[blockIdx.y] : (int)blockIdx.y;     // longest sequences first
+  // blockIdx.y = (sequence, tile of 64 nodes); longest sequences first
+  const int ntile = (N + 63) >> 6, qt = (int)blockIdx.y % ntile, node0 = 64 * qt;
+  const int b = order ? order[blockIdx.y / ntile] : (int)blockIdx.y / ntile;
   const int nv = nvalid[b], ctx = ctx_len[b];
   const int total = ctx + nv;
   const int npages = nv > 0 ? (total + kKvBlock - 1) / kKvBlock : 0;
@@ -134,8 +137,8 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
     }
     if (lane == 0 && ntiles > 0) {
       mbar_expect_tx(bar_q, 2 * kAttTileBytes);
-      tma_load_3d(q_addr, &tmQ, bar_q, h * 64, b * N, 0);
-      tma_load_3d(q_addr + kAttTileBytes, &tmQ, bar_q, h * 64, b * N, 0);      // the same rows again: lanes 64..127
+      tma_load_3d(q_addr, &tmQ, bar_q, h * 64, b * N + node0, 0);
+      tma_load_3d(q_addr + kAttTileBytes, &tmQ, bar_q, h * 64, b * N + node0, 0);      // the same rows again: lanes 64..127
     }
     bool ok = true;
     for (int i = 0; i < ntiles; ++i) {
@@ -195,7 +198,8 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
   } else {
     // ---- softmax: thread tid owns TMEM lane tid = query row (tid & 63), keys 32*half .. 32*half+31 of each page
     const int row = tid & 63, half = tid >> 6;
-    const unsigned long long amask = row < nv ? tree.anc[tree.off(b) + row] : 0ull;
+    unsigned long long alo = 0ull, ahi = 0ull;                     // ancestor-or-self bits of this row's node
+    if (node0 + row < nv) tree.anc_of(b, node0 + row, alo, ahi);
     const uint32_t trow = tmem + ((uint32_t)(32 * warp) << 16);
     for (int i = 0; i < ntiles; ++i) {
       if (!mbar_wait(bar_s0 + 8 * (i & 1), (i >> 1) & 1, err)) break;
@@ -209,8 +213,8 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
         // word has no bits at or above the node count).  Selects, not branches: the rows of a warp differ.
         const int rel = key0 - ctx;           // > -32 here
         uint32_t vis;
-        if (rel >= 0) vis = rel < 64 ? (uint32_t)(amask >> rel) : 0u;
-        else vis = ((1u << (-rel)) - 1u) | (uint32_t)(amask << (-rel));
+        if (rel >= 0) vis = rel < 128 ? bits32_at(alo, ahi, rel) : 0u;
+        else vis = ((1u << (-rel)) - 1u) | (uint32_t)(alo << (-rel));
 #pragma unroll
         for (int j = 0; j < 32; ++j) sc[j] = ((vis >> j) & 1u) ? sc[j] : -INFINITY;
       }                                       // else: all 32 keys inside the context, every key visible
@@ -314,9 +318,9 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
     m_use = mm;
   }
   if (splits == 1) {
-    if (tid < 64 && tid < N) {
-      const float inv = (tid < nv && l_run > 0.f) ? 1.f / l_run : 0.f;
-      uint4* dst = reinterpret_cast<uint4*>(out + ((long long)b * N + tid) * d_model + h * 64);
+    if (tid < 64 && node0 + tid < N) {
+      const float inv = (node0 + tid < nv && l_run > 0.f) ? 1.f / l_run : 0.f;
+      uint4* dst = reinterpret_cast<uint4*>(out + ((long long)b * N + node0 + tid) * d_model + h * 64);
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         uint4 v;
@@ -369,12 +373,12 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
             L = fmaf(ll[p], w, L);
             o.x = fmaf(oo[p].x, w, o.x); o.y = fmaf(oo[p].y, w, o.y); o.z = fmaf(oo[p].z, w, o.z); o.w = fmaf(oo[p].w, w, o.w);
           }
-        if (n < N) {
-          const float inv = (n < nv && L > 0.f) ? 1.f / L : 0.f;
+        if (node0 + n < N) {
+          const float inv = (node0 + n < nv && L > 0.f) ? 1.f / L : 0.f;
           uint2 v;
           v.x = pack_bf16(o.x * inv, o.y * inv);
           v.y = pack_bf16(o.z * inv, o.w * inv);
-          *reinterpret_cast<uint2*>(out + ((long long)b * N + n) * d_model + h * 64 + e4) = v;
+          *reinterpret_cast<uint2*>(out + ((long long)b * N + node0 + n) * d_model + h * 64 + e4) = v;
         }
       }
     }

@@ -9,7 +9,7 @@ namespace vadusa {
 typedef __nv_bfloat16 bf16;
 
 constexpr int kKvBlock = 64;         // tokens per KV block
-constexpr int kMaxNodes = 64;        // one 64-bit ancestor word per node
+constexpr int kMaxNodes = 128;       // two 64-bit ancestor words per node
 constexpr int kMaxPath = 16;         // longest root path
 constexpr int kStatDepth = 15;       // acceptance statistics: draft heads x top-k ranks (the C ABI's maxima)
 constexpr int kStatTopk = 16;
@@ -75,11 +75,28 @@ struct TreeView {
   const int32_t* parent;
   const int32_t* depth;
   const int32_t* rank;
-  const unsigned long long* anc;   // ancestor-or-self bits
+  const unsigned long long* anc;   // ancestor-or-self bits, two words per node (bits 0..63, 64..127)
   int n_nodes;
   int per_seq;
   __device__ __forceinline__ int off(int b) const { return per_seq ? b * n_nodes : 0; }
+  __device__ __forceinline__ void anc_of(int b, int n, unsigned long long& lo, unsigned long long& hi) const {
+    const unsigned long long* p = anc + 2ll * (off(b) + n);
+    lo = p[0]; hi = p[1];
+  }
 };
+
+// Bits [rel, rel + 32) of the 128-bit word (hi:lo), rel in [0, 128); bits beyond 127 read as zero.
+__device__ __forceinline__ uint32_t bits32_at(unsigned long long lo, unsigned long long hi, int rel) {
+  if (rel < 64) {
+    uint32_t v = (uint32_t)(lo >> rel);
+    if (rel > 32) v |= (uint32_t)(hi << (64 - rel));
+    return v;
+  }
+  return (uint32_t)(hi >> (rel - 64));
+}
+__device__ __forceinline__ bool bit_at(unsigned long long lo, unsigned long long hi, int i) {
+  return ((i < 64 ? lo >> i : hi >> (i - 64)) & 1ull) != 0ull;
+}
 
 // Four consecutive values rounded to T and stored as one vector.
 template <typename T> __device__ __forceinline__ void store4(T* p, float a, float b, float c, float d);

@@ -100,8 +100,8 @@ struct WorkspaceLayout {
   int64_t ctx_len, nvalid, gen_count, commit_base, commit_len, best, root, saved_nvalid;   // int32 [B]
   int64_t commit_path;                   // int32 [B][16]
   int64_t seq_order;                     // int32 [R]: rows by descending context length
-  int64_t tree_parent, tree_depth, tree_rank, tree_anc;       // [B*64] (anc: uint64)
-  int64_t chain_parent, chain_depth, chain_rank, chain_anc;   // [64]
+  int64_t tree_parent, tree_depth, tree_rank, tree_anc;       // [B*128] (anc: two uint64 per node)
+  int64_t chain_parent, chain_depth, chain_rank, chain_anc;   // [128]
   int64_t tokens, stage_tokens;          // int32 [M]
   int64_t kv_row;                        // int64 [M]: element offset of the row's K slot (head 0) in a layer's pool, -1: none
   int64_t topk;                          // int32 [B][heads][k]
@@ -134,10 +134,11 @@ inline WorkspaceLayout workspace_layout(const vadusa_config* c) {
   w.saved_nvalid = take(B * 4);
   w.commit_path = take(B * 16 * 4);
   w.seq_order = take(R * 4);
-  w.tree_parent = take(B * 64 * 4); w.tree_depth = take(B * 64 * 4); w.tree_rank = take(B * 64 * 4);
-  w.tree_anc = take(B * 64 * 8);
-  w.chain_parent = take(64 * 4); w.chain_depth = take(64 * 4); w.chain_rank = take(64 * 4);
-  w.chain_anc = take(64 * 8);
+  const int64_t T = VADUSA_MAX_TREE_NODES;
+  w.tree_parent = take(B * T * 4); w.tree_depth = take(B * T * 4); w.tree_rank = take(B * T * 4);
+  w.tree_anc = take(B * T * 16);
+  w.chain_parent = take(T * 4); w.chain_depth = take(T * 4); w.chain_rank = take(T * 4);
+  w.chain_anc = take(T * 16);
   w.tokens = take(M * 4); w.stage_tokens = take(M * 4);
   w.kv_row = take(M * 8);
   w.topk = take(B * hd * c->draft_topk * 4);

@@ -109,7 +109,8 @@ def lockstep(g, table, model, states: Dict[int, "O.State"], template, sp_oracle,
     pnodes = torch.zeros(B, MAX_PATH, dtype=torch.int32, device=dev)
     ptoks = torch.zeros(B, MAX_PATH, dtype=torch.int32, device=dev)
     slots = torch.zeros(B, MAX_PATH, dtype=torch.int64, device=dev)
-    ebits = torch.zeros(B, dtype=torch.int64, device=dev)
+    ewords = 2 if g.cfg.max_tree_nodes > 64 else 1             # one 64-bit word of edge bits per 64 nodes
+    ebits = torch.zeros(B, ewords, dtype=torch.int64, device=dev)
     nroot = torch.zeros(B, dtype=torch.int32, device=dev)
     tol = TOL[dtype]
     MARGIN = MARGINS[dtype]
@@ -163,6 +164,7 @@ def lockstep(g, table, model, states: Dict[int, "O.State"], template, sp_oracle,
         at = attn.float().cpu().numpy().astype(np.float64) if check_attn else None
         al, pn, pt, sl = acc_len.cpu().numpy(), pnodes.cpu().numpy(), ptoks.cpu().numpy(), slots.cpu().numpy()
         eb = ebits.cpu().numpy().astype(np.uint64)
+        eb = [sum(int(eb[b, w]) << (64 * w) for w in range(ewords)) for b in range(B)]
         for b, tr in traces.items():
             err = float(np.abs(lg[b] - tr.node_logits).max())
             rep.max_logit_err = max(rep.max_logit_err, err)

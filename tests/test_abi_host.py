@@ -76,7 +76,7 @@ def test_pack_weights_round_trip():
 
 
 @pytest.mark.parametrize("field,value", [("d_model", 100), ("n_heads", 3), ("kv_block", 32), ("dtype", 2),
-                                          ("max_tree_nodes", 65), ("draft_topk", 0), ("n_draft_heads", 16),
+                                          ("max_tree_nodes", 129), ("prefill_rows", -1), ("draft_topk", 0), ("n_draft_heads", 16),
                                           ("struct_size", 8), ("abi_version", 99), ("kv_num_blocks", 0)])
 def test_bad_configurations_are_rejected(field, value):
     L = P.lib()

@@ -212,6 +212,28 @@ def test_unmasked_eos_ends_a_sequence_and_drops_what_follows_it():
     g.check()
 
 
+@pytest.mark.parametrize("dtype,nodes", [("bf16", 96), ("fp32", 128), ("bf16", 128)])
+def test_trees_of_96_and_128_nodes(dtype, nodes):
+    """The paper's larger candidate trees (Sec. III-A.3): two ancestor words per node, two 64-node query tiles per
+    (head, sequence); tensor-core attention (bf16, head_dim 64) and the plain one (fp32); prefill in 96/128-token
+    chunks; planted continuation so that deep paths are accepted."""
+    wl = W.toy_workload(dtype=dtype, d_model=128, n_heads=2, d_ffn=256, vocab=203, n_draft_heads=4, tree_nodes=nodes,
+                        tree_caps=(10, 5, 3, 2), tau=3, temperature=1.0, batch=2, phoneme_len=(20, 60), prompt_len=150,
+                        index=18)
+    w, model, tpl, g, table = _setup(wl, 4, range(2))
+    assert [int((tpl.depth == d).sum()) for d in range(5)] == {96: [1, 9, 30, 42, 14], 128: [1, 10, 35, 53, 29]}[nodes]
+    states, _ = _prefill_both(wl, g, table, model, range(2), oracle_chunk=53)
+    so, sg = _sampling(wl)
+    so1 = O.Sampling(tau=1, temperature=1.0, top_p=1.0, seed=so.seed, accept_rule=0)
+    planted = {}
+    for b in range(2):
+        ph, pr = W.prefix_for(wl, b)
+        planted[b] = O.ar_decode(model, O.prefill(model, ph, pr, seq=b), so1, 24)
+    rep = lockstep(g, table, model, states, tpl, so, sg, 4, dtype, oracle_mode="memo", check_attn=True, planted=planted)
+    assert rep.iterations == 4 and max(rep.accept_lens) == 5
+    g.check()
+
+
 def test_six_draft_heads_accept_up_to_seven_tokens():
     """The paper's six-head ablation (Sec. III-A.3): depth-6 tree, planted continuation, paths of 7 tokens."""
     from workloads.trees import _from_rank_paths

@@ -127,14 +127,17 @@ def depths_of(parent: np.ndarray) -> np.ndarray:
 
 
 def ancestor_masks(parent: np.ndarray) -> np.ndarray:
-    """uint64 word per node with the bits of the node itself and all its ancestors."""
+    """Per node the bits of the node itself and all its ancestors: uint64 [n_nodes] for up to 64 nodes,
+    uint64 [n_nodes][2] (bits 0..63, 64..127) for up to 128."""
     n_nodes = len(parent)
-    if n_nodes > 64:
-        raise ValueError("one 64-bit word holds at most 64 nodes")
+    if n_nodes > 128:
+        raise ValueError("two 64-bit words hold at most 128 nodes")
     m = [0] * n_nodes
     for n in range(n_nodes):
         m[n] = (1 << n) | (m[int(parent[n])] if n > 0 else 0)
-    return np.array(m, dtype=np.uint64)
+    if n_nodes <= 64:
+        return np.array(m, dtype=np.uint64)
+    return np.array([[x & (2**64 - 1), x >> 64] for x in m], dtype=np.uint64)
 
 
 def validate_template(t: TreeTemplate, caps: Sequence[int] | None = None) -> None:
