@@ -29,6 +29,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 WORKLOAD = "C2"
+TREE_NODES = 0          # 0: the workload's own tree; --tree-nodes 96 / 128: the paper's larger candidate trees
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the 49 projection launches of one C2 step, from the
@@ -105,6 +106,9 @@ class ClockSampler:
 def _setup_inputs(rank: int):
     import workloads as W
     wl = W.workload(WORKLOAD)
+    if TREE_NODES:
+        from dataclasses import replace
+        wl = replace(wl, tree_nodes=TREE_NODES)
     weights = W.make_weights(wl.shape, wl.seed())
     tpl = W.static_template(wl.tree_nodes, wl.tree_caps)
     # every replica decodes its own sequence: item index = rank
@@ -161,7 +165,7 @@ def run_reference(args):
 
 def workload_config(extra=None):
     """The `config` object both arms print."""
-    c = {"workload": f"{WORKLOAD}: 12L d1024 16H FFN4096 vocab1025 bf16, batch 1 per GPU, 64-node tree "
+    c = {"workload": f"{WORKLOAD}: 12L d1024 16H FFN4096 vocab1025 bf16, batch 1 per GPU, {TREE_NODES or 64}-node tree "
                      f"(top-10/5/3/2), tau 3, T 1.0, 325-token prefix, random-init weights",
          "step": "one draft+verify+accept/commit iteration"}
     if extra:
@@ -516,11 +520,15 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="C5 only: smaller batch (for profiler captures)")
     ap.add_argument("--prefill-rows", type=int, default=64,
                     help="C3, C4: prefix chunks of 64 tokens scored per prefill pass (0: one per sequence)")
+    ap.add_argument("--tree-nodes", type=int, default=0, choices=[0, 64, 96, 128],
+                    help="C2 only: candidate-tree size (default: the workload's 64 nodes)")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
+    global TREE_NODES
+    TREE_NODES = 0 if args.tree_nodes == 64 else args.tree_nodes
     if args.steps is None:
         args.steps = 20 if args.impl == "reference" else 400
     if args.impl == "reference":
