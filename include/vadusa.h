@@ -71,7 +71,7 @@ typedef struct {
   uint32_t struct_size;        /* sizeof(vadusa_config) */
   uint32_t abi_version;        /* VADUSA_ABI_VERSION */
   int32_t n_layers, d_model, n_heads, d_ffn;
-  int32_t vocab;               /* speech-token ids, the last one (vocab-1) is EOS */
+  int32_t vocab;               /* speech-token ids, the last one (vocab-1) is EOS; 2..24576 */
   int32_t n_phonemes;
   int32_t max_pos;             /* rows of the position table */
   int32_t dtype;               /* 0 fp32, 1 bf16 */

@@ -657,6 +657,9 @@ vadusa_status set_kernel_attributes(vadusa_ctx* ctx) {
   CU(cudaFuncSetAttribute(tree_attention_simt_kernel<bf16, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(64)));
   CU(cudaFuncSetAttribute(tree_attention_simt_kernel<bf16, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(32)));
   CU(cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmemBytes));
+  // the accept kernel keeps one row of keys and one of probabilities in shared memory
+  if (2 * vpad(&ctx->cfg) * (int)sizeof(float) > 48 * 1024)
+    CU(cudaFuncSetAttribute(accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * vpad(&ctx->cfg) * (int)sizeof(float)));
   // ask for the largest shared-memory carve-out so that several CTAs fit on an SM
   CU(cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
   return VADUSA_OK;

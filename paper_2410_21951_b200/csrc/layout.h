@@ -30,7 +30,7 @@ inline const char* check_config(const vadusa_config* c) {
     if (dh != 32 && dh != 64) return "head_dim must be 32 or 64";
   }
   if (c->d_ffn < 16 || c->d_ffn % 16) return "d_ffn must be a positive multiple of 16";
-  if (c->vocab < 2) return "vocab must be at least 2";
+  if (c->vocab < 2 || c->vocab > 24576) return "vocab must be in 2..24576 (two rows of it live in shared memory)";
   if (c->n_phonemes < 0) return "n_phonemes must be >= 0";
   if (c->max_pos < 1) return "max_pos must be positive";
   if (c->n_draft_heads < 1 || c->n_draft_heads > VADUSA_MAX_DEPTH) return "n_draft_heads out of range";

@@ -234,6 +234,19 @@ def test_trees_of_96_and_128_nodes(dtype, nodes):
     g.check()
 
 
+def test_large_vocabulary_of_16001_tokens():
+    """The paper's largest codebook (wav2vec 2.0 tokens, top-16000, Sec. III-D): the vocabulary heads, the draft
+    top-k and the acceptance test at a 16-times larger vocabulary, nucleus on."""
+    wl = W.toy_workload(dtype="bf16", d_model=128, n_heads=2, d_ffn=256, vocab=16001, n_draft_heads=3, tree_nodes=16,
+                        tree_caps=(6, 3, 2), tau=4, temperature=0.9, batch=2, phoneme_len=(9, 9), prompt_len=60, index=19)
+    w, model, tpl, g, table = _setup(wl, 4, range(2))
+    states, _ = _prefill_both(wl, g, table, model, range(2))
+    so, sg = _sampling(wl, top_p=0.95)
+    rep = lockstep(g, table, model, states, tpl, so, sg, 4, "bf16", oracle_mode="memo")
+    assert rep.iterations == 4 and rep.root_checked + rep.draft_sets_checked > 0
+    g.check()
+
+
 def test_six_draft_heads_accept_up_to_seven_tokens():
     """The paper's six-head ablation (Sec. III-A.3): depth-6 tree, planted continuation, paths of 7 tokens."""
     from workloads.trees import _from_rank_paths
