@@ -151,7 +151,9 @@ vadusa_status vadusa_weight_info(const vadusa_config *cfg, int32_t index, vadusa
 
 /* ---- life cycle ------------------------------------------------------------------ */
 /* Validates the configuration, records the pointers, clears the state area of the
- * workspace.  Synchronises the stream once. */
+ * workspace.  Synchronises the stream once.  Makes cfg->device the calling thread's current
+ * CUDA device; every later call on the context must be made with that device current.  A
+ * context is not thread-safe: one thread at a time. */
 vadusa_status vadusa_init(const vadusa_weights *weights, const vadusa_config *cfg, vadusa_ctx **h_out);
 vadusa_status vadusa_destroy(vadusa_ctx *ctx);
 const char *vadusa_last_error(const vadusa_ctx *ctx);   /* NUL-terminated, owned by the context */

@@ -255,12 +255,13 @@ vadusa_status launch_gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void
                              int batches, long long x_z, long long w_z, int ksplit, const Epi& epi,
                              const LnFuse* ln = nullptr) {
   using Cfg = GemmTcCfg<TN>;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static unsigned long long attr_done = 0ull;              // per device: function attributes belong to a device's context
+  const unsigned long long dev_bit = 1ull << (ctx->cfg.device & 63);
+  if (!(attr_done & dev_bit)) {
     CU(cudaFuncSetAttribute(gemm_tc_kernel<TN, Epi, LN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemMax));
     CU(cudaFuncSetAttribute(gemm_tc_kernel<TN, Epi, LN>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
     CU(cudaFuncSetAttribute(gemm_tc_kernel<TN, Epi, LN>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
-    attr_done = true;
+    attr_done |= dev_bit;
   }
   const int chunks = K / kGemmBK / ksplit;
   const int smem = Cfg::smem_for(chunks, ksplit);
