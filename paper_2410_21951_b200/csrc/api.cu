@@ -310,13 +310,13 @@ static bool residual_leaves_stats(int M, int d, int K) {
 // cluster are 128 columns.  Returns false (nothing launched) when the shape does not qualify.
 template <typename Epi>
 bool gemm_tc_ln(vadusa_ctx* ctx, int cls, const float* x, const float* g, const float* b, const void* W, int w_rows,
-                int M, int N, int K, const Epi& epi, vadusa_status* st) {
+                int M, int N, int K, const Epi& epi, vadusa_status* st, bf16* y = nullptr) {
   if (M > 64 || K % 128 || K / 128 > 8) return false;
   const int tn = M <= 16 ? 16 : M <= 32 ? 32 : 64;
   const int tiles = (N + kGemmRowsW - 1) / kGemmRowsW;
   const int ksplit = K / 128;                            // one CTA of the cluster per group of 128 columns
   if (ksplit < 2 || ksplit > tn || (long long)tiles * ksplit * tn * kGemmRowsW * 4 > kGemmPartBytes) return false;
-  const LnFuse ln{x, g, b, wsptr<float2>(ctx, ctx->ws.ln_stats), K, ctx->cfg.ln_eps};
+  const LnFuse ln{x, g, b, wsptr<float2>(ctx, ctx->ws.ln_stats), y, K, ctx->cfg.ln_eps};
   switch (tn) {
     case 16: *st = launch_gemm_tc<16, Epi, true>(ctx, cls, nullptr, W, w_rows, M, N, K, 1, 0, 0, ksplit, epi, &ln); break;
     case 32: *st = launch_gemm_tc<32, Epi, true>(ctx, cls, nullptr, W, w_rows, M, N, K, 1, 0, 0, ksplit, epi, &ln); break;
@@ -359,8 +359,8 @@ vadusa_status product(vadusa_ctx* ctx, int cls, const T* X, const T* W, int w_ro
 // LayerNorm followed by a product, in one kernel where the shape allows (bf16 models, few tokens).
 template <typename T, typename Epi>
 bool ln_product(vadusa_ctx* ctx, int cls, const float* x, const float* g, const float* b, const T* W, int w_rows, int M,
-                int N, int K, const Epi& epi, vadusa_status* st) {
-  if constexpr (std::is_same<T, bf16>::value) return gemm_tc_ln(ctx, cls, x, g, b, W, w_rows, M, N, K, epi, st);
+                int N, int K, const Epi& epi, vadusa_status* st, T* y = nullptr) {
+  if constexpr (std::is_same<T, bf16>::value) return gemm_tc_ln(ctx, cls, x, g, b, W, w_rows, M, N, K, epi, st, y);
   return false;
 }
 
@@ -463,28 +463,29 @@ vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* overri
   int32_t* ctx_len = wsptr<int32_t>(ctx, ctx->ws.ctx_len);
   int32_t* nvalid = wsptr<int32_t>(ctx, ctx->ws.nvalid);
 
+  // LayerNorm statistics for the products that normalise their own operand (bf16 models, few tokens): left by
+  // the embedding kernel and by the residual products
+  const bool tc = std::is_same<T, bf16>::value;
+  const bool embed_stats = tc && M <= 64 && d % 128 == 0 && d / 128 <= 8;
+  const bool stats_out = tc && residual_leaves_stats(M, d, d), stats_ffn = tc && residual_leaves_stats(M, d, f);
+  float2* stats = wsptr<float2>(ctx, ctx->ws.ln_stats);
   PROF(ctx, K_EMBED);
   tree_embed_kernel<T><<<M, 128, 0, ctx->stream>>>(
       tv, override_tokens, wsptr<int32_t>(ctx, ctx->ws.root), wsptr<int32_t>(ctx, ctx->ws.topk), c.n_draft_heads,
       c.draft_topk, ctx_len, nvalid, as<T>(ctx->emb_audio), as<T>(ctx->emb_phon), as<T>(ctx->pos),
       c.vocab, c.n_phonemes, c.max_pos, d, wsptr<int32_t>(ctx, ctx->ws.tokens), x, ctx->block_table, g,
-      wsptr<long long>(ctx, ctx->ws.kv_row), err_word(ctx));
+      wsptr<long long>(ctx, ctx->ws.kv_row), embed_stats ? stats : nullptr, err_word(ctx));
   LAUNCH_CHECK();
   if (B > 1) {
     PROF(ctx, K_MISC);
     seq_order_kernel<<<1, 256, 0, ctx->stream>>>(ctx_len, nvalid, B, wsptr<int32_t>(ctx, ctx->ws.seq_order));
     LAUNCH_CHECK();
   }
-  // residual products that can leave LayerNorm statistics for the product after them (bf16 models, few tokens)
-  const bool tc = std::is_same<T, bf16>::value;
-  const bool stats_out = tc && residual_leaves_stats(M, d, d), stats_ffn = tc && residual_leaves_stats(M, d, f);
-  float2* stats = wsptr<float2>(ctx, ctx->ws.ln_stats);
-  bool have_stats = false;
+  bool have_stats = embed_stats;
   for (int l = 0; l < c.n_layers; ++l) {
     const LayerW& w = ctx->layers[l];
     T* pool = reinterpret_cast<T*>(c.kv_pool) + (long long)l * g.layer_stride;
     vadusa_status s = VADUSA_OK;
-    // (layer 0 reads the embedding kernel's x, which comes without statistics)
     EpiQKV<T> eq{w.bqkv, q, pool, wsptr<long long>(ctx, ctx->ws.kv_row), (long long)c.n_heads * kKvBlock * g.head_dim,
                  kKvBlock * g.head_dim, g.head_dim, d};
     if (!(have_stats && ln_product<T>(ctx, K_GEMM_QKV, x, w.ln1_g, w.ln1_b, as<T>(w.wqkv), 3 * d, M, 3 * d, d, eq, &s))) {
@@ -523,8 +524,13 @@ vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* overri
     have_stats = stats_ffn;
     if (s) return s;
   }
-  if (vadusa_status s = layernorm<T>(ctx, x, ctx->lnf_g, ctx->lnf_b, hfinal, M)) return s;
   EpiLogits el{logits, vp, 0};
+  vadusa_status s = VADUSA_OK;
+  // the final LayerNorm folds into the vocabulary head, which also stores the normalised rows (the draft heads
+  // and the carried state read them)
+  if (have_stats && ln_product<T>(ctx, K_GEMM_LM, x, ctx->lnf_g, ctx->lnf_b, as<T>(ctx->lm), vp, M, vp, d, el, &s, hfinal))
+    return s;
+  if ((s = layernorm<T>(ctx, x, ctx->lnf_g, ctx->lnf_b, hfinal, M))) return s;
   return product<T>(ctx, K_GEMM_LM, hfinal, as<T>(ctx->lm), vp, M, vp, d, 1, 0, 0, el);
 }
 
@@ -989,14 +995,14 @@ vadusa_status vadusa_draft(vadusa_ctx* ctx, const vadusa_sampling* sampling, int
             wsptr<int32_t>(ctx, ctx->ws.ctx_len), wsptr<int32_t>(ctx, ctx->ws.nvalid), as<bf16>(ctx->emb_audio),
             as<bf16>(ctx->emb_phon), as<bf16>(ctx->pos), c.vocab, c.n_phonemes, c.max_pos, c.d_model,
             wsptr<int32_t>(ctx, ctx->ws.tokens), wsptr<float>(ctx, ctx->ws.x), ctx->block_table, geom_of(ctx),
-            (long long*)nullptr, err_word(ctx));
+            (long long*)nullptr, (float2*)nullptr, err_word(ctx));
       else
         tree_embed_kernel<float><<<M, 128, 0, ctx->stream>>>(
             tv, nullptr, wsptr<int32_t>(ctx, ctx->ws.root), wsptr<int32_t>(ctx, ctx->ws.topk), c.n_draft_heads, c.draft_topk,
             wsptr<int32_t>(ctx, ctx->ws.ctx_len), wsptr<int32_t>(ctx, ctx->ws.nvalid), as<float>(ctx->emb_audio),
             as<float>(ctx->emb_phon), as<float>(ctx->pos), c.vocab, c.n_phonemes, c.max_pos, c.d_model,
             wsptr<int32_t>(ctx, ctx->ws.tokens), wsptr<float>(ctx, ctx->ws.x), ctx->block_table, geom_of(ctx),
-            (long long*)nullptr, err_word(ctx));
+            (long long*)nullptr, (float2*)nullptr, err_word(ctx));
       LAUNCH_CHECK();
       CU(cudaMemcpyAsync(tree_tokens, ctx->wsp + ctx->ws.tokens, (size_t)M * 4, cudaMemcpyDeviceToDevice, ctx->stream));
     }

@@ -17,7 +17,7 @@ __global__ void tree_embed_kernel(TreeView tree, const int32_t* __restrict__ ove
                                   const T* __restrict__ pos_table, int vocab, int n_phonemes, int max_pos, int d,
                                   int32_t* __restrict__ tokens_out, float* __restrict__ x,
                                   const int32_t* __restrict__ block_table, KvGeom geom, long long* __restrict__ kv_row,
-                                  uint32_t* err) {
+                                  float2* __restrict__ stats /*[rows][d/128] or null*/, uint32_t* err) {
   const int m = blockIdx.x;
   const int b = m / tree.n_nodes, n = m % tree.n_nodes;
   const int to = tree.off(b);
@@ -47,6 +47,24 @@ __global__ void tree_embed_kernel(TreeView tree, const int32_t* __restrict__ ove
     if (kv_row) kv_row[m] = row;
   }
   const T* p = pos_table + (long long)pos * d;
+  if (stats) {
+    // d is a multiple of 128: warp w takes the groups of 128 features w, w + 4, ... (lane l: features 4l .. 4l+3 of
+    // the group) and leaves each group's mean and sum of squared deviations for the LayerNorm folded into the
+    // first product
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nt = d >> 7;
+    for (int gi = warp; gi < nt; gi += (int)(blockDim.x >> 5)) {
+      const int c0 = 128 * gi + 4 * lane;
+      float4 v;
+      v.x = to_f<T>(e[c0]) + to_f<T>(p[c0]);         v.y = to_f<T>(e[c0 + 1]) + to_f<T>(p[c0 + 1]);
+      v.z = to_f<T>(e[c0 + 2]) + to_f<T>(p[c0 + 2]); v.w = to_f<T>(e[c0 + 3]) + to_f<T>(p[c0 + 3]);
+      *reinterpret_cast<float4*>(x + (long long)m * d + c0) = v;
+      const float mu = warp_sum((v.x + v.y) + (v.z + v.w)) * (1.0f / 128.0f);
+      const float d0 = v.x - mu, d1 = v.y - mu, d2 = v.z - mu, d3 = v.w - mu;
+      const float q = warp_sum((d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3));
+      if (lane == 0) stats[(long long)m * nt + gi] = make_float2(mu, q);
+    }
+    return;
+  }
   for (int i = threadIdx.x; i < d; i += blockDim.x) x[(long long)m * d + i] = to_f<T>(e[i]) + to_f<T>(p[i]);
 }
 

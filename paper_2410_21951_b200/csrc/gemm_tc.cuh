@@ -54,6 +54,7 @@ struct LnFuse {
   const float* g;        // [K] gain
   const float* b;        // [K] shift
   const float2* stats;   // [M][K/128] (mean, sum of squared deviations) of each group of 128 features
+  bf16* y;               // if not null: the CTAs of feature tile 0 also store the normalised rows here ([M][ld] bf16)
   int ld;
   float eps;
 };
@@ -87,19 +88,20 @@ __device__ __forceinline__ void ln_operand(const LnFuse& ln, int M, int K, int k
   }
   // row statistics from the groups': lane = 8 * (row in a group of four rows) + feature group
   float mean_g[RPW / 4], rstd_g[RPW / 4];
+  const float inv_nt = 1.0f / (float)nt, inv_k = 1.0f / (float)K;     // (exact for the usual powers of two)
   {
 #pragma unroll
     for (int it = 0; it < RPW / 4; ++it) {
       float m = st[it].x;
 #pragma unroll
       for (int o = 4; o > 0; o >>= 1) m += __shfl_xor_sync(0xffffffffu, m, o);
-      m /= (float)nt;
+      m *= inv_nt;
       const float dv = st[it].x - m;
       float m2 = t < nt ? st[it].y + 128.0f * dv * dv : 0.f;
 #pragma unroll
       for (int o = 4; o > 0; o >>= 1) m2 += __shfl_xor_sync(0xffffffffu, m2, o);
       mean_g[it] = m;
-      rstd_g[it] = 1.0f / sqrtf(m2 / (float)K + ln.eps);
+      rstd_g[it] = rsqrtf(fmaf(m2, inv_k, ln.eps));
     }
   }
   // normalise into the swizzled K-major operand tiles: column 4*lane is in tile lane/16, 16-byte unit
@@ -119,6 +121,8 @@ __device__ __forceinline__ void ln_operand(const LnFuse& ln, int M, int K, int k
     }
     const uint32_t unit = (uint32_t)((lane & 15) >> 1) ^ (uint32_t)(row & 7);
     asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(tile + (uint32_t)row * 128u + (unit << 4)), "r"(lo), "r"(hi));
+    if (ln.y != nullptr && blockIdx.x == 0 && row < M)
+      *reinterpret_cast<uint2*>(ln.y + (long long)row * ln.ld + k0 + 4 * lane) = make_uint2(lo, hi);
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tensor-core reads
 }
