@@ -247,6 +247,44 @@ def test_large_vocabulary_of_16001_tokens():
     g.check()
 
 
+def test_degenerate_trees_root_only_and_deepest_chain():
+    """A one-node tree is plain decoding (one token per iteration); a chain of 16 nodes over 15 draft heads is the
+    deepest path the interface allows: planted, all 16 tokens are committed in one iteration."""
+    import torch
+    import paper_2410_21951_b200 as P
+    # root only
+    wl = W.toy_workload(dtype="fp32", d_model=64, n_heads=2, d_ffn=128, vocab=61, n_draft_heads=1, tree_nodes=1,
+                        tree_caps=(1,), batch=2, phoneme_len=(5, 9), prompt_len=30, index=20)
+    w, model, tpl, g, table = _setup(wl, 12, range(2))
+    assert tpl.n_nodes == 1
+    states, _ = _prefill_both(wl, g, table, model, range(2))
+    so, sg = _sampling(wl, seed=9, tau=2, temperature=0.7)
+    rep = lockstep(g, table, model, states, tpl, so, sg, 10, "fp32", oracle_mode="memo")
+    assert rep.accept_lens == [1] * 20
+    so1 = O.Sampling(tau=1, temperature=0.7, top_p=1.0, seed=9)
+    for b in range(2):
+        ph, pr = W.prefix_for(wl, b)
+        assert states[b].tokens == O.ar_decode(model, O.prefill(model, ph, pr, seq=b), so1, 10)
+    g.check()
+    g.close()
+    # chain of 16 over 15 heads
+    wl = W.toy_workload(dtype="bf16", d_model=64, n_heads=2, d_ffn=128, vocab=61, n_draft_heads=15, tree_nodes=16,
+                        tree_caps=tuple([1] * 15), batch=1, phoneme_len=(7, 7), prompt_len=40, index=21)
+    tpl = W.chain_template(16)
+    w = W.make_weights(wl.shape, wl.seed())
+    model = O.Model.from_shape(wl.shape, w)
+    need = [sum(len(x) for x in W.prefix_for(wl, 0)) + 3 * 16 + 16]
+    g, table = make_gpu(wl.shape, w, 1, 16, need, 13, draft_topk=4)
+    g.set_tree(tpl.parent, tpl.rank)
+    states, _ = _prefill_both(wl, g, table, model, range(1))
+    so, sg = _sampling(wl, seed=4, tau=1, temperature=0.0)
+    ph, pr = W.prefix_for(wl, 0)
+    planted = {0: O.ar_decode(model, O.prefill(model, ph, pr, seq=0), so, 40)}
+    rep = lockstep(g, table, model, states, tpl, so, sg, 2, "bf16", oracle_mode="memo", planted=planted)
+    assert max(rep.accept_lens) == 16
+    g.check()
+
+
 def test_six_draft_heads_accept_up_to_seven_tokens():
     """The paper's six-head ablation (Sec. III-A.3): depth-6 tree, planted continuation, paths of 7 tokens."""
     from workloads.trees import _from_rank_paths
