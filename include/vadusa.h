@@ -249,6 +249,18 @@ vadusa_status vadusa_get_lengths(vadusa_ctx *ctx, int32_t *h_ctx_len);  /* synch
 vadusa_status vadusa_check(vadusa_ctx *ctx);                            /* synchronises; device error word */
 int64_t vadusa_kernel_launches(const vadusa_ctx *ctx);                  /* total kernels enqueued so far */
 
+/* ---- sampler hook (paper Sec. II-C, last paragraph) ----------------------------------------
+ * The paper notes that improved sampling strategies (e.g. avoiding repetitions) are used by taking
+ * their outcomes as the predictions of the original head, with the tau draws made by the same
+ * strategy.  The strategies this hook serves are those that reshape the base head's distribution
+ * per sequence: bias is fp32 [batch][ld] (ld >= vocab) in device memory, owned by the caller, and
+ * is added (one fp32 addition, before temperature, nucleus and noise) to every base-head logits
+ * row of the sequence wherever it is sampled: the root, the tau draws of Algorithm 1 and the next
+ * root.  -inf bans a token.  The draft heads and the returned logits are not changed.  The caller
+ * may rewrite the table between iterations (stream-ordered); NULL switches the hook off.  The
+ * pointer is read by the kernels of later calls; it must stay valid until replaced. */
+vadusa_status vadusa_set_logit_bias(vadusa_ctx *ctx, const float *bias, int32_t ld);
+
 /* ---- sparse-tree construction (paper Sec. II-D) --------------------------------------
  * The paper grows its sparse candidate tree greedily so as to maximise the expected accepted
  * length within a fixed number of nodes, from acceptance probabilities measured with the

@@ -35,6 +35,7 @@ class Sampling:
     eos_masked: bool = True
     accept_rule: int = 0          # 0: Alg. 1 (tau noisy draws); 1: plain top-tau of the logits
     seed: int = 0
+    bias: Optional[np.ndarray] = None   # [sequences][vocab] fp32 added to the base head's logits wherever it samples
 
 
 @dataclass
@@ -81,6 +82,10 @@ def prefill_blocked(model: Model, phon: Sequence[int], prompt: Sequence[int], se
 
 def _keys_and_nucleus(model: Model, logits, sp: Sampling, seq: int, pos: int, noise: bool = True):
     l32 = masked_logits32(logits, model.eos_id, sp.eos_masked)
+    if sp.bias is not None:
+        # a reshaped base-head distribution (Sec. II-C, last paragraph: other sampling strategies enter as the
+        # original head's predictions): one fp32 addition before temperature, nucleus and noise
+        l32 = (l32 + np.asarray(sp.bias[seq], dtype=np.float32)).astype(np.float32)
     keys = decision_keys(l32, sp.temperature, sp.seed, seq, pos, noise=noise)
     nuc = nucleus_sorted(l32, sp.temperature, sp.top_p)
     return l32, keys, nuc

@@ -69,7 +69,7 @@ EXPORTS = ["vadusa_workspace_bytes", "vadusa_weights_bytes", "vadusa_kv_pool_byt
            "vadusa_begin", "vadusa_prefill", "vadusa_load_state", "vadusa_draft", "vadusa_verify_step",
            "vadusa_accept_and_commit", "vadusa_generate", "vadusa_generate_host", "vadusa_get_lengths",
            "vadusa_check", "vadusa_kernel_launches", "vadusa_profile_begin", "vadusa_profile_end",
-           "vadusa_accept_stats", "vadusa_build_sparse_tree",
+           "vadusa_accept_stats", "vadusa_build_sparse_tree", "vadusa_set_logit_bias",
            "vadusa_draft_topk_static", "vadusa_static_scratch_bytes", "vadusa_static_last_error"]
 
 _lib = None
@@ -105,6 +105,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "vadusa_static_scratch_bytes": (I64, []),
         "vadusa_static_last_error": (C.c_char_p, []),
         "vadusa_accept_stats": (I32, [P, P, P, I32]),
+        "vadusa_set_logit_bias": (I32, [P, P, I32]),
         "vadusa_build_sparse_tree": (I32, [P, I32, I32, I32, P, P, P]),
         "vadusa_profile_begin": (I32, [P]),
         "vadusa_profile_end": (I32, [P, C.POINTER(KernelTime), I32, C.POINTER(I32)]),
@@ -369,6 +370,11 @@ class Vadusa:
 
     def check(self):
         self._ck(self.L.vadusa_check(self.ctx))
+
+    def set_logit_bias(self, bias=None):
+        """bias: fp32 device tensor [batch][>= vocab] added to the base head's logits when sampling, or None."""
+        self._keep["logit_bias"] = bias
+        self._ck(self.L.vadusa_set_logit_bias(self.ctx, self._p(bias), 0 if bias is None else bias.shape[1]))
 
     def accept_stats(self, reset: bool = False):
         """(tested, accepted) int64 [MAX_DEPTH][MAX_DRAFT_TOPK]: acceptance tests by (draft head, rank)."""

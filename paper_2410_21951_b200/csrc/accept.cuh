@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(256) accept_kernel(
       __syncthreads();
       const int nchild = s_nchild;
       if (nchild == 0) continue;
-      const float* row = logits + ((long long)b * N + p) * ld;
+      const BaseRow row = base_row(logits + ((long long)b * N + p) * ld, sp, b);
       const uint64_t rs = noise_row_state(sp.seed, b, S + d + 1);
       const bool noise = sp.accept_rule == 0;
       for (int j = tid; j < vocab; j += blockDim.x) keys[j] = key_of(row[j], j, rs, sp, noise);
@@ -160,7 +160,7 @@ __global__ void __launch_bounds__(256) accept_kernel(
   }
   __syncthreads();
   const int best = s_best, len = s_len;
-  const int nroot = sample_row(logits + ((long long)b * N + best) * ld, vocab, b, S + len, sp, bscratch, fscratch);
+  const int nroot = sample_row(base_row(logits + ((long long)b * N + best) * ld, sp, b), vocab, b, S + len, sp, bscratch, fscratch);
 
   if (tid < kMaxPath) {
     const bool in = tid < len;

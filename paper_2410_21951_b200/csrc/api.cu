@@ -39,6 +39,8 @@ struct vadusa_ctx {
   char* wsp = nullptr;
   cudaStream_t stream = nullptr;
   int batch = 0;
+  const float* logit_bias = nullptr;   // caller's [batch][logit_bias_ld] fp32 added to the base head's logits (sampler hook)
+  int logit_bias_ld = 0;
   int n_nodes = 0;            // current tree size (0: none set)
   int tree_per_seq = 0;
   int max_rank_used = 0;
@@ -204,6 +206,8 @@ vadusa_status sampling_dev(vadusa_ctx* ctx, const vadusa_sampling* s, SamplingDe
   o->accept_rule = s->accept_rule;
   o->eos_id = ctx->cfg.vocab - 1;
   o->seed = s->seed;
+  o->bias = ctx->logit_bias;
+  o->bias_ld = ctx->logit_bias_ld;
   return VADUSA_OK;
 }
 
@@ -1157,6 +1161,15 @@ vadusa_status vadusa_get_lengths(vadusa_ctx* ctx, int32_t* h_ctx_len) {
 vadusa_status vadusa_check(vadusa_ctx* ctx) {
   if (!ctx || !ctx->wsp) return VADUSA_EINVAL;
   return device_errors(ctx);
+}
+
+vadusa_status vadusa_set_logit_bias(vadusa_ctx* ctx, const float* bias, int32_t ld) {
+  if (!ctx) return VADUSA_EINVAL;
+  if (!ctx->wsp) return fail(ctx, VADUSA_ESTATE, "context is not initialised");
+  if (bias && ld < ctx->cfg.vocab) return fail(ctx, VADUSA_EINVAL, "bias rows must hold at least vocab entries");
+  ctx->logit_bias = bias;
+  ctx->logit_bias_ld = bias ? ld : 0;
+  return VADUSA_OK;
 }
 
 vadusa_status vadusa_accept_stats(vadusa_ctx* ctx, int64_t* h_tested, int64_t* h_accepted, int32_t reset) {

@@ -29,8 +29,20 @@ struct SamplingDev {
   int tau;
   float temperature, inv_temperature, top_p;
   int eos_masked, accept_rule, eos_id;
+  int bias_ld;                    // row length of bias
   unsigned long long seed;
+  const float* bias;              // [batch][bias_ld] added to the base head's logits before anything else, or null
 };
+
+// A logits row of the base head as the sampler sees it: logit + bias (one fp32 addition) when a bias is set.
+struct BaseRow {
+  const float* row;
+  const float* bias;
+  __device__ __forceinline__ float operator[](int j) const { return bias ? __fadd_rn(row[j], bias[j]) : row[j]; }
+};
+__device__ __forceinline__ BaseRow base_row(const float* row, const SamplingDev& sp, int seq) {
+  return BaseRow{row, sp.bias ? sp.bias + (long long)seq * sp.bias_ld : nullptr};
+}
 
 // fp32 key of a token: logit * (1/T) + g, formed with separately rounded operations.
 __device__ __forceinline__ float key_of(float logit, int token, uint64_t row_state, const SamplingDev& sp, bool noise) {

@@ -62,7 +62,7 @@ __device__ __forceinline__ float block_max(float x, float* scratch) {
 // Softmax statistics of a logits row at the sampling temperature (EOS masked).
 struct RowStats { float maxl, z; };
 
-__device__ __forceinline__ RowStats row_stats(const float* __restrict__ row, int vocab, const SamplingDev& sp,
+__device__ __forceinline__ RowStats row_stats(const BaseRow row, int vocab, const SamplingDev& sp,
                                               float* scratch) {
   float mx = -INFINITY;
   for (int j = threadIdx.x; j < vocab; j += blockDim.x) mx = fmaxf(mx, masked_logit(row[j], j, sp));
@@ -76,7 +76,7 @@ __device__ __forceinline__ RowStats row_stats(const float* __restrict__ row, int
 
 // Nucleus membership of token c (top-p of softmax(logits/T)): the probability mass of the
 // tokens ahead of c (larger logit, or equal logit and lower id) is below top_p.
-__device__ __forceinline__ bool in_nucleus(const float* __restrict__ row, int vocab, int c, RowStats st,
+__device__ __forceinline__ bool in_nucleus(const BaseRow row, int vocab, int c, RowStats st,
                                            const SamplingDev& sp, float* scratch) {
   const float lc = masked_logit(row[c], c, sp);
   if (lc == -INFINITY) return false;
@@ -95,7 +95,7 @@ __device__ __forceinline__ bool nucleus_on(const SamplingDev& sp) {
 
 // The base head's single sample for absolute position pos: the first token, in key order,
 // that lies in the nucleus.  Same result in every thread.
-__device__ int sample_row(const float* __restrict__ row, int vocab, int seq, int pos, const SamplingDev& sp,
+__device__ int sample_row(const BaseRow row, int vocab, int seq, int pos, const SamplingDev& sp,
                           Best* bscratch, float* fscratch) {
   const uint64_t rs = noise_row_state(sp.seed, seq, pos);
   const bool nuc = nucleus_on(sp);
@@ -128,7 +128,7 @@ __global__ void __launch_bounds__(256) draft_select_kernel(
   const int b = blockIdx.y, head = blockIdx.x;
   if (nvalid[b] == 0) return;
   if (head == n_heads) {
-    const int r = sample_row(logits_star + (long long)b * ld, vocab, b, ctx_len[b], sp, bscratch, fscratch);
+    const int r = sample_row(base_row(logits_star + (long long)b * ld, sp, b), vocab, b, ctx_len[b], sp, bscratch, fscratch);
     if (threadIdx.x == 0) root[b] = r;
     return;
   }

@@ -247,6 +247,35 @@ def test_large_vocabulary_of_16001_tokens():
     g.check()
 
 
+def test_logit_bias_hook_follows_the_oracle():
+    """The sampler hook: a per-sequence bias on the base head's logits (some tokens banned) in the root sample, the
+    tau draws of the acceptance test and the next root; planted continuation decoded under the same bias."""
+    import torch
+    from dataclasses import replace
+    wl = W.toy_workload(dtype="fp32", d_model=64, n_heads=2, d_ffn=128, vocab=61, tree_nodes=12, tree_caps=(4, 3, 2),
+                        batch=2, phoneme_len=(9, 9), prompt_len=60, index=22)
+    w, model, tpl, g, table = _setup(wl, 8, range(2))
+    states, _ = _prefill_both(wl, g, table, model, range(2))
+    rng = np.random.Generator(np.random.Philox(key=[22, 1]))
+    bias = rng.normal(0, 1.5, size=(2, wl.shape.vocab)).astype(np.float32)
+    bias[0, [3, 11, 40]] = -np.inf
+    bias[1, [0, 59]] = -np.inf
+    so, sg = _sampling(wl, seed=6, tau=2, temperature=0.9, top_p=0.9)
+    so = replace(so, bias=bias)
+    g.set_logit_bias(torch.from_numpy(bias).to(g.dev))
+    so1 = O.Sampling(tau=1, temperature=0.9, top_p=0.9, seed=6, bias=bias)
+    planted = {}
+    for b in range(2):
+        ph, pr = W.prefix_for(wl, b)
+        planted[b] = O.ar_decode(model, O.prefill(model, ph, pr, seq=b), so1, 40)
+    rep = lockstep(g, table, model, states, tpl, so, sg, 8, "fp32", oracle_mode="memo", planted=planted)
+    assert rep.root_checked > 0 and rep.accept_checked > 0 and max(rep.accept_lens) == tpl.max_depth + 1
+    for b, banned in ((0, {3, 11, 40}), (1, {0, 59})):
+        assert not set(states[b].tokens) & banned
+    g.set_logit_bias(None)
+    g.check()
+
+
 def test_degenerate_trees_root_only_and_deepest_chain():
     """A one-node tree is plain decoding (one token per iteration); a chain of 16 nodes over 15 draft heads is the
     deepest path the interface allows: planted, all 16 tokens are committed in one iteration."""

@@ -84,6 +84,35 @@ def test_unmasked_eos_ends_the_sequence_exactly_where_plain_ar_ends_it():
     assert st.finished and st.tokens[-2:] == [3, m.eos_id]
 
 
+def test_logit_bias_reshapes_the_base_head_only_where_it_samples():
+    """Sec. II-C, last paragraph: another sampling strategy enters as the original head's predictions.  A zero
+    bias changes nothing; banned tokens (-inf) never appear; a dominant bias forces its token; tolerance 1
+    stays plain decoding under the same bias."""
+    wl, m, ph, pr = _setup()
+    V = wl.shape.vocab
+    tpl = W.static_template(10, (4, 3, 2))
+    base = O.Sampling(tau=2, temperature=1.0, seed=5)
+    st0 = O.prefill(m, ph, pr); O.vadusa_generate(m, st0, tpl, base, 16)
+    zero = O.Sampling(tau=2, temperature=1.0, seed=5, bias=np.zeros((1, V), dtype=np.float32))
+    st1 = O.prefill(m, ph, pr); O.vadusa_generate(m, st1, tpl, zero, 16)
+    assert st1.tokens == st0.tokens
+    banned = sorted(set(st0.tokens[:6]))
+    b = np.zeros((1, V), dtype=np.float32); b[0, banned] = -np.inf
+    ban = O.Sampling(tau=2, temperature=1.0, seed=5, bias=b)
+    st2 = O.prefill(m, ph, pr); O.vadusa_generate(m, st2, tpl, ban, 16)
+    assert not set(st2.tokens) & set(banned)
+    b = np.zeros((1, V), dtype=np.float32); b[0, 7] = 1e4
+    st3 = O.prefill(m, ph, pr); O.vadusa_generate(m, st3, tpl, O.Sampling(tau=1, temperature=0.9, seed=1, bias=b), 8)
+    assert set(st3.tokens) == {7}
+    g = np.random.Generator(np.random.Philox(key=[3, 3]))
+    b = g.normal(0, 2.0, size=(1, V)).astype(np.float32)
+    sp1 = O.Sampling(tau=1, temperature=1.0, seed=9, bias=b)
+    want = O.ar_decode(m, O.prefill(m, ph, pr), sp1, 20)
+    st4 = O.prefill(m, ph, pr); O.vadusa_generate(m, st4, tpl, sp1, 20)
+    assert st4.tokens[:20] == want
+    assert want != O.ar_decode(m, O.prefill(m, ph, pr), O.Sampling(tau=1, temperature=1.0, seed=9), 20)
+
+
 def test_planted_continuation_is_fully_accepted_and_cache_equals_ar_cache():
     """If the tree holds the true continuation, all of it is accepted (tau = 1),
     and afterwards the cache holds exactly what plain AR decoding stores."""
