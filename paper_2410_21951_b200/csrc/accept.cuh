@@ -47,6 +47,7 @@ __global__ void __launch_bounds__(256) accept_kernel(
   __shared__ int s_child[kMaxNodes], s_ok[kMaxNodes], s_nchild;
   __shared__ unsigned long long s_edges[2], s_acc[2];    // bits 0..63, 64..127
   __shared__ int s_path[kMaxPath], s_best, s_len, s_eos;
+  __shared__ int s_first[kMaxPath + 2];    // nodes are ordered by depth: first node of every depth, then nv
   __shared__ Best bscratch[32];
   __shared__ float fscratch[32];
 
@@ -75,15 +76,22 @@ __global__ void __launch_bounds__(256) accept_kernel(
     s_tok[tid] = in ? tokens[(long long)b * N + tid] : -1;
   }
   if (tid == 0) { s_edges[0] = 1ull; s_acc[0] = 1ull; s_edges[1] = 0ull; s_acc[1] = 0ull; }
+  if (tid < kMaxPath + 2) s_first[tid] = nv;
   __syncthreads();
-  int maxdepth = 0;
-  for (int n = 0; n < nv; ++n) maxdepth = max(maxdepth, s_depth[n]);
+  if (tid < nv && (tid == 0 || s_depth[tid] != s_depth[tid - 1])) s_first[min(s_depth[tid], kMaxPath)] = tid;
+  __syncthreads();
+  const int maxdepth = min(s_depth[nv - 1], kMaxPath - 1);
   const bool nuc = nucleus_on(sp);
   const int fb = forced_best ? forced_best[b] : -1;
 
   for (int d = 0; d < maxdepth && fb < 0; ++d) {
-    for (int p = 0; p < nv; ++p) {
-      if (s_depth[p] != d || !bit_at(s_acc[0], s_acc[1], p)) continue;  // uniform: shared memory
+    __syncthreads();                               // the accepted set of depth d is final
+    const unsigned long long a0 = s_acc[0], a1 = s_acc[1];
+    const int p_end = s_first[d + 1];
+    bool any = false;
+    for (int p = s_first[d]; p < p_end; ++p) {
+      if (!bit_at(a0, a1, p)) continue;            // uniform
+      any = true;
       __syncthreads();
       if (tid == 0) s_nchild = 0;
       __syncthreads();
@@ -140,14 +148,19 @@ __global__ void __launch_bounds__(256) accept_kernel(
       }
       __syncthreads();
     }
+    if (!any) break;                               // nothing accepted at this depth: nothing below it either
   }
   __syncthreads();
   if (tid == 0) {
     int best = 0;
     if (fb >= 0 && fb < nv) best = fb;
-    else
-      for (int n = 1; n < nv; ++n)
-        if (bit_at(s_acc[0], s_acc[1], n) && s_depth[n] > s_depth[best]) best = n;
+    else {
+      // deepest accepted node, the first (leftmost) of that depth
+      const unsigned long long a0 = s_acc[0], a1 = s_acc[1];
+      for (int d = maxdepth; d >= 1 && best == 0; --d)
+        for (int n = s_first[d]; n < s_first[d + 1]; ++n)
+          if (bit_at(a0, a1, n)) { best = n; break; }
+    }
     int len = min(s_depth[best] + 1, kMaxPath);
     int n = best;
     for (int j = len - 1; j >= 0; --j) { s_path[j] = n; n = s_parent[n]; }
