@@ -14,29 +14,35 @@ __device__ __forceinline__ Best better(Best a, Best b) {
   return precedes(a.v, a.i, b.v, b.i) ? a : b;
 }
 
+// fp32 -> uint32 that orders like the value (-0 counted as +0); every finite value and -inf map above 0.
+__device__ __forceinline__ uint32_t ordered_bits(float v) {
+  const uint32_t u = __float_as_uint(__fadd_rn(v, 0.0f));
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_bits(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
 // First element of the block in the order "larger value, then lower id" (i < 0: none).
-// scratch: 32 Best entries of shared memory.  Result is the same in every thread.
+// scratch: 32 Best entries of shared memory.  Result is the same in every thread.  The value travels as
+// its ordered bit pattern, so a warp needs two reduction instructions: the largest value, then the lowest
+// id among the lanes that hold it.
 __device__ __forceinline__ Best block_first(Best x, Best* scratch) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    Best y;
-    y.v = __shfl_xor_sync(0xffffffffu, x.v, o);
-    y.i = __shfl_xor_sync(0xffffffffu, x.i, o);
-    x = better(x, y);
-  }
+  const uint32_t none = 0xffffffffu;
+  uint32_t k = x.i < 0 ? 0u : ordered_bits(x.v);
+  uint32_t wk = __reduce_max_sync(0xffffffffu, k);
+  uint32_t wi = __reduce_min_sync(0xffffffffu, (x.i >= 0 && k == wk) ? (uint32_t)x.i : none);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = (blockDim.x + 31) >> 5;
   __syncthreads();
-  if (lane == 0) scratch[warp] = x;
+  if (lane == 0) scratch[warp] = Best{__uint_as_float(wk), (int)wi};
   __syncthreads();
-  Best r = (lane < nw) ? scratch[lane] : Best{0.f, -1};
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    Best y;
-    y.v = __shfl_xor_sync(0xffffffffu, r.v, o);
-    y.i = __shfl_xor_sync(0xffffffffu, r.i, o);
-    r = better(r, y);
-  }
-  return r;
+  const bool have = lane < nw && scratch[lane].i != (int)none;
+  k = have ? __float_as_uint(scratch[lane].v) : 0u;
+  const uint32_t id = have ? (uint32_t)scratch[lane].i : none;
+  wk = __reduce_max_sync(0xffffffffu, k);
+  wi = __reduce_min_sync(0xffffffffu, (have && k == wk) ? id : none);
+  if (wi == none) return Best{0.f, -1};
+  return Best{from_ordered_bits(wk), (int)wi};
 }
 
 __device__ __forceinline__ float block_sum(float x, float* scratch) {
