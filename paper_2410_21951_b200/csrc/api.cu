@@ -17,6 +17,7 @@
 #include "elementwise.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_tc2.cuh"
 #include "layout.h"
 #include "select.cuh"
 
@@ -292,6 +293,38 @@ vadusa_status launch_gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void
   return VADUSA_OK;
 }
 
+// Many-token product on CTA pairs (256 features x TN tokens per pair, no K split).
+template <int TN, typename Epi>
+vadusa_status launch_gemm_tc2(vadusa_ctx* ctx, int cls, const void* X, const void* W, int w_rows, int M, int N, int K,
+                              const Epi& epi) {
+  using Cfg = GemmTc2Cfg<TN>;
+  static unsigned long long attr_done = 0ull;              // per device, like launch_gemm_tc
+  const unsigned long long dev_bit = 1ull << (ctx->cfg.device & 63);
+  if (!(attr_done & dev_bit)) {
+    CU(cudaFuncSetAttribute(gemm_tc2_kernel<TN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmem));
+    CU(cudaFuncSetAttribute(gemm_tc2_kernel<TN, Epi>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+    attr_done |= dev_bit;
+  }
+  const CUtensorMap *mw, *mx;
+  if (vadusa_status s = tensor_map(ctx, W, w_rows, K, kGemmRowsW, 1, 0, &mw)) return s;
+  if (vadusa_status s = tensor_map(ctx, X, M, K, TN / 2, 1, 0, &mx)) return s;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(N / kGemmRowsW, (M + TN - 1) / TN, 1);           // N is a multiple of 256: whole pairs
+  lc.blockDim = dim3(128);
+  lc.dynamicSmemBytes = Cfg::kSmem;
+  lc.stream = ctx->stream;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // the kernel calls griddepcontrol.wait
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at; lc.numAttrs = 2;
+  PROF(ctx, cls);
+  CU(cudaLaunchKernelEx(&lc, gemm_tc2_kernel<TN, Epi>, *mw, *mx, M, N, K / kGemmBK, epi, err_word(ctx)));
+  LAUNCH_CHECK();
+  return VADUSA_OK;
+}
+
 // K split of a product with `tiles` output tiles of tn tokens: about one CTA per SM streams weights.
 static int gemm_ksplit(int tiles, int chunks, int tn) {
   int ksplit = 1;
@@ -336,6 +369,11 @@ vadusa_status gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void* W, in
   // token tile: as narrow as the token count allows for weight streaming; 256 for the tensor-bound shapes
   // when that still gives every SM a CTA pair, else 128
   const int ntiles_n = (N + kGemmRowsW - 1) / kGemmRowsW;
+  // tensor-bound shapes whose features come in whole pairs of tiles: CTA pairs, when they fill the SMs
+  if (M > 1024 && batches == 1 && N % (2 * kGemmRowsW) == 0) {
+    if (ntiles_n * ((M + 255) / 256) >= 200) return launch_gemm_tc2<256>(ctx, cls, X, W, w_rows, M, N, K, epi);
+    if (ntiles_n * ((M + 127) / 128) >= 200) return launch_gemm_tc2<128>(ctx, cls, X, W, w_rows, M, N, K, epi);
+  }
   int tn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 1024 ? 128 : 256;
   if (tn == 256 && ntiles_n * ((M + 255) / 256) * batches < 200) tn = 128;
   const int tiles = ((N + kGemmRowsW - 1) / kGemmRowsW) * ((M + tn - 1) / tn) * batches;

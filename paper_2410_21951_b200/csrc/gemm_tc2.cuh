@@ -1,0 +1,159 @@
+// bf16 projections for many tokens (tensor-bound shapes) on CTA pairs: tcgen05.mma.cta_group::2.
+// The two CTAs of a cluster compute a 256-feature x TN-token tile together: each CTA stages its own 128
+// weight rows (the MMA's A operand) and half of the token tile (TN/2 rows of the B operand); the pair's
+// MMA reads both halves of B, so an SM fetches 16 KB + TN/2 * 128 B per 64-wide K step instead of the
+// 16 KB + TN * 128 B of the single-CTA kernel: fewer operand bytes from L2 per flop, and a deeper ring in
+// the same shared memory.  The accumulator of each CTA (its 128 features x TN tokens) is in its own TMEM.
+//
+// Protocol: CTA 0 of the pair leads.  Both CTAs issue their TMA loads with the leader's `full` barrier
+// as completion barrier (the leader expects the bytes of both); the leader's MMA thread issues the pair's
+// MMAs and signals, through tcgen05.commit to both CTAs, the `empty` barrier of a stage and at the
+// end the accumulator barrier.  TMEM is allocated and freed by warp 1 of both CTAs; the CTAs
+// meet at a cluster barrier after the barrier set-up and before the TMEM is freed.
+// No K split and no LayerNorm operand here; every wait is bounded like in the single-CTA kernel.
+#pragma once
+#include "tc.cuh"
+#include "gemm_tc.cuh"
+
+namespace vadusa {
+
+template <int TN> struct GemmTc2Cfg {
+  static constexpr int kXHalfBytes = (TN / 2) * kGemmBK * 2;
+  static constexpr int kStageBytes = kGemmRowsW * kGemmBK * 2 + kXHalfBytes;
+  // two CTAs (of different pairs) share an SM: one's epilogue overlaps the other's main loop
+  static constexpr int kStages = (kGemmSmemBudget / 2) / kStageBytes;
+  static constexpr int kTmemCols = TN;
+  static constexpr int kSmem = kStages * kStageBytes + 1024 /*alignment*/ + 256 /*barriers*/;
+};
+
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+  return remote;
+}
+// TMA tile load of a CTA pair: the data lands in this CTA's shared memory, the bytes are counted on an
+// mbarrier that may be the peer's (a shared::cluster address).
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t holder, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B^T for one K step of 16 elements; issued by one thread of the leader.
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"((uint32_t)accumulate)
+      : "memory");
+}
+// One arrival on the mbarrier at this shared-memory offset in both CTAs of the pair once all MMAs issued
+// so far by this thread have completed.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t both = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(both) : "memory");
+}
+
+template <int TN, typename Epi>
+__global__ void __launch_bounds__(128) gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmW,
+                                                       const __grid_constant__ CUtensorMap tmX /*box: TN/2 rows*/,
+                                                       int M, int N, int nchunks, Epi epi, uint32_t* err) {
+  using Cfg = GemmTc2Cfg<TN>;
+  constexpr int S = Cfg::kStages;
+  constexpr uint32_t kWBytes = kGemmRowsW * kGemmBK * 2, kXBytes = Cfg::kXHalfBytes;
+  constexpr int kRing = S * Cfg::kStageBytes;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* ring_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bars = base + kRing;                    // full[S], empty[S], accum, tmem holder
+  const uint32_t full0 = bars, empty0 = bars + 8 * S, accum_bar = bars + 16 * S, holder = bars + 16 * S + 8;
+  volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(ring_ptr + kRing + 16 * S + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();                  // 0: leader
+  const int n0 = blockIdx.x * kGemmRowsW, m0 = blockIdx.y * TN;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    mbar_init(accum_bar, 1);
+    mbar_fence_init();
+    tma_prefetch_desc(&tmW);
+    tma_prefetch_desc(&tmX);
+  }
+  if (warp == 1) { tmem_alloc_pair(holder, Cfg::kTmemCols); tmem_relinquish_pair(); }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                                    // the peer's barriers exist before anything signals them
+  tc_fence_after();
+  const uint32_t tmem = *holder_ptr;
+
+  if (warp == 0 && lane == 0) {
+    // ---- TMA producer (both CTAs): own weight rows, own half of the token tile
+    const int pre = nchunks < S ? nchunks : S;
+    for (int i = 0; i < pre; ++i) {                      // weights do not depend on the upstream kernel
+      if (rank == 0) mbar_expect_tx(full0 + 8 * i, 2 * (kWBytes + kXBytes));
+      tma_load_3d_pair(base + i * Cfg::kStageBytes, &tmW, map_to_cta(full0 + 8 * i, 0), i * kGemmBK, n0, 0);
+    }
+    grid_dep_wait();
+    for (int i = 0; i < pre; ++i)
+      tma_load_3d_pair(base + i * Cfg::kStageBytes + kWBytes, &tmX, map_to_cta(full0 + 8 * i, 0), i * kGemmBK,
+                       m0 + (int)rank * (TN / 2), 0);
+    for (int i = pre; i < nchunks; ++i) {
+      const int s = i % S;
+      if (!mbar_wait(empty0 + 8 * s, ((i / S) - 1) & 1, err)) break;
+      if (rank == 0) mbar_expect_tx(full0 + 8 * s, 2 * (kWBytes + kXBytes));
+      const uint32_t fb = map_to_cta(full0 + 8 * s, 0);
+      tma_load_3d_pair(base + s * Cfg::kStageBytes, &tmW, fb, i * kGemmBK, n0, 0);
+      tma_load_3d_pair(base + s * Cfg::kStageBytes + kWBytes, &tmX, fb, i * kGemmBK, m0 + (int)rank * (TN / 2), 0);
+    }
+  }
+  if (warp == 1 && lane == 0 && rank == 0) {
+    // ---- MMA issuer (leader only): 256 features x TN tokens per instruction
+    constexpr uint32_t idesc = umma_idesc_bf16(2 * kGemmRowsW, TN);
+    for (int i = 0; i < nchunks; ++i) {
+      const int s = i % S;
+      if (!mbar_wait(full0 + 8 * s, (i / S) & 1, err)) break;
+      tc_fence_after();
+      const uint32_t wa = base + s * Cfg::kStageBytes, xa = wa + kWBytes;
+#pragma unroll
+      for (int k = 0; k < kGemmBK / 16; ++k)
+        umma_bf16_pair(tmem, umma_desc_k_sw128(wa + 32 * k), umma_desc_k_sw128(xa + 32 * k), idesc, (i | k) != 0);
+      umma_commit_pair(empty0 + 8 * s);                  // the stage is reusable in both CTAs
+    }
+    umma_commit_pair(accum_bar);                         // both accumulators complete
+  }
+  __syncwarp();
+  grid_dep_wait();
+  const bool done = mbar_wait(accum_bar, 0, err);
+  tc_fence_after();
+  grid_dep_launch();
+
+  // ---- epilogue: warp w reads TMEM lanes 32w .. 32w+31 (features n0 + 32w + lane) of this CTA
+  const int n = n0 + 32 * warp + lane;
+  const uint32_t trow = tmem + ((uint32_t)(32 * warp) << 16);
+  if (done) {
+#pragma unroll 1
+    for (int c0 = 0; c0 < TN; c0 += 32) {
+      float v[32];
+      tmem_ld32(trow + c0, v);
+      if (n < N && m0 + c0 < M) epi.template col<32>(0, m0 + c0, n, v, M - (m0 + c0));
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                                    // neither CTA frees while the other still reads
+  if (warp == 1) tmem_dealloc_pair(tmem, Cfg::kTmemCols);
+}
+
+}  // namespace vadusa
