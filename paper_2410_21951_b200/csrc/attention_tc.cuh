@@ -9,15 +9,16 @@
 // warps 2-3 (lanes 64..127) on keys 32..63.  Per page:
 //   S = Q K^T      tcgen05.mma, A = Q tile, B = K tile, D in one of two TMEM score buffers (columns
 //                  0..63 / 64..127), issued one page ahead so that it overlaps the previous softmax
-//   softmax        each thread reads its 32 scores, keeps a scaling maximum of its own for its key
-//                  half of the row, and the weights go back to TMEM as
-//                  two bf16 halves (p = hi + lo, 16 significant bits) over the score columns,
-//                  zero in the other thread's key range
-//   O += P V       tcgen05.mma with A from TMEM (hi then lo), B = V tile (MN-major), accumulating
-//                  in TMEM columns 128..191; lanes r and r + 64 hold the two key-halves' sums
+//   softmax        each thread reads its 32 scores; the two threads of a row agree on the row's scaling
+//                  maximum through shared memory; each turns its 32 weights into two bf16 halves
+//                  (p = hi + lo, 16 significant bits).  Lane r of the P operand holds the hi halves of
+//                  all 64 keys and lane r + 64 the lo halves, so the two threads swap the half the other
+//                  one stores (through shared memory, a 64-thread named barrier per warp pair)
+//   O += P V       tcgen05.mma with A from TMEM, B = V tile (MN-major), accumulating in TMEM columns
+//                  128..191; lane r sums hi * V and lane r + 64 sums lo * V: no zero padding, one pass
 // The scaling maximum of a row only moves when the page maximum exceeds it by more than 2^6
-// (p <= 64 is harmless in fp32 / bf16); then the row's accumulator is rescaled in TMEM.
-// At the end rows r and r + 64 are brought to a common scale and added; splits are merged through an exchange area in global
+// (p <= 64 is harmless in fp32 / bf16); then the row's accumulators are rescaled in TMEM.
+// At the end rows r and r + 64 are added; splits are merged through an exchange area in global
 // memory (L2) in a fixed order.  Warps: 0-3 softmax, warp 4 lane 0 TMA producer, warp 5 TMEM owner / MMA issuer.
 #pragma once
 #include "tc.cuh"
@@ -28,7 +29,8 @@ constexpr int kAttStages = 4;
 constexpr int kAttThreads = 192;
 constexpr int kAttTileBytes = 64 * 64 * 2;                                   // one K or V page tile
 constexpr int kAttRingBytes = kAttStages * 2 * kAttTileBytes;                // 64 KB; also holds the 64x64 fp32 output exchange
-constexpr int kAttSmemBytes = 2 * kAttTileBytes /*Q, 128 rows*/ + kAttRingBytes + 1024 /*max exchange, block ids*/ +
+constexpr int kAttSwapBytes = 512 /*row maxima*/ + 128 * 64 /*16 words of bf16 pairs per thread*/;
+constexpr int kAttSmemBytes = 2 * kAttTileBytes /*Q, 128 rows*/ + kAttRingBytes + kAttSwapBytes + 1024 /*sums, maxima*/ +
                               1024 /*alignment*/ + 256 /*barriers*/;
 constexpr float kAttRescaleStep = 6.0f;                                      // log2 units
 
@@ -88,11 +90,13 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t q_addr = base, ring = base + 2 * kAttTileBytes;
   uint8_t* ring_ptr = base_ptr + 2 * kAttTileBytes;
-  float* lx = reinterpret_cast<float*>(ring_ptr + kAttRingBytes);            // end of the kernel: [128] partial sums, [128] scaling maxima
-  const uint32_t bars = ring + kAttRingBytes + 1024;
+  float* mxs = reinterpret_cast<float*>(ring_ptr + kAttRingBytes);           // [128] page maxima of the softmax threads
+  uint4* pxs = reinterpret_cast<uint4*>(ring_ptr + kAttRingBytes + 512);     // [4][128] weight halves handed to the row's other thread
+  float* lx = reinterpret_cast<float*>(ring_ptr + kAttRingBytes + kAttSwapBytes);   // end of the kernel: [128] partial sums, [128] scaling maxima
+  const uint32_t bars = ring + kAttRingBytes + kAttSwapBytes + 1024;
   const uint32_t full0 = bars, empty0 = bars + 8 * S, bar_q = bars + 16 * S, bar_s0 = bar_q + 8, bar_p = bar_q + 24,
                  bar_o = bar_q + 32, holder = bar_q + 40;      // bar_s0, bar_s0 + 8: one per score buffer
-  volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(ring_ptr + kAttRingBytes + 1024 + 16 * S + 40);
+  volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(ring_ptr + kAttRingBytes + kAttSwapBytes + 1024 + 16 * S + 40);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int h = blockIdx.x, split = blockIdx.z;
@@ -188,16 +192,15 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
 #pragma unroll
         for (int k = 0; k < 4; ++k)          // 16 keys per step: 8 TMEM columns of A, 16 rows (2048 bytes) of V
           umma_bf16_ts(tmem + 128, pa + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, (i | k) != 0);
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-          umma_bf16_ts(tmem + 128, pa + 32 + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, true);
         umma_commit(empty0 + 8 * (i % S));
         umma_commit(bar_o);
       }
     }
   } else {
     // ---- softmax: thread tid owns TMEM lane tid = query row (tid & 63), keys 32*half .. 32*half+31 of each page
-    const int row = tid & 63, half = tid >> 6;
+    const int row = tid & 63, half = tid >> 6, partner = tid ^ 64;
+    const uint32_t pair_bar = 1u + (uint32_t)(warp & 1);             // warps 0, 2 and warps 1, 3 hold the same rows
+    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory"); };
     unsigned long long alo = 0ull, ahi = 0ull;                     // ancestor-or-self bits of this row's node
     if (node0 + row < nv) tree.anc_of(b, node0 + row, alo, ahi);
     const uint32_t trow = tmem + ((uint32_t)(32 * warp) << 16);
@@ -231,8 +234,10 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
         }
         fence_proxy_async_smem();
       }
-      // each key half of a row keeps its own scaling maximum (the halves accumulate in separate TMEM lanes
-      // and are brought to a common scale once, at the end)
+      // the row's page maximum over both key halves: lanes r and r + 64 of the accumulator share a scale
+      mxs[tid] = mx;
+      pair_sync();
+      mx = fmaxf(mx, mxs[partner]);
       mx *= scale_log2e;                      // raw scores; the (positive) scale moves into the exponent
       // move the scaling maximum only when the page maximum exceeds it by more than the step
       float factor = 1.f;
@@ -268,15 +273,21 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
         lv[j] = pack_bf16(pa - ha, pb - hb);
       }
       l_run += (psum4[0] + psum4[1]) + (psum4[2] + psum4[3]);
-      // this thread's 32 keys sit in columns 16*half .. 16*half+15 of each 32-column group; zero elsewhere
+      // keys 0..31 sit in columns 0..15 and keys 32..63 in columns 16..31 of the P operand; lane r (half 0)
+      // takes the hi halves of the whole row, lane r + 64 (half 1) the lo halves: hand over the other one
       {
-        uint32_t zero[16];
+        const uint32_t* give = half ? hv : lv;
 #pragma unroll
-        for (int j = 0; j < 16; ++j) zero[j] = 0u;
-        tmem_st16(tsp + 16 * half, hv);
-        tmem_st16(tsp + 16 * (1 - half), zero);
-        tmem_st16(tsp + 32 + 16 * half, lv);
-        tmem_st16(tsp + 32 + 16 * (1 - half), zero);
+        for (int c = 0; c < 4; ++c) pxs[c * 128 + tid] = make_uint4(give[4 * c], give[4 * c + 1], give[4 * c + 2], give[4 * c + 3]);
+        pair_sync();
+        uint32_t got[16];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const uint4 v = pxs[c * 128 + partner];
+          got[4 * c] = v.x; got[4 * c + 1] = v.y; got[4 * c + 2] = v.z; got[4 * c + 3] = v.w;
+        }
+        if (half == 0) { tmem_st16(tsp, hv); tmem_st16(tsp + 16, got); }
+        else { tmem_st16(tsp, got); tmem_st16(tsp + 16, lv); }
       }
       tmem_st_wait();
       tc_fence_before();
