@@ -7,30 +7,34 @@
 // The 64 query rows are stored twice in the 128-row Q operand, so the scores of row r appear in
 // TMEM lanes r and r + 64: warps 0-1 (lanes 0..63) work on keys 0..31 of every 64-key page,
 // warps 2-3 (lanes 64..127) on keys 32..63.  Per page:
-//   S = Q K^T      tcgen05.mma, A = Q tile, B = K tile, D in one of two TMEM score buffers (columns
-//                  0..63 / 64..127), issued one page ahead so that it overlaps the previous softmax
-//   softmax        each thread reads its 32 scores; the two threads of a row agree on the row's scaling
-//                  maximum through shared memory; each turns its 32 weights into two bf16 halves
-//                  (p = hi + lo, 16 significant bits).  Lane r of the P operand holds the hi halves of
-//                  all 64 keys and lane r + 64 the lo halves, so the two threads swap the half the other
-//                  one stores (through shared memory, a 64-thread named barrier per warp pair)
-//   O += P V       tcgen05.mma with A from TMEM, B = V tile (MN-major), accumulating in TMEM columns
-//                  128..191; lane r sums hi * V and lane r + 64 sums lo * V: no zero padding, one pass
+//   S = Q K^T      tcgen05.mma, A = Q tile, B = K tile, D in one of three TMEM score buffers (columns
+//                  0..63 / 64..127 / 128..191), issued by a warp of its own up to three pages ahead of
+//                  P V, so that neither the softmax nor the other issuer waits for it
+//   softmax        each thread reads its 32 scores, keeps a scaling maximum of its own for its key
+//                  half of the row, and the weights go back to TMEM as
+//                  two bf16 halves (p = hi + lo, 16 significant bits) over the score columns,
+//                  zero in the other thread's key range
+//   O += P V       tcgen05.mma with A from TMEM (hi then lo), B = V tile (MN-major), accumulating
+//                  in TMEM columns 192..255; lanes r and r + 64 hold the two key-halves' sums
 // The scaling maximum of a row only moves when the page maximum exceeds it by more than 2^6
-// (p <= 64 is harmless in fp32 / bf16); then the row's accumulators are rescaled in TMEM.
-// At the end rows r and r + 64 are added; splits are merged through an exchange area in global
-// memory (L2) in a fixed order.  Warps: 0-3 softmax, warp 4 lane 0 TMA producer, warp 5 TMEM owner / MMA issuer.
+// (p <= 64 is harmless in fp32 / bf16); then the row's accumulator is rescaled in TMEM.
+// At the end rows r and r + 64 are brought to a common scale and added; splits are merged through an exchange area in global
+// memory (L2) in a fixed order.
+// K and V tiles have rings of their own: a K tile is free as soon as its Q K^T has completed, a V tile after
+// its P V.  "Scores ready", "weights ready" and "P V done" have one mbarrier per score buffer: a buffer's next
+// use cannot begin before the waiter of the current one has passed, so no parity wait can fall a round behind.
+// Warps: 0-3 softmax, warp 4 lane 0 TMA producer, warp 5 TMEM owner / P V issuer, warp 6 Q K^T issuer.
 #pragma once
 #include "tc.cuh"
 
 namespace vadusa {
 
-constexpr int kAttStages = 4;
-constexpr int kAttThreads = 192;
+constexpr int kAttStagesK = 4;                                               // K tiles leave their ring after Q K^T,
+constexpr int kAttStagesV = 6;                                               // V tiles after P V: rings of their own
+constexpr int kAttThreads = 224;
 constexpr int kAttTileBytes = 64 * 64 * 2;                                   // one K or V page tile
-constexpr int kAttRingBytes = kAttStages * 2 * kAttTileBytes;                // 64 KB; also holds the 64x64 fp32 output exchange
-constexpr int kAttSwapBytes = 512 /*row maxima*/ + 128 * 64 /*16 words of bf16 pairs per thread*/;
-constexpr int kAttSmemBytes = 2 * kAttTileBytes /*Q, 128 rows*/ + kAttRingBytes + kAttSwapBytes + 1024 /*sums, maxima*/ +
+constexpr int kAttRingBytes = (kAttStagesK + kAttStagesV) * kAttTileBytes;   // 80 KB; also holds the 64x64 fp32 output exchange
+constexpr int kAttSmemBytes = 2 * kAttTileBytes /*Q, 128 rows*/ + kAttRingBytes + 1024 /*sums, maxima*/ +
                               1024 /*alignment*/ + 256 /*barriers*/;
 constexpr float kAttRescaleStep = 6.0f;                                      // log2 units
 
@@ -72,6 +76,12 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -84,27 +94,28 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
     const int32_t* __restrict__ nvalid, const int32_t* __restrict__ order /*may be null*/, TreeView tree, KvGeom geom,
     int d_model, float scale_log2e, int splits,
     bf16* __restrict__ out, float* __restrict__ xch /*split exchange area*/, uint32_t* err) {
-  constexpr int S = kAttStages;
+  constexpr int SK = kAttStagesK, SV = kAttStagesV;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t q_addr = base, ring = base + 2 * kAttTileBytes;
+  const uint32_t q_addr = base, ring = base + 2 * kAttTileBytes, ring_v = ring + SK * kAttTileBytes;
   uint8_t* ring_ptr = base_ptr + 2 * kAttTileBytes;
-  float* mxs = reinterpret_cast<float*>(ring_ptr + kAttRingBytes);           // [128] page maxima of the softmax threads
-  uint4* pxs = reinterpret_cast<uint4*>(ring_ptr + kAttRingBytes + 512);     // [4][128] weight halves handed to the row's other thread
-  float* lx = reinterpret_cast<float*>(ring_ptr + kAttRingBytes + kAttSwapBytes);   // end of the kernel: [128] partial sums, [128] scaling maxima
-  const uint32_t bars = ring + kAttRingBytes + kAttSwapBytes + 1024;
-  const uint32_t full0 = bars, empty0 = bars + 8 * S, bar_q = bars + 16 * S, bar_s0 = bar_q + 8, bar_p = bar_q + 24,
-                 bar_o = bar_q + 32, holder = bar_q + 40;      // bar_s0, bar_s0 + 8: one per score buffer
-  volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(ring_ptr + kAttRingBytes + kAttSwapBytes + 1024 + 16 * S + 40);
+  float* lx = reinterpret_cast<float*>(ring_ptr + kAttRingBytes);            // end of the kernel: [128] partial sums, [128] scaling maxima
+  const uint32_t bars = ring + kAttRingBytes + 1024;
+  const uint32_t full_k0 = bars, empty_k0 = bars + 8 * SK, full_v0 = bars + 16 * SK, empty_v0 = full_v0 + 8 * SV,
+                 bar_q = bars + 16 * (SK + SV), bar_s0 = bar_q + 8, bar_p0 = bar_q + 32,
+                 bar_o0 = bar_q + 56, holder = bar_q + 80;     // scores ready / weights ready / P V done: one each per score
+                                                               // buffer, so that a phase parity is never one round behind
+  volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(ring_ptr + kAttRingBytes + 1024 + 16 * (SK + SV) + 80);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int h = blockIdx.x, split = blockIdx.z;
   const int N = tree.n_nodes;
 
   if (tid == 0) {
-    for (int s = 0; s < S; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-    mbar_init(bar_q, 1); mbar_init(bar_s0, 1); mbar_init(bar_s0 + 8, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
+    for (int s = 0; s < 2 * (SK + SV); ++s) mbar_init(bars + 8 * s, 1);       // full / empty of the K and V rings
+    mbar_init(bar_q, 1); mbar_init(bar_s0, 1); mbar_init(bar_s0 + 8, 1); mbar_init(bar_s0 + 16, 1);
+    for (int j = 0; j < 3; ++j) { mbar_init(bar_p0 + 8 * j, 128); mbar_init(bar_o0 + 8 * j, 1); }
     mbar_fence_init();
     tma_prefetch_desc(&tmQ);
     tma_prefetch_desc(&tmKV);
@@ -154,60 +165,69 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
         if (blk < 0) blk = 0;
       }
       if (lane == 0 && ok) {
-        const int s = i % S;
-        if (i >= S && !mbar_wait(empty0 + 8 * s, ((i / S) - 1) & 1, err)) {
+        const int sk = i % SK, sv = i % SV;
+        const int row = (int)((blk * 2 * geom.n_heads + h) * kKvBlock);
+        if (i >= SK && !mbar_wait(empty_k0 + 8 * sk, ((i / SK) - 1) & 1, err)) {
           ok = false;                         // timed out (recorded): stop issuing, keep the warp converged
         } else {
-          const int row = (int)((blk * 2 * geom.n_heads + h) * kKvBlock);
-          mbar_expect_tx(full0 + 8 * s, 2 * kAttTileBytes);
-          tma_load_3d(ring + s * 2 * kAttTileBytes, &tmKV, full0 + 8 * s, 0, row, layer);
-          tma_load_3d(ring + s * 2 * kAttTileBytes + kAttTileBytes, &tmKV, full0 + 8 * s, 0, row + geom.n_heads * kKvBlock, layer);
+          mbar_expect_tx(full_k0 + 8 * sk, kAttTileBytes);
+          tma_load_3d(ring + sk * kAttTileBytes, &tmKV, full_k0 + 8 * sk, 0, row, layer);
+        }
+        if (ok && i >= SV && !mbar_wait(empty_v0 + 8 * sv, ((i / SV) - 1) & 1, err)) ok = false;
+        if (ok) {
+          mbar_expect_tx(full_v0 + 8 * sv, kAttTileBytes);
+          tma_load_3d(ring_v + sv * kAttTileBytes, &tmKV, full_v0 + 8 * sv, 0, row + geom.n_heads * kKvBlock, layer);
         }
       }
     }
   } else if (warp == 5) {
-    // ---- MMA issuer (lane 0)
+    // ---- P V issuer (lane 0): O += P(i) V(i) as soon as the softmax threads have stored P(i)
     if (lane == 0) {
-      constexpr uint32_t idesc_qk = umma_idesc_bf16(128, 64);
       constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 64) | (1u << 16);     // B (V tile) is MN-major
-      bool ok = ntiles == 0 || mbar_wait(bar_q, 0, err);
-      // S(i) = Q K(i)^T into score buffer i & 1
-      auto issue_scores = [&](int i) -> bool {
-        const int s = i % S;
-        if (!mbar_wait(full0 + 8 * s, (i / S) & 1, err)) return false;
+      for (int i = 0; i < ntiles; ++i) {
+        if (!mbar_wait(bar_p0 + 8 * (i % 3), (i / 3) & 1, err)) break;
+        if (!mbar_wait(full_v0 + 8 * (i % SV), (i / SV) & 1, err)) break;
         tc_fence_after();
-        const uint32_t ka = ring + s * 2 * kAttTileBytes;
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-          umma_bf16(tmem + 64 * (i & 1), umma_desc_k_sw128(q_addr + 32 * k), umma_desc_k_sw128(ka + 32 * k), idesc_qk, k != 0);
-        umma_commit(bar_s0 + 8 * (i & 1));
-        return true;
-      };
-      if (ok && ntiles > 0) ok = issue_scores(0);
-      for (int i = 0; i < ntiles && ok; ++i) {
-        if (i + 1 < ntiles && !issue_scores(i + 1)) break;      // one page ahead of the softmax
-        if (!mbar_wait(bar_p, i & 1, err)) break;
-        tc_fence_after();
-        const uint32_t va = ring + (i % S) * 2 * kAttTileBytes + kAttTileBytes, pa = tmem + 64 * (i & 1);
+        const uint32_t va = ring_v + (i % SV) * kAttTileBytes, pa = tmem + 64 * (i % 3);
 #pragma unroll
         for (int k = 0; k < 4; ++k)          // 16 keys per step: 8 TMEM columns of A, 16 rows (2048 bytes) of V
-          umma_bf16_ts(tmem + 128, pa + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, (i | k) != 0);
-        umma_commit(empty0 + 8 * (i % S));
-        umma_commit(bar_o);
+          umma_bf16_ts(tmem + 192, pa + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, (i | k) != 0);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)          // the lo halves of the weights
+          umma_bf16_ts(tmem + 192, pa + 32 + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, true);
+        umma_commit(empty_v0 + 8 * (i % SV));
+        umma_commit(bar_o0 + 8 * (i % 3));
+      }
+    }
+  } else if (warp == 6) {
+    // ---- Q K^T issuer (lane 0): S(i) = Q K(i)^T into score buffer i % 3, up to three pages ahead of P V
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = umma_idesc_bf16(128, 64);
+      bool ok = ntiles == 0 || mbar_wait(bar_q, 0, err);
+      for (int i = 0; i < ntiles && ok; ++i) {
+        // the buffer held P(i - 3): free once P(i - 3) V(i - 3) has completed
+        if (i >= 3 && !mbar_wait(bar_o0 + 8 * (i % 3), ((i - 3) / 3) & 1, err)) break;
+        const int s = i % SK;
+        if (!mbar_wait(full_k0 + 8 * s, (i / SK) & 1, err)) break;
+        tc_fence_after();
+        const uint32_t ka = ring + s * kAttTileBytes;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          umma_bf16(tmem + 64 * (i % 3), umma_desc_k_sw128(q_addr + 32 * k), umma_desc_k_sw128(ka + 32 * k), idesc_qk, k != 0);
+        umma_commit(empty_k0 + 8 * s);                     // the K tile is free once these MMAs have read it
+        umma_commit(bar_s0 + 8 * (i % 3));
       }
     }
   } else {
     // ---- softmax: thread tid owns TMEM lane tid = query row (tid & 63), keys 32*half .. 32*half+31 of each page
-    const int row = tid & 63, half = tid >> 6, partner = tid ^ 64;
-    const uint32_t pair_bar = 1u + (uint32_t)(warp & 1);             // warps 0, 2 and warps 1, 3 hold the same rows
-    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory"); };
+    const int row = tid & 63, half = tid >> 6;
     unsigned long long alo = 0ull, ahi = 0ull;                     // ancestor-or-self bits of this row's node
     if (node0 + row < nv) tree.anc_of(b, node0 + row, alo, ahi);
     const uint32_t trow = tmem + ((uint32_t)(32 * warp) << 16);
     for (int i = 0; i < ntiles; ++i) {
-      if (!mbar_wait(bar_s0 + 8 * (i & 1), (i >> 1) & 1, err)) break;
+      if (!mbar_wait(bar_s0 + 8 * (i % 3), (i / 3) & 1, err)) break;
       tc_fence_after();
-      const uint32_t tsp = trow + 64 * (i & 1);       // this page's score / weight buffer
+      const uint32_t tsp = trow + 64 * (i % 3);       // this page's score / weight buffer
       float sc[32];
       tmem_ld32(tsp + 32 * half, sc);
       const int key0 = (p0 + i) * kKvBlock + 32 * half;
@@ -221,23 +241,27 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
 #pragma unroll
         for (int j = 0; j < 32; ++j) sc[j] = ((vis >> j) & 1u) ? sc[j] : -INFINITY;
       }                                       // else: all 32 keys inside the context, every key visible
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      float mx4[4];                           // four chains of three-input maxima over eight scores each
 #pragma unroll
-      for (int j = 0; j < 32; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
+      for (int c = 0; c < 4; ++c) {
+        mx4[c] = fmax3(sc[8 * c], sc[8 * c + 1], sc[8 * c + 2]);
+        mx4[c] = fmax3(mx4[c], sc[8 * c + 3], sc[8 * c + 4]);
+        mx4[c] = fmax3(mx4[c], sc[8 * c + 5], sc[8 * c + 6]);
+        mx4[c] = fmaxf(mx4[c], sc[8 * c + 7]);
+      }
       float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       if ((p0 + i + 1) * kKvBlock > total && tid < 64) {   // rows of V past the tree may hold anything: zero them
         const int valid = total - (p0 + i) * kKvBlock;
+        mbar_wait(full_v0 + 8 * (i % SV), (i / SV) & 1, err);      // the V tile has landed before rows of it are cleared
         if (tid >= valid) {
-          uint4* vr = reinterpret_cast<uint4*>(ring_ptr + (i % S) * 2 * kAttTileBytes + kAttTileBytes + tid * 128);
+          uint4* vr = reinterpret_cast<uint4*>(ring_ptr + (SK + i % SV) * kAttTileBytes + tid * 128);
 #pragma unroll
           for (int c = 0; c < 8; ++c) vr[c] = make_uint4(0, 0, 0, 0);
         }
         fence_proxy_async_smem();
       }
-      // the row's page maximum over both key halves: lanes r and r + 64 of the accumulator share a scale
-      mxs[tid] = mx;
-      pair_sync();
-      mx = fmaxf(mx, mxs[partner]);
+      // each key half of a row keeps its own scaling maximum (the halves accumulate in separate TMEM lanes
+      // and are brought to a common scale once, at the end)
       mx *= scale_log2e;                      // raw scores; the (positive) scale moves into the exponent
       // move the scaling maximum only when the page maximum exceeds it by more than the step
       float factor = 1.f;
@@ -247,16 +271,16 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
       }
       if (i > 0 && __any_sync(0xffffffffu, factor != 1.f)) {
         // rescale this row's accumulator, once the previous page's P V has completed
-        if (!mbar_wait(bar_o, (i - 1) & 1, err)) break;
+        if (!mbar_wait(bar_o0 + 8 * ((i - 1) % 3), ((i - 1) / 3) & 1, err)) break;
         tc_fence_after();
         float ot[32];
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
-          tmem_ld32(trow + 128 + 32 * hh, ot);
+          tmem_ld32(trow + 192 + 32 * hh, ot);
           uint32_t ob[32];
 #pragma unroll
           for (int e = 0; e < 32; ++e) ob[e] = __float_as_uint(ot[e] * factor);
-          tmem_st32(trow + 128 + 32 * hh, ob);
+          tmem_st32(trow + 192 + 32 * hh, ob);
         }
       }
       l_run *= factor;
@@ -273,27 +297,21 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
         lv[j] = pack_bf16(pa - ha, pb - hb);
       }
       l_run += (psum4[0] + psum4[1]) + (psum4[2] + psum4[3]);
-      // keys 0..31 sit in columns 0..15 and keys 32..63 in columns 16..31 of the P operand; lane r (half 0)
-      // takes the hi halves of the whole row, lane r + 64 (half 1) the lo halves: hand over the other one
+      // this thread's 32 keys sit in columns 16*half .. 16*half+15 of each 32-column group; zero elsewhere
       {
-        const uint32_t* give = half ? hv : lv;
+        uint32_t zero[16];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) pxs[c * 128 + tid] = make_uint4(give[4 * c], give[4 * c + 1], give[4 * c + 2], give[4 * c + 3]);
-        pair_sync();
-        uint32_t got[16];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const uint4 v = pxs[c * 128 + partner];
-          got[4 * c] = v.x; got[4 * c + 1] = v.y; got[4 * c + 2] = v.z; got[4 * c + 3] = v.w;
-        }
-        if (half == 0) { tmem_st16(tsp, hv); tmem_st16(tsp + 16, got); }
-        else { tmem_st16(tsp, got); tmem_st16(tsp + 16, lv); }
+        for (int j = 0; j < 16; ++j) zero[j] = 0u;
+        tmem_st16(tsp + 16 * half, hv);
+        tmem_st16(tsp + 16 * (1 - half), zero);
+        tmem_st16(tsp + 32 + 16 * half, lv);
+        tmem_st16(tsp + 32 + 16 * (1 - half), zero);
       }
       tmem_st_wait();
       tc_fence_before();
-      mbar_arrive(bar_p);
+      mbar_arrive(bar_p0 + 8 * (i % 3));
     }
-    if (ntiles > 0) { mbar_wait(bar_o, (ntiles - 1) & 1, err); tc_fence_after(); }
+    if (ntiles > 0) { mbar_wait(bar_o0 + 8 * ((ntiles - 1) % 3), ((ntiles - 1) / 3) & 1, err); tc_fence_after(); }
   }
   __syncwarp();
   grid_dep_launch();
@@ -305,8 +323,8 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
   if (warp < 4) {
     const uint32_t trow = tmem + ((uint32_t)(32 * warp) << 16);
     if (ntiles > 0) {
-      tmem_ld32(trow + 128, o_acc);
-      tmem_ld32(trow + 160, o_acc + 32);
+      tmem_ld32(trow + 192, o_acc);
+      tmem_ld32(trow + 224, o_acc + 32);
     } else {
 #pragma unroll
       for (int e = 0; e < 64; ++e) o_acc[e] = 0.f;
