@@ -421,8 +421,8 @@ def _random_context(model, S, rng, scale=1.0):
 def test_long_ragged_contexts_with_injected_kv(name):
     """BASELINE configs 4 and 5 at full batch and context lengths: the KV cache holds
     seeded random bf16 rows (so no prefill is needed on either side), tree tokens and the
-    carried state are random; the oracle scores three sampled sequences (shortest, longest,
-    one other).  C5 uses a random topology per sequence."""
+    carried state are random; the oracle scores four sampled sequences (shortest, longest,
+    two others).  C5 uses a random topology per sequence."""
     torch = _torch()
     wl = W.workload(name)
     w = W.make_weights(wl.shape, wl.seed())
@@ -439,6 +439,12 @@ def test_long_ragged_contexts_with_injected_kv(name):
         g.set_tree(tpls[0].parent, tpls[0].rank)
     order = np.argsort(lens)
     picks = [int(order[0]), int(order[-1]), int(order[B // 2])]
+    # The many-token products run on CTA pairs: each CTA of a pair stages half of a 128- or 256-token
+    # tile, i.e. whole sequences of 64 nodes.  One more sequence, so that the samples fall into both
+    # halves of both tile widths (b % 4 in {0, 1} and {2, 3}; b even and odd).
+    def both_halves(ps):
+        return {b % 4 < 2 for b in ps} == {True, False} and {b % 2 for b in ps} == {0, 1}
+    picks.append(next(b for b in range(B) if b not in picks and both_halves(picks + [b])))
     rng = np.random.default_rng(wl.seed(2))
     # every sequence gets random K/V on the GPU; the sampled ones also in the oracle
     view = g.kv_view()
