@@ -294,15 +294,15 @@ vadusa_status launch_gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void
 }
 
 // Many-token product on CTA pairs (256 features x TN tokens per pair, no K split).
-template <int TN, typename Epi>
+template <int TN, int ST, typename Epi>
 vadusa_status launch_gemm_tc2(vadusa_ctx* ctx, int cls, const void* X, const void* W, int w_rows, int M, int N, int K,
                               const Epi& epi) {
-  using Cfg = GemmTc2Cfg<TN>;
+  using Cfg = GemmTc2Cfg<TN, ST>;
   static unsigned long long attr_done = 0ull;              // per device, like launch_gemm_tc
   const unsigned long long dev_bit = 1ull << (ctx->cfg.device & 63);
   if (!(attr_done & dev_bit)) {
-    CU(cudaFuncSetAttribute(gemm_tc2_kernel<TN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmem));
-    CU(cudaFuncSetAttribute(gemm_tc2_kernel<TN, Epi>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+    CU(cudaFuncSetAttribute(gemm_tc2_kernel<TN, ST, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmem));
+    CU(cudaFuncSetAttribute(gemm_tc2_kernel<TN, ST, Epi>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
     attr_done |= dev_bit;
   }
   const CUtensorMap *mw, *mx;
@@ -320,7 +320,7 @@ vadusa_status launch_gemm_tc2(vadusa_ctx* ctx, int cls, const void* X, const voi
   at[1].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = at; lc.numAttrs = 2;
   PROF(ctx, cls);
-  CU(cudaLaunchKernelEx(&lc, gemm_tc2_kernel<TN, Epi>, *mw, *mx, M, N, K / kGemmBK, epi, err_word(ctx)));
+  CU(cudaLaunchKernelEx(&lc, gemm_tc2_kernel<TN, ST, Epi>, *mw, *mx, M, N, K / kGemmBK, epi, err_word(ctx)));
   LAUNCH_CHECK();
   return VADUSA_OK;
 }
@@ -369,10 +369,17 @@ vadusa_status gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void* W, in
   // token tile: as narrow as the token count allows for weight streaming; 256 for the tensor-bound shapes
   // when that still gives every SM a CTA pair, else 128
   const int ntiles_n = (N + kGemmRowsW - 1) / kGemmRowsW;
-  // tensor-bound shapes whose features come in whole pairs of tiles: CTA pairs, when they fill the SMs
+  // tensor-bound shapes whose features come in whole pairs of tiles: CTA pairs, when they fill the SMs.  Of
+  // the 256-token tile (two CTAs per SM) and the 128-token tile (two per SM with four stages when all CTAs are
+  // resident at once, else three per SM with three stages) the one whose last wave is fuller; ties to the wider.
   if (M > 1024 && batches == 1 && N % (2 * kGemmRowsW) == 0) {
-    if (ntiles_n * ((M + 255) / 256) >= 200) return launch_gemm_tc2<256>(ctx, cls, X, W, w_rows, M, N, K, epi);
-    if (ntiles_n * ((M + 127) / 128) >= 200) return launch_gemm_tc2<128>(ctx, cls, X, W, w_rows, M, N, K, epi);
+    auto fill = [](int ctas, int slots) { return (double)ctas / (double)(((ctas + slots - 1) / slots) * slots); };
+    const int c256 = ntiles_n * ((M + 255) / 256), c128 = ntiles_n * ((M + 127) / 128);
+    const double f256 = c256 >= 200 ? fill(c256, 296) : 0.0;
+    const double f128 = c128 >= 200 ? fill(c128, c128 <= 296 ? 296 : 444) : 0.0;
+    if (f256 > 0.0 && f256 >= f128) return launch_gemm_tc2<256, 3>(ctx, cls, X, W, w_rows, M, N, K, epi);
+    if (f128 > 0.0 && c128 <= 296) return launch_gemm_tc2<128, 4>(ctx, cls, X, W, w_rows, M, N, K, epi);
+    if (f128 > 0.0) return launch_gemm_tc2<128, 3>(ctx, cls, X, W, w_rows, M, N, K, epi);
   }
   int tn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 1024 ? 128 : 256;
   if (tn == 256 && ntiles_n * ((M + 255) / 256) * batches < 200) tn = 128;

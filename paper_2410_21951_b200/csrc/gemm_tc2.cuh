@@ -17,11 +17,12 @@
 
 namespace vadusa {
 
-template <int TN> struct GemmTc2Cfg {
+// ST stages of 16 KB of weights + TN/2 token rows.  Several CTAs (of different pairs) share an SM, so that one's
+// epilogue overlaps another's main loop: two with <256, 3> (TMEM: 2 x 256 columns) and <128, 4>, three with <128, 3>.
+template <int TN, int ST> struct GemmTc2Cfg {
   static constexpr int kXHalfBytes = (TN / 2) * kGemmBK * 2;
   static constexpr int kStageBytes = kGemmRowsW * kGemmBK * 2 + kXHalfBytes;
-  // two CTAs (of different pairs) share an SM: one's epilogue overlaps the other's main loop
-  static constexpr int kStages = (kGemmSmemBudget / 2) / kStageBytes;
+  static constexpr int kStages = ST;
   static constexpr int kTmemCols = TN;
   static constexpr int kSmem = kStages * kStageBytes + 1024 /*alignment*/ + 256 /*barriers*/;
 };
@@ -65,11 +66,11 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
                ::"r"(bar), "h"(both) : "memory");
 }
 
-template <int TN, typename Epi>
+template <int TN, int ST, typename Epi>
 __global__ void __launch_bounds__(128) gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmW,
                                                        const __grid_constant__ CUtensorMap tmX /*box: TN/2 rows*/,
                                                        int M, int N, int nchunks, Epi epi, uint32_t* err) {
-  using Cfg = GemmTc2Cfg<TN>;
+  using Cfg = GemmTc2Cfg<TN, ST>;
   constexpr int S = Cfg::kStages;
   constexpr uint32_t kWBytes = kGemmRowsW * kGemmBK * 2, kXBytes = Cfg::kXHalfBytes;
   constexpr int kRing = S * Cfg::kStageBytes;
