@@ -372,11 +372,11 @@ vadusa_status gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void* W, in
   // tensor-bound shapes whose features come in whole pairs of tiles: CTA pairs, when they fill the SMs.  Of
   // the 256-token tile (two CTAs per SM) and the 128-token tile (two per SM with four stages when all CTAs are
   // resident at once, else three per SM with three stages) the one whose last wave is fuller; ties to the wider.
-  if (M > 1024 && batches == 1 && N % (2 * kGemmRowsW) == 0) {
+  if (M > 512 && batches == 1 && N % (2 * kGemmRowsW) == 0) {
     auto fill = [](int ctas, int slots) { return (double)ctas / (double)(((ctas + slots - 1) / slots) * slots); };
     const int c256 = ntiles_n * ((M + 255) / 256), c128 = ntiles_n * ((M + 127) / 128);
-    const double f256 = c256 >= 200 ? fill(c256, 296) : 0.0;
-    const double f128 = c128 >= 200 ? fill(c128, c128 <= 296 ? 296 : 444) : 0.0;
+    const double f256 = c256 >= 128 ? fill(c256, 296) : 0.0;
+    const double f128 = c128 >= 128 ? fill(c128, c128 <= 296 ? 296 : 444) : 0.0;
     if (f256 > 0.0 && f256 >= f128) return launch_gemm_tc2<256, 3>(ctx, cls, X, W, w_rows, M, N, K, epi);
     if (f128 > 0.0 && c128 <= 296) return launch_gemm_tc2<128, 4>(ctx, cls, X, W, w_rows, M, N, K, epi);
     if (f128 > 0.0) return launch_gemm_tc2<128, 3>(ctx, cls, X, W, w_rows, M, N, K, epi);
