@@ -48,6 +48,26 @@ def _gemm_traffic():
     return _NCU_TRAFFIC["bytes_per_step"] if h.hexdigest()[:16] == _NCU_TRAFFIC["src_sha256_16"] else None
 
 
+# DRAM bytes of one tree_attention_tc_kernel launch relative to its algorithmic K/V bytes, from the ncu capture at
+# 24 sequences summarised in profiles/tree_attention_tc_kernel_c5_batch24.md (163.17 MB read + 3.83 MB written for
+# 163.1 MB of K/V); every (head, sequence) CTA reads its own pages once, so the traffic of a launch grows in
+# proportion to its sequences' bytes.  Valid for the kernel sources with this hash only.
+_NCU_ATTN = {"src_sha256_16": "a1b015d014f84a83", "dram_over_algorithmic": 167.0 / 163.1}
+
+
+def _attn_traffic(algorithmic_bytes):
+    import hashlib
+    h = hashlib.sha256()
+    try:
+        for f in ("attention_tc.cuh", "tc.cuh"):
+            h.update(open(os.path.join(ROOT, "paper_2410_21951_b200", "csrc", f), "rb").read())
+    except OSError:
+        return None
+    if h.hexdigest()[:16] != _NCU_ATTN["src_sha256_16"]:
+        return None
+    return algorithmic_bytes * _NCU_ATTN["dram_over_algorithmic"]
+
+
 def _peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -435,7 +455,9 @@ def run_c5(args):
                        "verify_step_us": ms / K * 1e3, "mean_accepted_tokens": tokens / (K * B)},
             "roofline": {"bound": "hbm", "kernel": "tree_attention_tc_kernel", "achieved": att_bytes / (att_us * 1e-6) / 1e9,
                          "peak": hbm, "unit": "GB/s", "frac": att_bytes / (att_us * 1e-6) / 1e9 / hbm,
-                         "peak_source": f"{kind} copy bandwidth", "traffic": None, "avg_launch_us": round(att_us, 1),
+                         "peak_source": f"{kind} copy bandwidth", "traffic": _attn_traffic(att_bytes),
+                         "traffic_unit": "DRAM bytes per launch, scaled from the ncu capture at 24 sequences (null if the kernel changed since)",
+                         "avg_launch_us": round(att_us, 1),
                          "algorithmic_bytes_per_launch": att_bytes,
                          "kernel_time_shares": {k: round(v[1] / tot_ms, 4) for k, v in sorted(prof.items(), key=lambda kv: -kv[1][1])}},
             "tensor_roofline": {"peak_tflops": tf_peak, "peak_source": "measured sustained bf16 matmul", "kernels": gemm},
