@@ -249,6 +249,17 @@ vadusa_status vadusa_get_lengths(vadusa_ctx *ctx, int32_t *h_ctx_len);  /* synch
 vadusa_status vadusa_check(vadusa_ctx *ctx);                            /* synchronises; device error word */
 int64_t vadusa_kernel_launches(const vadusa_ctx *ctx);                  /* total kernels enqueued so far */
 
+/* A verify pass over ONE sequence of at most 64 tree nodes (the batch-1 step of Sec. II-A: one tree per
+ * iteration) runs, for bf16 models with head_dim 64 and 8 or 16 heads, as a single persistent kernel that
+ * keeps the whole grid resident and hands activations from step to step through shared memory of thread-block
+ * clusters and counters in L2, instead of one kernel per projection.  It computes the same quantities with
+ * the same rounding points.  enable = 0 selects the kernel-per-step path for such passes too (used to
+ * compare the two); the default is 1.  Host-side switch: takes effect with the next call. */
+vadusa_status vadusa_set_fused_pass(vadusa_ctx *ctx, int32_t enable);
+/* How many of that kernel's clusters (one per head) the device can hold at once, as found when the first
+ * such pass was enqueued (-1 before).  The persistent kernel is used only if this is >= n_heads. */
+int32_t vadusa_fused_pass_clusters(const vadusa_ctx *ctx);
+
 /* ---- sampler hook (paper Sec. II-C, last paragraph) ----------------------------------------
  * The paper notes that improved sampling strategies (e.g. avoiding repetitions) are used by taking
  * their outcomes as the predictions of the original head, with the tau draws made by the same

@@ -153,7 +153,7 @@ class IterationTrace:
     margin_draft: np.ndarray         # [n_draft]
     draft_gaps: np.ndarray           # [n_draft, kmax]: logit gap between candidates r and r+1 of each head
     margin_accept: float
-    attn: Optional[List[np.ndarray]] = None     # per layer [N, d] (tree mode only)
+    attn: Optional[List[np.ndarray]] = None     # per layer [N, d]: attention output (before the output projection)
     K: Optional[np.ndarray] = None              # [L, N, H, dh] rows of every node (tree/memo mode)
     V: Optional[np.ndarray] = None
     finished: bool = False                      # EOS was committed in this iteration
@@ -224,13 +224,15 @@ def vadusa_iteration(model: Model, st: State, template, sp: Sampling, mode: str 
     node_h = np.full((N, model.d), np.nan)
     node_K = np.zeros((model.L, N, model.H, model.dh)); node_V = np.zeros_like(node_K)
     have = np.zeros(N, dtype=bool)
-    attn = None
+    attn = [np.zeros((N, model.d)) for _ in range(model.L)]      # per layer: attention output of every node
 
     def record(n, out, K1, V1):
         if have[n]:
             assert np.array_equal(node_logits[n], out.logits), "a node's scores depend on the branch"
         node_logits[n], node_h[n] = out.logits, out.h
         node_K[:, n], node_V[:, n] = K1[:, 0], V1[:, 0]
+        for l in range(model.L):
+            attn[l][n] = out.attn[l]
         have[n] = True
 
     leaves = template.leaves()
@@ -238,7 +240,7 @@ def vadusa_iteration(model: Model, st: State, template, sp: Sampling, mode: str 
         for leaf in leaves:
             bkv = st.kv.branch()
             for i, n in enumerate(template.node_path(leaf)):
-                out = forward_token(model, bkv, AUDIO, int(toks[n]), S + i)
+                out = forward_token(model, bkv, AUDIO, int(toks[n]), S + i, taps=True)
                 record(n, out, *bkv.own_rows(i, 1))
     elif mode == "memo":
         for n in range(N):
@@ -246,7 +248,7 @@ def vadusa_iteration(model: Model, st: State, template, sp: Sampling, mode: str 
             bkv = st.kv.branch()
             if len(path) > 1:
                 bkv.extend(node_K[:, path[:-1]], node_V[:, path[:-1]])
-            out = forward_token(model, bkv, AUDIO, int(toks[n]), S + len(path) - 1)
+            out = forward_token(model, bkv, AUDIO, int(toks[n]), S + len(path) - 1, taps=True)
             record(n, out, *bkv.own_rows(len(path) - 1, 1))
     elif mode == "tree":
         mask = np.zeros((N, N), dtype=bool)

@@ -69,7 +69,7 @@ EXPORTS = ["vadusa_workspace_bytes", "vadusa_weights_bytes", "vadusa_kv_pool_byt
            "vadusa_begin", "vadusa_prefill", "vadusa_load_state", "vadusa_draft", "vadusa_verify_step",
            "vadusa_accept_and_commit", "vadusa_generate", "vadusa_generate_host", "vadusa_get_lengths",
            "vadusa_check", "vadusa_kernel_launches", "vadusa_profile_begin", "vadusa_profile_end",
-           "vadusa_accept_stats", "vadusa_build_sparse_tree", "vadusa_set_logit_bias",
+           "vadusa_accept_stats", "vadusa_build_sparse_tree", "vadusa_set_logit_bias", "vadusa_set_fused_pass", "vadusa_fused_pass_clusters",
            "vadusa_draft_topk_static", "vadusa_static_scratch_bytes", "vadusa_static_last_error"]
 
 _lib = None
@@ -101,6 +101,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "vadusa_generate_host": (I32, [P, C.POINTER(Sampling), I32, P, P, P, I32, I32, P, P, C.POINTER(Stats)]),
         "vadusa_get_lengths": (I32, [P, P]), "vadusa_check": (I32, [P]),
         "vadusa_kernel_launches": (I64, [P]),
+        "vadusa_set_fused_pass": (I32, [P, I32]),
+        "vadusa_fused_pass_clusters": (I32, [P]),
         "vadusa_draft_topk_static": (I32, [P, P, P, P, I32, I32, I32, I32, I32, I32, I32, P, P]),
         "vadusa_static_scratch_bytes": (I64, []),
         "vadusa_static_last_error": (C.c_char_p, []),
@@ -385,6 +387,12 @@ class Vadusa:
 
     def kernel_launches(self) -> int:
         return int(self.L.vadusa_kernel_launches(self.ctx))
+
+    def set_fused_pass(self, enable: bool):
+        self._ck(self.L.vadusa_set_fused_pass(self.ctx, 1 if enable else 0))
+
+    def fused_pass_clusters(self) -> int:
+        return int(self.L.vadusa_fused_pass_clusters(self.ctx))
 
     def profile_begin(self):
         self._ck(self.L.vadusa_profile_begin(self.ctx))

@@ -15,6 +15,7 @@
 #include "attention_simt.cuh"
 #include "attention_tc.cuh"
 #include "elementwise.cuh"
+#include "fwd_fused.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "gemm_tc2.cuh"
@@ -46,6 +47,8 @@ struct vadusa_ctx {
   int tree_per_seq = 0;
   int max_rank_used = 0;
   int tree_max_depth = 0;
+  int fused_enabled = 1;      // single-sequence passes may run as one persistent kernel
+  int fused_clusters = -1;    // clusters of that kernel that can be resident at once on this device (-1: not asked yet)
   long long ctx_bound = 0;    // host-side upper bound of the longest context (grows by the longest path per commit)
   const int32_t* block_table = nullptr;
   bool have_draft = false, have_verify = false;
@@ -67,10 +70,10 @@ struct vadusa_ctx {
 };
 
 enum KClass { K_EMBED, K_LAYERNORM, K_GEMM_QKV, K_ATTENTION, K_GEMM_OUT, K_GEMM_FFN1, K_GEMM_FFN2, K_GEMM_LM,
-              K_DRAFT_HIDDEN, K_DRAFT_LOGITS, K_DRAFT_SELECT, K_ACCEPT, K_COMMIT, K_MISC, K_NCLASS };
+              K_DRAFT_HIDDEN, K_DRAFT_LOGITS, K_DRAFT_SELECT, K_ACCEPT, K_COMMIT, K_MISC, K_FUSED, K_NCLASS };
 static const char* const kClassName[K_NCLASS] = {
     "tree_embed", "layernorm", "gemm_qkv", "tree_attention", "gemm_out", "gemm_ffn1", "gemm_ffn2", "gemm_lm",
-    "draft_hidden", "draft_logits", "draft_select", "accept", "commit", "misc"};
+    "draft_hidden", "draft_logits", "draft_select", "accept", "commit", "misc", "fused_forward"};
 
 namespace {
 
@@ -496,12 +499,109 @@ vadusa_status layernorm(vadusa_ctx* ctx, const float* x, const float* g, const f
   return VADUSA_OK;
 }
 
+// Can this pass run as the single persistent kernel?  One sequence of at most 64 nodes, bf16, head_dim 64,
+// 8 or 16 heads (a cluster of 8 CTAs per head; K slices of 64 or 128 columns), feed-forward width in whole
+// 128-row blocks per cluster, and a device that holds all clusters at once.
+bool fused_shape_ok(const vadusa_ctx* ctx, const TreeView& tv) {
+  const vadusa_config& c = ctx->cfg;
+  if (!ctx->fused_enabled || c.dtype != 1 || ctx->batch != 1 || tv.n_nodes > 64) return false;
+  const int H = c.n_heads, d = c.d_model, F = c.d_ffn;
+  if (d != 64 * H || (H != 8 && H != 16)) return false;
+  if (F % (128 * H) || F % 512) return false;
+  const int nkc = d / 8 / 64, nrb = F / H / 128, nk2 = F / 8 / 64;
+  if (nrb * nkc > 6 || nk2 > kFfSlots || nrb * 128 > 256) return false;
+  if ((ctx->ctx_bound + 64) / kKvBlock / kFfCluster + 1 > kFfMaxPages) return false;
+  if (c.n_layers > 1) {
+    // the per-layer tensors must repeat at a constant stride (they do in the blob this library lays out)
+    const long long st = find(ctx, "l1.wqkv")->offset - find(ctx, "l0.wqkv")->offset;
+    if (st % 16) return false;
+  }
+  return true;
+}
+
+vadusa_status fused_forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* override_tokens, bf16* attn_tap, bool* launched) {
+  *launched = false;
+  const vadusa_config& c = ctx->cfg;
+  const int H = c.n_heads, d = c.d_model, F = c.d_ffn, L = c.n_layers, M = tv.n_nodes, vp = vpad(&c);
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(kFfCluster * H);
+  lc.blockDim = dim3(kFfThreads);
+  lc.dynamicSmemBytes = kFfSmemBytes;
+  lc.stream = ctx->stream;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = kFfCluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at; lc.numAttrs = 1;
+  if (ctx->fused_clusters < 0) {
+    CU(cudaFuncSetAttribute(fused_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFfSmemBytes));
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, fused_forward_kernel, &lc) != cudaSuccess) { cudaGetLastError(); n = 0; }
+    ctx->fused_clusters = n;
+  }
+  if (ctx->fused_clusters < H) return VADUSA_OK;            // not all clusters fit at once: the caller takes the other path
+  lc.numAttrs = 2;
+  const long long lstride = L > 1 ? find(ctx, "l1.wqkv")->offset - find(ctx, "l0.wqkv")->offset : 0;
+  const LayerW& w0 = ctx->layers[0];
+  const KvGeom g = geom_of(ctx);
+  const CUtensorMap *mqkv, *mwo, *mw1, *mw2, *mlm, *mo, *mmid, *mkv;
+  if (vadusa_status s = tensor_map(ctx, w0.wqkv, 3 * d, d, 64, L, lstride / 2, &mqkv)) return s;
+  if (vadusa_status s = tensor_map(ctx, w0.wo, d, d, 64, L, lstride / 2, &mwo)) return s;
+  if (vadusa_status s = tensor_map(ctx, w0.w1, F, d, 128, L, lstride / 2, &mw1)) return s;
+  if (vadusa_status s = tensor_map(ctx, w0.w2, d, F, 64, L, lstride / 2, &mw2)) return s;
+  if (vadusa_status s = tensor_map(ctx, ctx->lm, vp, d, 128, 1, 0, &mlm)) return s;
+  if (vadusa_status s = tensor_map(ctx, ctx->wsp + ctx->ws.o, M, d, 64, 1, 0, &mo)) return s;
+  if (vadusa_status s = tensor_map(ctx, ctx->wsp + ctx->ws.mid, M, F, 64, 1, 0, &mmid)) return s;
+  const long long rows = (long long)c.kv_num_blocks * 2 * c.n_heads * kKvBlock;
+  if (rows > 0x7fffffffLL) return fail(ctx, VADUSA_EINVAL, "KV pool too large for one tensor map");
+  if (vadusa_status s = tensor_map(ctx, c.kv_pool, (int)rows, 64, 64, c.n_layers, g.layer_stride, &mkv)) return s;
+  FusedArgs a;
+  memset(&a, 0, sizeof(a));
+  a.L = L; a.d = d; a.H = H; a.F = F; a.vocab = c.vocab; a.vpad = vp; a.n_phonemes = c.n_phonemes; a.max_pos = c.max_pos; a.M = M;
+  a.eps = c.ln_eps;
+  a.scale_log2e = (float)(1.0 / sqrt(64.0)) * 1.4426950408889634f;
+  a.ln1_g = w0.ln1_g; a.ln1_b = w0.ln1_b; a.bqkv = w0.bqkv; a.bo = w0.bo; a.ln2_g = w0.ln2_g; a.ln2_b = w0.ln2_b;
+  a.b1 = w0.b1; a.b2 = w0.b2;
+  a.layer_stride = lstride;
+  a.lnf_g = ctx->lnf_g; a.lnf_b = ctx->lnf_b;
+  a.emb_audio = as<bf16>(ctx->emb_audio); a.emb_phon = as<bf16>(ctx->emb_phon); a.pos = as<bf16>(ctx->pos);
+  a.xa = wsptr<float>(ctx, ctx->ws.x); a.xb = wsptr<float>(ctx, ctx->ws.f_xb);
+  a.stats_a = wsptr<float2>(ctx, ctx->ws.f_stats_a); a.stats_b = wsptr<float2>(ctx, ctx->ws.f_stats_b);
+  a.o = wsptr<bf16>(ctx, ctx->ws.o); a.mid = wsptr<bf16>(ctx, ctx->ws.mid); a.hfinal = wsptr<bf16>(ctx, ctx->ws.hfinal);
+  a.logits = wsptr<float>(ctx, ctx->ws.logits);
+  a.attn_tap = attn_tap;
+  a.tokens = wsptr<int32_t>(ctx, ctx->ws.tokens);
+  a.kv_row = wsptr<long long>(ctx, ctx->ws.kv_row);
+  a.override_tokens = override_tokens;
+  a.root = wsptr<int32_t>(ctx, ctx->ws.root); a.topk = wsptr<int32_t>(ctx, ctx->ws.topk);
+  a.n_draft_heads = c.n_draft_heads; a.draft_topk = c.draft_topk;
+  a.ctx_len = wsptr<int32_t>(ctx, ctx->ws.ctx_len); a.nvalid = wsptr<int32_t>(ctx, ctx->ws.nvalid);
+  a.block_table = ctx->block_table;
+  a.tree = tv; a.geom = g;
+  a.kv_pool = reinterpret_cast<bf16*>(c.kv_pool);
+  a.sync = wsptr<uint32_t>(ctx, ctx->ws.f_sync);
+  a.err = err_word(ctx);
+  PROF(ctx, K_FUSED);
+  CU(cudaLaunchKernelEx(&lc, fused_forward_kernel, *mqkv, *mwo, *mw1, *mw2, *mlm, *mo, *mmid, *mkv, a));
+  LAUNCH_CHECK();
+  *launched = true;
+  return VADUSA_OK;
+}
+
 // One forward pass of the base model over batch * tv.n_nodes rows (verify step).
 template <typename T>
 vadusa_status forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* override_tokens, T* attn_tap) {
   const vadusa_config& c = ctx->cfg;
   const int B = ctx->batch, N = tv.n_nodes, M = B * N, d = c.d_model, f = c.d_ffn, vp = vpad(&c);
   const KvGeom g = geom_of(ctx);
+  if constexpr (std::is_same<T, bf16>::value) {
+    if (fused_shape_ok(ctx, tv)) {
+      bool launched = false;
+      if (vadusa_status s = fused_forward(ctx, tv, override_tokens, attn_tap, &launched)) return s;
+      if (launched) return VADUSA_OK;
+    }
+  }
   float* x = wsptr<float>(ctx, ctx->ws.x);
   T* a = wsptr<T>(ctx, ctx->ws.a);
   T* q = wsptr<T>(ctx, ctx->ws.q);
@@ -885,6 +985,7 @@ vadusa_status vadusa_init(const vadusa_weights* weights, const vadusa_config* cf
   CU(cudaMallocHost(&ctx->h_pinned, 4 * sizeof(int32_t)));
   CU(cudaMemsetAsync(ctx->wsp, 0, ctx->ws.tokens, ctx->stream));     // scalars, per-sequence state, trees
   CU(cudaMemsetAsync(ctx->wsp + ctx->ws.acc_stats, 0, 2ull * kStatDepth * kStatTopk * 8, ctx->stream));
+  CU(cudaMemsetAsync(ctx->wsp + ctx->ws.f_sync, 0, 256, ctx->stream));
   // chain-shaped tree used by prefill: node i is the child of node i-1
   constexpr int T = VADUSA_MAX_TREE_NODES;
   static_assert(T == kMaxNodes, "node limit of the kernels");
@@ -982,6 +1083,7 @@ vadusa_status vadusa_begin(vadusa_ctx* ctx, int32_t batch, const int32_t* block_
   ctx->block_table = block_table;
   ctx->have_draft = ctx->have_verify = false;
   CU(cudaMemsetAsync(ctx->wsp + ctx->ws.scalars, 0, 256, ctx->stream));
+  CU(cudaMemsetAsync(ctx->wsp + ctx->ws.f_sync, 0, 256, ctx->stream));
   CU(cudaMemsetAsync(ctx->wsp + ctx->ws.gen_count, 0, batch * 4, ctx->stream));
   ctx->ctx_bound = 0;
   if (h_ctx_len) {
@@ -1073,7 +1175,7 @@ vadusa_status vadusa_verify_step(vadusa_ctx* ctx, const int32_t* tree_tokens_ove
   const int M = ctx->batch * tv.n_nodes;
   const std::string key = KeyBuilder("verify").add(tree_tokens_override).add(logits_out).add(attn_tap).add(hidden_out)
                               .add(ctx->batch).add(ctx->n_nodes).add(ctx->tree_per_seq).add(ctx->block_table)
-                              .add(attention_splits(ctx, ctx->n_nodes)).k;
+                              .add(attention_splits(ctx, ctx->n_nodes)).add(ctx->fused_enabled).k;
   vadusa_status s = run_graphed(ctx, key, [&]() -> vadusa_status {
     vadusa_status s = DISPATCH(forward<float>(ctx, tv, tree_tokens_override, reinterpret_cast<float*>(attn_tap)),
                                forward<bf16>(ctx, tv, tree_tokens_override, reinterpret_cast<bf16*>(attn_tap)));
@@ -1135,7 +1237,7 @@ vadusa_status vadusa_generate(vadusa_ctx* ctx, const vadusa_sampling* sampling, 
       if (ctx->h_pinned[0] >= ctx->batch) break;
     }
     const std::string iter_key = KeyBuilder("iteration").add(sp).add(out_tokens).add(max_new_tokens).add(ctx->batch)
-                                     .add(ctx->n_nodes).add(ctx->block_table).add(attention_splits(ctx, ctx->n_nodes)).k;
+                                     .add(ctx->n_nodes).add(ctx->block_table).add(attention_splits(ctx, ctx->n_nodes)).add(ctx->fused_enabled).k;
     vadusa_status s = run_graphed(ctx, iter_key, [&]() -> vadusa_status {
       vadusa_status s = DISPATCH(draft<float>(ctx, sp), draft<bf16>(ctx, sp));
       if (s) return s;
@@ -1279,6 +1381,14 @@ vadusa_status vadusa_build_sparse_tree(const double* h_prob, int32_t depth, int3
 }
 
 int64_t vadusa_kernel_launches(const vadusa_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int32_t vadusa_fused_pass_clusters(const vadusa_ctx* ctx) { return ctx ? ctx->fused_clusters : -1; }
+
+vadusa_status vadusa_set_fused_pass(vadusa_ctx* ctx, int32_t enable) {
+  if (!ctx) return VADUSA_EINVAL;
+  ctx->fused_enabled = enable ? 1 : 0;
+  return VADUSA_OK;
+}
 
 vadusa_status vadusa_profile_begin(vadusa_ctx* ctx) {
   if (!ctx || !ctx->wsp) return VADUSA_EINVAL;

@@ -83,6 +83,7 @@ class LockstepReport:
     accept_undecidable: int = 0
     max_logit_err: float = 0.0
     max_attn_err: float = 0.0
+    attn_checked: int = 0
     accept_lens: List[int] = field(default_factory=list)
     # acceptance tests by (draft head, rank) on the compared iterations: applied / passed
     tested: np.ndarray = field(default_factory=lambda: np.zeros((15, 16), dtype=np.int64))
@@ -169,7 +170,9 @@ def lockstep(g, table, model, states: Dict[int, "O.State"], template, sp_oracle,
             err = float(np.abs(lg[b] - tr.node_logits).max())
             rep.max_logit_err = max(rep.max_logit_err, err)
             assert err <= tol, f"it {it} seq {b}: logits differ by {err}"
-            if check_attn and tr.attn is not None:
+            if check_attn:
+                assert tr.attn is not None, "the oracle trace carries no attention outputs"
+                rep.attn_checked += 1
                 for l in range(L):
                     e = float(np.abs(at[l, b] - tr.attn[l]).max())
                     rep.max_attn_err = max(rep.max_attn_err, e)
@@ -202,7 +205,8 @@ def lockstep(g, table, model, states: Dict[int, "O.State"], template, sp_oracle,
     print(f"lockstep[{dtype}]: {rep.iterations} iterations, {len(states)} sequences; roots checked {rep.root_checked}, "
           f"draft heads fully checked {rep.draft_heads_checked}/{rep.draft_heads_total} (top-r sets {rep.draft_sets_checked}), "
           f"accept decisions checked {rep.accept_checked} (undecidable {rep.accept_undecidable}); "
-          f"max |logit err| {rep.max_logit_err:.2e}, max |attn err| {rep.max_attn_err:.2e}; "
+          f"max |logit err| {rep.max_logit_err:.2e}, max |attn err| "
+          f"{(format(rep.max_attn_err, '.2e') + ' over ' + str(rep.attn_checked) + ' passes') if rep.attn_checked else 'not checked'}; "
           f"mean accepted {np.mean(rep.accept_lens):.2f}")
     return rep
 
