@@ -253,11 +253,13 @@ int64_t vadusa_kernel_launches(const vadusa_ctx *ctx);                  /* total
  * iteration) runs, for bf16 models with head_dim 64 and 8 or 16 heads, as a single persistent kernel that
  * keeps the whole grid resident and hands activations from step to step through shared memory of thread-block
  * clusters and counters in L2, instead of one kernel per projection.  It computes the same quantities with
- * the same rounding points.  enable = 0 selects the kernel-per-step path for such passes too (used to
- * compare the two); the default is 1.  Host-side switch: takes effect with the next call. */
+ * the same rounding points.  Its clusters (one per head) have 8 CTAs where the device can hold all of them at
+ * once, else 6.  enable = 0 selects the kernel-per-step path for such passes too (used to compare the two);
+ * 1 (the default) lets the library choose; 6 or 8 ask for that cluster size where it fits.  Host-side switch:
+ * takes effect with the next call. */
 vadusa_status vadusa_set_fused_pass(vadusa_ctx *ctx, int32_t enable);
-/* How many of that kernel's clusters (one per head) the device can hold at once, as found when the first
- * such pass was enqueued (-1 before).  The persistent kernel is used only if this is >= n_heads. */
+/* How many of that kernel's clusters (one per head, of the chosen size) the device can hold at once, as found
+ * when the first such pass was enqueued (-1 before).  The persistent kernel is used only if this is >= n_heads. */
 int32_t vadusa_fused_pass_clusters(const vadusa_ctx *ctx);
 
 /* ---- sampler hook (paper Sec. II-C, last paragraph) ----------------------------------------

@@ -388,8 +388,9 @@ class Vadusa:
     def kernel_launches(self) -> int:
         return int(self.L.vadusa_kernel_launches(self.ctx))
 
-    def set_fused_pass(self, enable: bool):
-        self._ck(self.L.vadusa_set_fused_pass(self.ctx, 1 if enable else 0))
+    def set_fused_pass(self, enable):
+        """False / True, or 6 / 8 to ask for that cluster size."""
+        self._ck(self.L.vadusa_set_fused_pass(self.ctx, int(enable)))
 
     def fused_pass_clusters(self) -> int:
         return int(self.L.vadusa_fused_pass_clusters(self.ctx))

@@ -49,6 +49,8 @@ struct vadusa_ctx {
   int tree_max_depth = 0;
   int fused_enabled = 1;      // single-sequence passes may run as one persistent kernel
   int fused_clusters = -1;    // clusters of that kernel that can be resident at once on this device (-1: not asked yet)
+  int fused_cs = -1;          // CTAs per cluster chosen for it (8 or 6; 0: the device cannot hold one cluster per head)
+  int fused_n8 = 0, fused_n6 = 0;
   long long ctx_bound = 0;    // host-side upper bound of the longest context (grows by the longest path per commit)
   const int32_t* block_table = nullptr;
   bool have_draft = false, have_verify = false;
@@ -500,17 +502,15 @@ vadusa_status layernorm(vadusa_ctx* ctx, const float* x, const float* g, const f
 }
 
 // Can this pass run as the single persistent kernel?  One sequence of at most 64 nodes, bf16, head_dim 64,
-// 8 or 16 heads (a cluster of 8 CTAs per head; K slices of 64 or 128 columns), feed-forward width in whole
-// 128-row blocks per cluster, and a device that holds all clusters at once.
+// 8 or 16 heads (one cluster per head), feed-forward width in whole 128-row blocks per cluster (at most two),
+// and a device that holds all clusters at once (asked when the kernel is first wanted).
 bool fused_shape_ok(const vadusa_ctx* ctx, const TreeView& tv) {
   const vadusa_config& c = ctx->cfg;
   if (!ctx->fused_enabled || c.dtype != 1 || ctx->batch != 1 || tv.n_nodes > 64) return false;
   const int H = c.n_heads, d = c.d_model, F = c.d_ffn;
   if (d != 64 * H || (H != 8 && H != 16)) return false;
-  if (F % (128 * H) || F % 512) return false;
-  const int nkc = d / 8 / 64, nrb = F / H / 128, nk2 = F / 8 / 64;
-  if (nrb * nkc > 6 || nk2 > kFfSlots || nrb * 128 > 256) return false;
-  if ((ctx->ctx_bound + 64) / kKvBlock / kFfCluster + 1 > kFfMaxPages) return false;
+  if (F % (128 * H) || F / H > 256) return false;
+  if ((ctx->ctx_bound + 64) / kKvBlock / 6 + 1 > kFfMaxPages) return false;
   if (c.n_layers > 1) {
     // the per-layer tensors must repeat at a constant stride (they do in the blob this library lays out)
     const long long st = find(ctx, "l1.wqkv")->offset - find(ctx, "l0.wqkv")->offset;
@@ -519,43 +519,65 @@ bool fused_shape_ok(const vadusa_ctx* ctx, const TreeView& tv) {
   return true;
 }
 
+template <int CS>
+vadusa_status fused_launch(vadusa_ctx* ctx, bool query_only, int* clusters, const CUtensorMap* const* maps, const FusedArgs* a) {
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(CS * ctx->cfg.n_heads);
+  lc.blockDim = dim3(kFfThreads);
+  lc.dynamicSmemBytes = FfCfg<CS>::kSmemBytes;
+  lc.stream = ctx->stream;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = CS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at;
+  if (query_only) {
+    lc.numAttrs = 1;
+    CU(cudaFuncSetAttribute(fused_forward_kernel<CS>, cudaFuncAttributeMaxDynamicSharedMemorySize, FfCfg<CS>::kSmemBytes));
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, fused_forward_kernel<CS>, &lc) != cudaSuccess) { cudaGetLastError(); n = 0; }
+    *clusters = n;
+    return VADUSA_OK;
+  }
+  lc.numAttrs = 2;
+  PROF(ctx, K_FUSED);
+  CU(cudaLaunchKernelEx(&lc, fused_forward_kernel<CS>, *maps[0], *maps[1], *maps[2], *maps[3], *maps[4], *maps[5], *maps[6], *maps[7], *a));
+  LAUNCH_CHECK();
+  return VADUSA_OK;
+}
+
 vadusa_status fused_forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* override_tokens, bf16* attn_tap, bool* launched) {
   *launched = false;
   const vadusa_config& c = ctx->cfg;
   const int H = c.n_heads, d = c.d_model, F = c.d_ffn, L = c.n_layers, M = tv.n_nodes, vp = vpad(&c);
-  cudaLaunchConfig_t lc = {};
-  lc.gridDim = dim3(kFfCluster * H);
-  lc.blockDim = dim3(kFfThreads);
-  lc.dynamicSmemBytes = kFfSmemBytes;
-  lc.stream = ctx->stream;
-  cudaLaunchAttribute at[2];
-  at[0].id = cudaLaunchAttributeClusterDimension;
-  at[0].val.clusterDim.x = kFfCluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  at[1].val.programmaticStreamSerializationAllowed = 1;
-  lc.attrs = at; lc.numAttrs = 1;
-  if (ctx->fused_clusters < 0) {
-    CU(cudaFuncSetAttribute(fused_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFfSmemBytes));
-    int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, fused_forward_kernel, &lc) != cudaSuccess) { cudaGetLastError(); n = 0; }
-    ctx->fused_clusters = n;
+  if (ctx->fused_cs < 0) {
+    // clusters of 8 where the device holds one per head at once, else clusters of 6
+    int n8 = 0, n6 = 0;
+    if (vadusa_status s = fused_launch<8>(ctx, true, &n8, nullptr, nullptr)) return s;
+    if (vadusa_status s = fused_launch<6>(ctx, true, &n6, nullptr, nullptr)) return s;
+    ctx->fused_cs = n8 >= H ? 8 : n6 >= H ? 6 : 0;
+    ctx->fused_clusters = ctx->fused_cs == 8 ? n8 : n6;
+    ctx->fused_n8 = n8; ctx->fused_n6 = n6;
   }
-  if (ctx->fused_clusters < H) return VADUSA_OK;            // not all clusters fit at once: the caller takes the other path
-  lc.numAttrs = 2;
+  int cs = ctx->fused_cs;
+  if (ctx->fused_enabled == 8 && ctx->fused_n8 >= H) cs = 8;
+  if (ctx->fused_enabled == 6 && ctx->fused_n6 >= H) cs = 6;
+  if (cs == 0) return VADUSA_OK;                            // not all clusters fit at once: the caller takes the other path
   const long long lstride = L > 1 ? find(ctx, "l1.wqkv")->offset - find(ctx, "l0.wqkv")->offset : 0;
   const LayerW& w0 = ctx->layers[0];
   const KvGeom g = geom_of(ctx);
-  const CUtensorMap *mqkv, *mwo, *mw1, *mw2, *mlm, *mo, *mmid, *mkv;
-  if (vadusa_status s = tensor_map(ctx, w0.wqkv, 3 * d, d, 64, L, lstride / 2, &mqkv)) return s;
-  if (vadusa_status s = tensor_map(ctx, w0.wo, d, d, 64, L, lstride / 2, &mwo)) return s;
-  if (vadusa_status s = tensor_map(ctx, w0.w1, F, d, 128, L, lstride / 2, &mw1)) return s;
-  if (vadusa_status s = tensor_map(ctx, w0.w2, d, F, 64, L, lstride / 2, &mw2)) return s;
-  if (vadusa_status s = tensor_map(ctx, ctx->lm, vp, d, 128, 1, 0, &mlm)) return s;
-  if (vadusa_status s = tensor_map(ctx, ctx->wsp + ctx->ws.o, M, d, 64, 1, 0, &mo)) return s;
-  if (vadusa_status s = tensor_map(ctx, ctx->wsp + ctx->ws.mid, M, F, 64, 1, 0, &mmid)) return s;
+  const CUtensorMap* maps[8];
+  if (vadusa_status s = tensor_map(ctx, w0.wqkv, 3 * d, d, 64, L, lstride / 2, &maps[0])) return s;
+  if (vadusa_status s = tensor_map(ctx, w0.wo, d, d, 64, L, lstride / 2, &maps[1])) return s;
+  if (vadusa_status s = tensor_map(ctx, w0.w1, F, d, 128, L, lstride / 2, &maps[2])) return s;
+  if (vadusa_status s = tensor_map(ctx, w0.w2, d, F, 64, L, lstride / 2, &maps[3])) return s;
+  if (vadusa_status s = tensor_map(ctx, ctx->lm, vp, d, 128, 1, 0, &maps[4])) return s;
+  if (vadusa_status s = tensor_map(ctx, ctx->wsp + ctx->ws.o, M, d, 64, 1, 0, &maps[5])) return s;
+  if (vadusa_status s = tensor_map(ctx, ctx->wsp + ctx->ws.mid, M, F, 64, 1, 0, &maps[6])) return s;
   const long long rows = (long long)c.kv_num_blocks * 2 * c.n_heads * kKvBlock;
   if (rows > 0x7fffffffLL) return fail(ctx, VADUSA_EINVAL, "KV pool too large for one tensor map");
-  if (vadusa_status s = tensor_map(ctx, c.kv_pool, (int)rows, 64, 64, c.n_layers, g.layer_stride, &mkv)) return s;
+  if (vadusa_status s = tensor_map(ctx, c.kv_pool, (int)rows, 64, 64, c.n_layers, g.layer_stride, &maps[7])) return s;
   FusedArgs a;
   memset(&a, 0, sizeof(a));
   a.L = L; a.d = d; a.H = H; a.F = F; a.vocab = c.vocab; a.vpad = vp; a.n_phonemes = c.n_phonemes; a.max_pos = c.max_pos; a.M = M;
@@ -582,9 +604,8 @@ vadusa_status fused_forward(vadusa_ctx* ctx, const TreeView& tv, const int32_t* 
   a.kv_pool = reinterpret_cast<bf16*>(c.kv_pool);
   a.sync = wsptr<uint32_t>(ctx, ctx->ws.f_sync);
   a.err = err_word(ctx);
-  PROF(ctx, K_FUSED);
-  CU(cudaLaunchKernelEx(&lc, fused_forward_kernel, *mqkv, *mwo, *mw1, *mw2, *mlm, *mo, *mmid, *mkv, a));
-  LAUNCH_CHECK();
+  vadusa_status s = cs == 8 ? fused_launch<8>(ctx, false, nullptr, maps, &a) : fused_launch<6>(ctx, false, nullptr, maps, &a);
+  if (s) return s;
   *launched = true;
   return VADUSA_OK;
 }
@@ -1386,7 +1407,8 @@ int32_t vadusa_fused_pass_clusters(const vadusa_ctx* ctx) { return ctx ? ctx->fu
 
 vadusa_status vadusa_set_fused_pass(vadusa_ctx* ctx, int32_t enable) {
   if (!ctx) return VADUSA_EINVAL;
-  ctx->fused_enabled = enable ? 1 : 0;
+  if (enable != 0 && enable != 1 && enable != 6 && enable != 8) return fail(ctx, VADUSA_EINVAL, "enable must be 0, 1, 6 or 8");
+  ctx->fused_enabled = enable;
   return VADUSA_OK;
 }
 

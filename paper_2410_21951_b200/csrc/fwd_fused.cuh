@@ -8,14 +8,15 @@
 // dependency chain through a TMA ring, and partial results are exchanged inside thread-block clusters
 // through distributed shared memory.
 //
-// Grid: n_heads clusters of 8 CTAs, one CTA per SM.  Cluster c owns head c (q/k/v rows of head c and its
+// Grid: n_heads clusters of CS CTAs (CS = 8, or 6 where the device cannot hold n_heads clusters of 8 at once),
+// one CTA per SM.  Cluster c owns head c (q/k/v rows of head c and its
 // attention), rows [64c, 64c+64) of the output projection and of the second feed-forward matrix, rows
 // [c F/H, (c+1) F/H) of the first one, and vocabulary tiles c, c+H, ...  Inside a cluster CTA r owns K slice
-// r (an eighth of the inner dimension) of every product and context pages [r per, (r+1) per) of the
-// attention.  Every product is computed as D[token][feature] = X[token][k] W[feature][k]^T with the tokens as
+// r of every product (the 64-column chunks of the inner dimension are dealt out as evenly as CS allows) and
+// context pages [r per, (r+1) per) of the attention.  Every product is computed as D[token][feature] = X[token][k] W[feature][k]^T with the tokens as
 // the MMA's 128-row operand (64 tokens, stored twice where the epilogue is wide) and the CTA's weight rows as
-// the narrow operand.  A product's K-slice partials are summed by the cluster: CTA r receives, from all eight
-// CTAs, the partial rows of tokens 8r..8r+7 in its shared memory, adds them in a fixed order, applies the
+// the narrow operand.  A product's K-slice partials are summed by the cluster: CTA r receives, from all CTAs
+// of the cluster, the partial rows of its share of the tokens in its shared memory, adds them in a fixed order, applies the
 // epilogue (bias, residual, ReLU, LayerNorm statistics) and publishes the result.
 //
 // Exchanges between clusters go through global memory (L2) with monotonic counters: producers store, fence
@@ -31,28 +32,46 @@
 
 namespace vadusa {
 
-constexpr int kFfCluster = 8;                  // CTAs per cluster = K slices of every product
 constexpr int kFfThreads = 192;
 constexpr int kFfWorkers = 128;
-constexpr int kFfSlots = 8;                    // ring slots
-constexpr uint32_t kFfSlotBytes = 16384;
+constexpr uint32_t kFfSlotBytes = 16384;       // ring slot
 constexpr uint32_t kFfTileBytes = 8192;        // 64 rows of 128 bytes
-constexpr uint32_t kFfRingBytes = kFfSlots * kFfSlotBytes;
-constexpr uint32_t kFfXaBytes = 32768;         // LayerNorm operand (two 128-row tiles) / Q tile + tree K and V tiles
-constexpr uint32_t kFfRbBytes = 65536;         // receive buffer of the cluster reductions
 constexpr uint32_t kFfMiscBytes = 1024;
-constexpr int kFfSmemBytes = (int)(kFfRingBytes + kFfXaBytes + kFfRbBytes + kFfMiscBytes + 1024 /*alignment*/);
 constexpr int kFfMaxPages = 32;                // context pages per CTA
 constexpr int kFfGroup = 3;                    // pages per softmax group (three score buffers)
-constexpr int kFfTreeRank = kFfCluster - 1;    // the CTA that also scores the tree nodes' own keys
 constexpr unsigned long long kFfWaitNs = 400ull * 1000 * 1000;
+
+// Shared-memory plan for a cluster of CS CTAs (d_model <= 1024: at most 16 chunks of 64 columns).
+template <int CS> struct FfCfg {
+  static constexpr int kTpo = (64 + CS - 1) / CS;                       // tokens per owner, at most
+  static constexpr int kMaxKc = (16 + CS - 1) / CS;                     // chunks of a CTA's K slice of d_model, at most
+  static constexpr int kSlots = CS >= 8 ? 8 : 6;                        // ring slots
+  static constexpr uint32_t kRingBytes = kSlots * kFfSlotBytes;
+  // LayerNorm operand: one 128-row tile (16 KB) per chunk; also the Q tile + the tree's K and V tiles (32 KB)
+  static constexpr uint32_t kXaBytes = kMaxKc * 16384u < 32768u ? 32768u : kMaxKc * 16384u;
+  static constexpr uint32_t kRbBytes = CS * kTpo * 256 * 4;             // receive buffer of the cluster reductions
+  static constexpr int kSmemBytes = (int)(kRingBytes + kXaBytes + kRbBytes + kFfMiscBytes + 1024 /*alignment*/);
+  static constexpr int kRounds = (kTpo * 16 + kFfWorkers - 1) / kFfWorkers;   // passes of 128 threads over (token, 4 features)
+};
 
 constexpr uint32_t kFfColAcc = 0;              // TMEM columns: product accumulator (up to 256 features)
 constexpr uint32_t kFfColS = 256;              // three score / weight buffers of 64 columns
 constexpr uint32_t kFfColO = 448;              // attention output accumulator
 
-// words of the synchronisation area (uint32)
-constexpr int kFfSyncXa = 0, kFfSyncXb = 1, kFfSyncDone = 2, kFfSyncO = 8, kFfSyncMid = 16, kFfSyncWords = 32;
+// words of the synchronisation area (uint32): two counters, the pass counter, one word per head for the
+// attention outputs and one per cluster for the feed-forward hidden layer
+constexpr int kFfSyncXa = 0, kFfSyncXb = 1, kFfSyncDone = 2, kFfSyncO = 16, kFfSyncMid = 32, kFfSyncWords = 64;
+
+// Items [first, first + count) of `total` dealt to part r of `parts` (the first total % parts parts get one more).
+__host__ __device__ __forceinline__ void ff_split(int total, int parts, int r, int& first, int& count) {
+  const int base = total / parts, rem = total % parts;
+  count = base + (r < rem ? 1 : 0);
+  first = r * base + (r < rem ? r : rem);
+}
+__host__ __device__ __forceinline__ int ff_owner(int item, int total, int parts) {
+  const int base = total / parts, rem = total % parts, edge = rem * (base + 1);
+  return item < edge ? item / (base + 1) : rem + (item - edge) / base;
+}
 
 struct FusedArgs {
   int L, d, H, F, vocab, vpad, n_phonemes, max_pos, M;
@@ -154,6 +173,8 @@ __device__ __forceinline__ uint4 ff_pack8(const float* v) {
   return r;
 }
 
+
+template <int CS>
 __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
     const __grid_constant__ CUtensorMap tmQkv,   // [L][3d][d]    box 64 rows x 64
     const __grid_constant__ CUtensorMap tmWo,    // [L][d][d]     box 64 x 64
@@ -164,13 +185,15 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
     const __grid_constant__ CUtensorMap tmMid,   // [1][M][F]     box 64 x 64
     const __grid_constant__ CUtensorMap tmKV,    // [L][blocks * 2 * H * 64][64]  box 64 x 64
     const FusedArgs a) {
+  using Cfg = FfCfg<CS>;
+  constexpr int R = Cfg::kSlots, TPO = Cfg::kTpo, KCMAX = Cfg::kMaxKc;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_p = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t ring = base, xa = base + kFfRingBytes, rb = xa + kFfXaBytes, bars = rb + kFfRbBytes;
+  const uint32_t ring = base, xa = base + Cfg::kRingBytes, rb = xa + Cfg::kXaBytes, bars = rb + Cfg::kRbBytes;
   uint8_t* ring_p = base_p;
-  float* rb_p = reinterpret_cast<float*>(base_p + kFfRingBytes + kFfXaBytes);
-  uint8_t* misc_p = base_p + kFfRingBytes + kFfXaBytes + kFfRbBytes;
+  float* rb_p = reinterpret_cast<float*>(base_p + Cfg::kRingBytes + Cfg::kXaBytes);
+  uint8_t* misc_p = base_p + Cfg::kRingBytes + Cfg::kXaBytes + Cfg::kRbBytes;
   const uint32_t full0 = bars, empty0 = bars + 64, bar_xa = bars + 128, bar_acc = bars + 136, bar_accfree = bars + 144,
                  bar_s = bars + 152, bar_p = bars + 160, bar_o = bars + 168, bar_qkv = bars + 176,
                  bar_rbfull = bars + 184, bar_rbfree = bars + 192, holder = bars + 200;
@@ -178,25 +201,27 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc_p + 204);
   float2* s_rowstat = reinterpret_cast<float2*>(misc_p + 256);         // [64] (mean, rstd)
   int* s_pageblk = reinterpret_cast<int*>(misc_p + 768);               // [kFfMaxPages] pool row of each of this CTA's pages
-  long long* s_kvrow = reinterpret_cast<long long*>(misc_p + 896);     // [8] K slot of this CTA's tokens (head 0), or -1
+  long long* s_kvrow = reinterpret_cast<long long*>(misc_p + 896);     // [TPO] K slot of this CTA's tokens (head 0), or -1
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const uint32_t rank = cluster_rank();
-  const int c = (int)blockIdx.x / kFfCluster;            // cluster = head
-  const int NC = (int)gridDim.x / kFfCluster;
+  const int rank = (int)cluster_rank();
+  const int c = (int)blockIdx.x / CS;                    // cluster = head
+  const int NC = (int)gridDim.x / CS;
   const int G = (int)gridDim.x;
   const int d = a.d, F = a.F, L = a.L, M = a.M;
-  const int ks_d = d / kFfCluster, nkc = ks_d / 64;      // K slice of the d-wide products, its 64-wide chunks (1 or 2)
-  const int ks_f = F / kFfCluster, nk2 = ks_f / 64;      // the same for the second feed-forward matrix
+  int kc0, nkc, kf0, nk2;                                // this CTA's 64-column chunks of d_model and of the feed-forward width
+  ff_split(d / 64, CS, rank, kc0, nkc);
+  ff_split(F / 64, CS, rank, kf0, nk2);
   const int n1 = F / NC, nrb = n1 / 128;                 // rows of the first feed-forward matrix per cluster, in blocks of 128
   const int nlm = a.vpad / 128;                          // vocabulary tiles
+  const int npair = (nkc + 1) / 2;                       // ring items of a list of nkc 8 KB tiles (two per item)
   uint32_t* err = a.err;
 
   if (tid == 0) {
-    for (int s = 0; s < kFfSlots; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    for (int s = 0; s < R; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
     mbar_init(bar_xa, kFfWorkers); mbar_init(bar_acc, 1); mbar_init(bar_accfree, kFfWorkers);
     mbar_init(bar_s, 1); mbar_init(bar_p, kFfWorkers); mbar_init(bar_o, 1);
-    mbar_init(bar_qkv, 4 * kFfCluster); mbar_init(bar_rbfull, 4 * kFfCluster); mbar_init(bar_rbfree, kFfCluster);
+    mbar_init(bar_qkv, 4 * CS); mbar_init(bar_rbfull, 4 * CS); mbar_init(bar_rbfree, CS);
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmQkv); tma_prefetch_desc(&tmWo); tma_prefetch_desc(&tmW1); tma_prefetch_desc(&tmW2);
@@ -204,7 +229,7 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
   }
   // the operand area starts out finite (rows of it that no one writes are read by MMAs whose results are unused,
   // and as keys / values with zero weight)
-  for (int i = tid; i < (int)(kFfXaBytes / 16); i += kFfThreads) reinterpret_cast<uint4*>(base_p + kFfRingBytes)[i] = make_uint4(0, 0, 0, 0);
+  for (int i = tid; i < (int)(Cfg::kXaBytes / 16); i += kFfThreads) reinterpret_cast<uint4*>(base_p + Cfg::kRingBytes)[i] = make_uint4(0, 0, 0, 0);
   if (warp == 1) { tmem_alloc(holder, 512); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
@@ -212,22 +237,32 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
   tc_fence_after();
   const uint32_t tmem = *holder_ptr;
 
-  // per-layer ring items, in issue order (the same arithmetic in every role)
-  //   [0, nkc)            q|k rows of chunk kc          [nkc]        v rows, all chunks
-  //   offKV + i           context page i (K tile | V tile)
-  //   offOutW             output-projection rows, all chunks
-  //   offF1 + rb*nkc + kc rows 128 rb .. of the first feed-forward matrix, chunk kc
-  //   offOutX             attention output (tokens), all chunks           (waits for the heads of this K slice)
-  //   offF2 + j           chunk j of: hidden activations (tokens) | rows of the second feed-forward matrix
+  // Per-layer ring items, numbered in issue order (the same arithmetic in every role):
+  //   offQK + kc       q rows | k rows of head c, chunk kc
+  //   offV + kc/2      v rows, chunks kc (two tiles per item)
+  //   offKV + i        context page i of this CTA (K tile | V tile)
+  //   offOutW + kc/2   output-projection rows [64c, 64c+64), chunks kc
+  //   offOutX + kc/2   attention output (tokens), chunks kc; waits for the heads that make those columns
+  //   offF1 + rb*nkc + kc   rows 128 rb .. of the first feed-forward matrix, chunk kc
+  //   offF2 + j        chunk j of: hidden activations (tokens) | rows of the second feed-forward matrix
+  // The first feed-forward matrix is issued ahead of the (gated) attention output when the ring has room for both.
   int ctx = 0, nv = 0, np_mine = 0, p0 = 0;
+  int offV = 0, offKV = 0, offOutW = 0, offOutX = 0, offF1 = 0, offF2 = 0, ipl = 0;
+  bool f1_first = false;
   auto plan = [&]() {                           // after griddepcontrol.wait
     ctx = a.ctx_len[0]; nv = a.nvalid[0];
     const int npages = nv > 0 ? (ctx + kKvBlock - 1) / kKvBlock : 0;
-    const int per = (npages + kFfCluster - 1) / kFfCluster;
-    p0 = (int)rank * per;
+    const int per = (npages + CS - 1) / CS;
+    p0 = rank * per;
     const int p1 = min(npages, p0 + per);
     np_mine = max(0, p1 - p0);
     if (np_mine > kFfMaxPages) { np_mine = kFfMaxPages; atomicOr(err, kErrCapacity); }
+    const int nf1 = nrb * nkc;
+    offV = nkc; offKV = offV + npair; offOutW = offKV + np_mine;
+    f1_first = npair + nf1 + npair - 1 < R;
+    if (f1_first) { offF1 = offOutW + npair; offOutX = offF1 + nf1; offF2 = offOutX + npair; }
+    else { offOutX = offOutW + npair; offF1 = offOutX + npair; offF2 = offF1 + nf1; }
+    ipl = offF2 + nk2;
   };
   const bool lm_mine = c < nlm;
 
@@ -241,77 +276,78 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
     }
     __syncwarp();
     if (lane == 0) {
-      const int offKV = nkc + 1, offOutW = offKV + np_mine, offF1 = offOutW + 1, offOutX = offF1 + nrb * nkc, offF2 = offOutX + 1;
-      const int ipl = offF2 + nk2;
-      const int kd0 = (int)rank * ks_d, kf0 = (int)rank * ks_f;
       bool ok = true;
       // slot of item `seq`: waits until the item that used it before has been consumed; arms the barrier
       auto acquire = [&](int seq, uint32_t bytes) -> uint32_t {
-        const int s = seq % kFfSlots;
-        if (seq >= kFfSlots)
-          ok = ok && ff_wait([&] { return mbar_try_wait(empty0 + 8 * s, ((seq / kFfSlots) - 1) & 1); }, err, abort_flag);
+        const int s = seq % R;
+        if (seq >= R)
+          ok = ok && ff_wait([&] { return mbar_try_wait(empty0 + 8 * s, ((seq / R) - 1) & 1); }, err, abort_flag);
         if (ok) mbar_expect_tx(full0 + 8 * s, bytes);
         return ring + s * kFfSlotBytes;
       };
-      auto gate = [&](const uint32_t* word, uint32_t target) {
-        ok = ok && ff_wait([&] { return ff_ld_acquire(word) >= target; }, err, abort_flag);
-        ff_fence_proxy_global();
+      auto fullbar = [&](int seq) -> uint32_t { return full0 + 8 * (seq % R); };
+      auto gate = [&](int word, uint32_t target) {
+        ok = ok && ff_wait([&] { return ff_ld_acquire(a.sync + word) >= target; }, err, abort_flag);
+      };
+      // a list of nkc tiles (64 rows x chunk kc of `map` at row `row`), two per item
+      auto issue_pairs = [&](int seq0, const CUtensorMap* map, int row, int z) {
+        for (int i = 0; i < npair && ok; ++i) {
+          const int nt = min(2, nkc - 2 * i);
+          const uint32_t dst = acquire(seq0 + i, nt * kFfTileBytes);
+          if (!ok) break;
+          for (int t = 0; t < nt; ++t) tma_load_3d(dst + t * kFfTileBytes, map, fullbar(seq0 + i), 64 * (kc0 + 2 * i + t), row, z);
+        }
       };
       for (int l = 0; l < L && ok; ++l) {
         const int b0 = l * ipl;
         for (int kc = 0; kc < nkc && ok; ++kc) {
           const uint32_t dst = acquire(b0 + kc, 2 * kFfTileBytes);
           if (!ok) break;
-          const uint32_t fb = full0 + 8 * ((b0 + kc) % kFfSlots);
-          tma_load_3d(dst, &tmQkv, fb, kd0 + 64 * kc, c * 64, l);
-          tma_load_3d(dst + kFfTileBytes, &tmQkv, fb, kd0 + 64 * kc, d + c * 64, l);
+          tma_load_3d(dst, &tmQkv, fullbar(b0 + kc), 64 * (kc0 + kc), c * 64, l);
+          tma_load_3d(dst + kFfTileBytes, &tmQkv, fullbar(b0 + kc), 64 * (kc0 + kc), d + c * 64, l);
         }
-        if (ok) {
-          const uint32_t dst = acquire(b0 + nkc, nkc * kFfTileBytes);
-          if (ok) {
-            const uint32_t fb = full0 + 8 * ((b0 + nkc) % kFfSlots);
-            for (int kc = 0; kc < nkc; ++kc) tma_load_3d(dst + kc * kFfTileBytes, &tmQkv, fb, kd0 + 64 * kc, 2 * d + c * 64, l);
-          }
-        }
+        issue_pairs(b0 + offV, &tmQkv, 2 * d + c * 64, l);
         for (int i = 0; i < np_mine && ok; ++i) {
           const uint32_t dst = acquire(b0 + offKV + i, 2 * kFfTileBytes);
           if (!ok) break;
-          const uint32_t fb = full0 + 8 * ((b0 + offKV + i) % kFfSlots);
-          tma_load_3d(dst, &tmKV, fb, 0, s_pageblk[i], l);
-          tma_load_3d(dst + kFfTileBytes, &tmKV, fb, 0, s_pageblk[i] + a.geom.n_heads * kKvBlock, l);
+          tma_load_3d(dst, &tmKV, fullbar(b0 + offKV + i), 0, s_pageblk[i], l);
+          tma_load_3d(dst + kFfTileBytes, &tmKV, fullbar(b0 + offKV + i), 0, s_pageblk[i] + a.geom.n_heads * kKvBlock, l);
         }
-        if (ok) {
-          const uint32_t dst = acquire(b0 + offOutW, nkc * kFfTileBytes);
-          if (ok) {
-            const uint32_t fb = full0 + 8 * ((b0 + offOutW) % kFfSlots);
-            for (int kc = 0; kc < nkc; ++kc) tma_load_3d(dst + kc * kFfTileBytes, &tmWo, fb, kd0 + 64 * kc, c * 64, l);
+        issue_pairs(b0 + offOutW, &tmWo, c * 64, l);
+        auto issue_f1 = [&]() {
+          for (int i = 0; i < nrb * nkc && ok; ++i) {
+            const uint32_t dst = acquire(b0 + offF1 + i, 2 * kFfTileBytes);
+            if (!ok) break;
+            tma_load_3d(dst, &tmW1, fullbar(b0 + offF1 + i), 64 * (kc0 + i % nkc), c * n1 + 128 * (i / nkc), l);
           }
-        }
-        for (int i = 0; i < nrb * nkc && ok; ++i) {
-          const uint32_t dst = acquire(b0 + offF1 + i, 2 * kFfTileBytes);
-          if (!ok) break;
-          tma_load_3d(dst, &tmW1, full0 + 8 * ((b0 + offF1 + i) % kFfSlots), kd0 + 64 * (i % nkc), c * n1 + 128 * (i / nkc), l);
-        }
-        if (ok) {
-          const uint32_t dst = acquire(b0 + offOutX, nkc * kFfTileBytes);
-          if (ok) {
-            gate(a.sync + kFfSyncO + rank, (uint32_t)((NC / kFfCluster) * kFfCluster * (l + 1)));
-            if (ok) {
-              const uint32_t fb = full0 + 8 * ((b0 + offOutX) % kFfSlots);
-              for (int kc = 0; kc < nkc; ++kc) tma_load_3d(dst + kc * kFfTileBytes, &tmO, fb, kd0 + 64 * kc, 0, 0);
-            }
-          }
-        }
-        // second feed-forward matrix: all weight tiles first (they stream while the hidden layer is computed),
-        // then the hidden activations once every cluster that makes this K slice has published them
-        for (int j = 0; j < nk2 && ok; ++j) {
+        };
+        auto issue_outx = [&]() {
+          // every head whose 64 output columns lie in this K slice has published them
+          for (int kc = 0; kc < nkc; ++kc) gate(kFfSyncO + kc0 + kc, (uint32_t)(CS * (l + 1)));
+          ff_fence_proxy_global();
+          issue_pairs(b0 + offOutX, &tmO, 0, 0);
+        };
+        if (f1_first) { issue_f1(); issue_outx(); } else { issue_outx(); issue_f1(); }
+        // second feed-forward matrix: weight tiles first, as far as the ring goes (they stream while the hidden
+        // layer is computed), then the hidden activations once every cluster that makes this K slice has
+        // published them; the rest in pairs as slots come free
+        const int nw = min(nk2, R);
+        for (int j = 0; j < nw && ok; ++j) {
           const uint32_t dst = acquire(b0 + offF2 + j, 2 * kFfTileBytes);
           if (!ok) break;
-          tma_load_3d(dst + kFfTileBytes, &tmW2, full0 + 8 * ((b0 + offF2 + j) % kFfSlots), kf0 + 64 * j, c * 64, l);
+          tma_load_3d(dst + kFfTileBytes, &tmW2, fullbar(b0 + offF2 + j), 64 * (kf0 + j), c * 64, l);
         }
-        if (ok) gate(a.sync + kFfSyncMid + rank, (uint32_t)((NC / kFfCluster) * kFfCluster * (l + 1)));
-        for (int j = 0; j < nk2 && ok; ++j)
-          tma_load_3d(ring + ((b0 + offF2 + j) % kFfSlots) * kFfSlotBytes, &tmMid, full0 + 8 * ((b0 + offF2 + j) % kFfSlots), kf0 + 64 * j, 0, 0);
+        if (nk2 > 0)
+          for (int cc = (64 * kf0) / n1; cc <= (64 * (kf0 + nk2) - 1) / n1; ++cc) gate(kFfSyncMid + cc, (uint32_t)(CS * (l + 1)));
+        ff_fence_proxy_global();
+        for (int j = 0; j < nw && ok; ++j)
+          tma_load_3d(ring + ((b0 + offF2 + j) % R) * kFfSlotBytes, &tmMid, fullbar(b0 + offF2 + j), 64 * (kf0 + j), 0, 0);
+        for (int j = nw; j < nk2 && ok; ++j) {
+          const uint32_t dst = acquire(b0 + offF2 + j, 2 * kFfTileBytes);
+          if (!ok) break;
+          tma_load_3d(dst + kFfTileBytes, &tmW2, fullbar(b0 + offF2 + j), 64 * (kf0 + j), c * 64, l);
+          tma_load_3d(dst, &tmMid, fullbar(b0 + offF2 + j), 64 * (kf0 + j), 0, 0);
+        }
       }
       if (lm_mine) {
         int seq = L * ipl;
@@ -319,29 +355,28 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
           for (int kc = 0; kc < nkc && ok; ++kc, ++seq) {
             const uint32_t dst = acquire(seq, 2 * kFfTileBytes);
             if (!ok) break;
-            tma_load_3d(dst, &tmLm, full0 + 8 * (seq % kFfSlots), kd0 + 64 * kc, 128 * t, 0);
+            tma_load_3d(dst, &tmLm, fullbar(seq), 64 * (kc0 + kc), 128 * t, 0);
           }
       }
     }
-  } else if (warp == 1) {
+  }
+  else if (warp == 1) {
     // =========================================================== MMA issuer
     grid_dep_wait();
     plan();
     if (lane == 0) {
-      const int offKV = nkc + 1, offOutW = offKV + np_mine, offF1 = offOutW + 1, offOutX = offF1 + nrb * nkc, offF2 = offOutX + 1;
-      const int ipl = offF2 + nk2;
       constexpr uint32_t id128 = umma_idesc_bf16(128, 128), id64 = umma_idesc_bf16(128, 64);
       constexpr uint32_t id_pv = umma_idesc_bf16(128, 64) | (1u << 16);        // B (V tile) is MN-major
       const uint32_t acc = tmem + kFfColAcc;
       bool ok = true;
-      uint32_t n_xa = 0, n_accfree = 0, n_p = 0;
+      uint32_t n_xa = 0, n_accfree = 0, n_p = 0, n_qkv = 0;
       bool first_acc = true;
       auto wait_full = [&](int seq) -> uint32_t {
-        const int s = seq % kFfSlots;
-        ok = ok && ff_wait([&] { return mbar_try_wait(full0 + 8 * s, (seq / kFfSlots) & 1); }, err, abort_flag);
+        const int s = seq % R;
+        ok = ok && ff_wait([&] { return mbar_try_wait(full0 + 8 * s, (seq / R) & 1); }, err, abort_flag);
         return ring + s * kFfSlotBytes;
       };
-      auto release = [&](int seq) { umma_commit(empty0 + 8 * (seq % kFfSlots)); };
+      auto release = [&](int seq) { umma_commit(empty0 + 8 * (seq % R)); };
       auto wait_local = [&](uint32_t bar, uint32_t& n) {
         ok = ok && ff_wait([&] { return mbar_try_wait(bar, n & 1); }, err, abort_flag);
         ++n;
@@ -352,8 +387,13 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
         first_acc = false;
         tc_fence_after();
       };
-      const int ntile = np_mine + ((rank == kFfTreeRank && nv > 0) ? 1 : 0);
-      uint32_t n_qkv = 0;
+      // four K steps of 16: D (+)= A[128 x 64] B[N x 64]^T
+      auto mma4 = [&](uint32_t dcol, uint32_t a_addr, uint32_t b_addr, uint32_t idesc, bool accumulate) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          umma_bf16(dcol, umma_desc_k_sw128(a_addr + 32 * k), umma_desc_k_sw128(b_addr + 32 * k), idesc, accumulate || k != 0);
+      };
+      const int ntile = np_mine + ((rank == CS - 1 && nv > 0) ? 1 : 0);
       for (int l = 0; l < L && ok; ++l) {
         const int b0 = l * ipl;
         // ---- q/k/v: D[:, 0:64) = q, [64:128) = k, [128:192) = v
@@ -364,24 +404,19 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
           const uint32_t w = wait_full(b0 + kc);
           if (!ok) break;
           tc_fence_after();
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
-            umma_bf16(acc, umma_desc_k_sw128(xa + kc * 16384 + 32 * k), umma_desc_k_sw128(w + 32 * k), id128, (kc | k) != 0);
+          mma4(acc, xa + kc * 16384, w, id128, kc != 0);
           release(b0 + kc);
         }
-        if (ok) {
-          const uint32_t w = wait_full(b0 + nkc);
-          if (ok) {
-            tc_fence_after();
-            for (int kc = 0; kc < nkc; ++kc)
-#pragma unroll
-              for (int k = 0; k < 4; ++k)
-                umma_bf16(acc + 128, umma_desc_k_sw128(xa + kc * 16384 + 32 * k), umma_desc_k_sw128(w + kc * kFfTileBytes + 32 * k), id64, (kc | k) != 0);
-            release(b0 + nkc);
-            umma_commit(bar_acc);
-          }
+        for (int kc = 0; kc < nkc && ok; ++kc) {
+          const uint32_t w = wait_full(b0 + offV + kc / 2);
+          if (!ok) break;
+          tc_fence_after();
+          mma4(acc + 128, xa + kc * 16384, w + (kc & 1) * kFfTileBytes, id64, kc != 0);
+          if ((kc & 1) || kc == nkc - 1) release(b0 + offV + kc / 2);
         }
-        // ---- attention of head c over this CTA's pages (and the tree's own keys in one CTA)
+        if (!ok) break;
+        umma_commit(bar_acc);
+        // ---- attention of head c over this CTA's pages (and the tree's own keys in the last CTA)
         ok = ok && ff_wait([&] { return ff_try_wait_cluster(bar_qkv, n_qkv & 1); }, err, abort_flag);
         ++n_qkv;
         ff_fence_proxy_all();
@@ -393,9 +428,7 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
             const uint32_t ka = t < np_mine ? wait_full(b0 + offKV + t) : xa + 16384;
             if (!ok) break;
             tc_fence_after();
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma_bf16(tmem + kFfColS + 64 * pi, umma_desc_k_sw128(xa + 32 * k), umma_desc_k_sw128(ka + 32 * k), id64, k != 0);
+            mma4(tmem + kFfColS + 64 * pi, xa, ka, id64, false);
           }
           if (!ok) break;
           umma_commit(bar_s);
@@ -404,7 +437,7 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
           tc_fence_after();
           for (int pi = 0; pi < npg; ++pi) {
             const int t = t0 + pi;
-            const uint32_t va = t < np_mine ? ring + ((b0 + offKV + t) % kFfSlots) * kFfSlotBytes + kFfTileBytes : xa + 24576;
+            const uint32_t va = t < np_mine ? ring + ((b0 + offKV + t) % R) * kFfSlotBytes + kFfTileBytes : xa + 24576;
             const uint32_t pa = tmem + kFfColS + 64 * pi;
 #pragma unroll
             for (int k = 0; k < 4; ++k)
@@ -419,19 +452,16 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
         if (!ok) break;
         // ---- output projection
         acc_begin();
-        {
-          const uint32_t w = wait_full(b0 + offOutW);
-          const uint32_t x = wait_full(b0 + offOutX);
+        for (int kc = 0; kc < nkc && ok; ++kc) {
+          const uint32_t w = wait_full(b0 + offOutW + kc / 2);
+          const uint32_t x = wait_full(b0 + offOutX + kc / 2);
           if (!ok) break;
           tc_fence_after();
-          for (int kc = 0; kc < nkc; ++kc)
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma_bf16(acc, umma_desc_k_sw128(x + kc * kFfTileBytes + 32 * k), umma_desc_k_sw128(w + kc * kFfTileBytes + 32 * k), id64, (kc | k) != 0);
-          release(b0 + offOutW);
-          release(b0 + offOutX);
-          umma_commit(bar_acc);
+          mma4(acc, x + (kc & 1) * kFfTileBytes, w + (kc & 1) * kFfTileBytes, id64, kc != 0);
+          if ((kc & 1) || kc == nkc - 1) { release(b0 + offOutW + kc / 2); release(b0 + offOutX + kc / 2); }
         }
+        if (!ok) break;
+        umma_commit(bar_acc);
         // ---- first feed-forward matrix
         acc_begin();
         wait_local(bar_xa, n_xa);
@@ -441,9 +471,7 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
           if (!ok) break;
           tc_fence_after();
           const int kc = i % nkc, rbk = i / nkc;
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
-            umma_bf16(acc + 128 * rbk, umma_desc_k_sw128(xa + kc * 16384 + 32 * k), umma_desc_k_sw128(w + 32 * k), id128, (kc | k) != 0);
+          mma4(acc + 128 * rbk, xa + kc * 16384, w, id128, kc != 0);
           release(b0 + offF1 + i);
         }
         if (!ok) break;
@@ -454,9 +482,7 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
           const uint32_t s = wait_full(b0 + offF2 + j);
           if (!ok) break;
           tc_fence_after();
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
-            umma_bf16(acc, umma_desc_k_sw128(s + 32 * k), umma_desc_k_sw128(s + kFfTileBytes + 32 * k), id64, (j | k) != 0);
+          mma4(acc, s, s + kFfTileBytes, id64, j != 0);
           release(b0 + offF2 + j);
         }
         if (!ok) break;
@@ -473,26 +499,28 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
             const uint32_t w = wait_full(seq);
             if (!ok) break;
             tc_fence_after();
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma_bf16(acc, umma_desc_k_sw128(xa + kc * 16384 + 32 * k), umma_desc_k_sw128(w + 32 * k), id128, (kc | k) != 0);
+            mma4(acc, xa + kc * 16384, w, id128, kc != 0);
             release(seq);
           }
           if (ok) umma_commit(bar_acc);
         }
       }
     }
-  } else {
+  }
+  else {
     // =========================================================== workers (128 threads)
     const int wtid = tid - 64, ww = warp - 2, wq = warp & 3;
     const int lane_t = 32 * wq + lane;                       // this thread's TMEM lane
     const int tok_t = lane_t & 63, half_t = lane_t >> 6;     // token of the lane, which copy of it
-    const uint32_t owner_t = (uint32_t)(tok_t >> 3);
-    const int tl_t = tok_t & 7;
+    const int owner_t = ff_owner(tok_t, 64, CS);             // the CTA that sums this token's partial rows
+    int own_first_t, own_cnt_t;
+    ff_split(64, CS, owner_t, own_first_t, own_cnt_t);
+    const int tl_t = tok_t - own_first_t;
+    int tok0, ntok;                                          // the tokens this CTA owns
+    ff_split(64, CS, rank, tok0, ntok);
     const uint32_t trow = tmem + ((uint32_t)(32 * wq) << 16);
-    const uint32_t rb_owner = ff_mapa(rb, owner_t);
+    const uint32_t rb_owner = ff_mapa(rb, (uint32_t)owner_t);
     uint32_t n_acc = 0, n_rb = 0, n_s = 0, n_o = 0;
-    const int kd0 = (int)rank * ks_d;
     const long long kv_stride = (long long)a.geom.n_heads * kKvBlock * a.geom.head_dim;   // K row -> V row of a head
     const int tile_elems = kKvBlock * a.geom.head_dim;
 
@@ -518,7 +546,7 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
       ff_fence_cluster();
       __syncwarp();
       if (lane == 0)
-        for (uint32_t p = 0; p < (uint32_t)kFfCluster; ++p) ff_arrive_remote(ff_mapa(bar_rbfull, p));
+        for (uint32_t p = 0; p < (uint32_t)CS; ++p) ff_arrive_remote(ff_mapa(bar_rbfull, p));
     };
     auto rb_wait = [&]() {
       ff_wait([&] { return ff_try_wait_cluster(bar_rbfull, n_rb & 1); }, err, abort_flag);
@@ -526,19 +554,19 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
     auto rb_done = [&]() {                                   // after this CTA's reads of its receive buffer
       ff_workers_sync();
       if (wtid == 0)
-        for (uint32_t p = 0; p < (uint32_t)kFfCluster; ++p) ff_arrive_remote(ff_mapa(bar_rbfree, p));
+        for (uint32_t p = 0; p < (uint32_t)CS; ++p) ff_arrive_remote(ff_mapa(bar_rbfree, p));
       ++n_rb;
     };
-    // K-slice partial D[token][0:N) of this CTA -> the owners of the tokens.  dup: tokens are stored twice in the
-    // operand, the second copy's lanes send the upper half of the columns; else lanes 0..63 send everything.
+    // K-slice partial D[token][0:N) of this CTA -> the owners of the tokens (receive buffer: [source][token][N]).
+    // dup: tokens are stored twice in the operand, the second copy's lanes send the upper half of the columns;
+    // else lanes 0..63 send everything.
     auto send_partial = [&](int N, bool dup) {
       wait_bar(bar_acc, n_acc);
       tc_fence_after();
       rb_begin();
       const int ncol = dup ? N / 2 : (half_t == 0 ? N : 0), col0 = dup ? half_t * (N / 2) : 0;
-      const uint32_t dst = rb_owner + (uint32_t)(((int)rank * 8 + tl_t) * N + col0) * 4u;
-      const int ncol_w = __shfl_sync(0xffffffffu, ncol, 0);          // uniform in a warp
-      for (int c0 = 0; c0 < ncol_w; c0 += 32) {
+      const uint32_t dst = rb_owner + (uint32_t)((rank * TPO + tl_t) * N + col0) * 4u;
+      for (int c0 = 0; c0 < ncol; c0 += 32) {                // (ncol is the same in all lanes of a warp)
         float v[32];
         tmem_ld32(trow + kFfColAcc + col0 + c0, v);
 #pragma unroll
@@ -548,34 +576,34 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
       tc_fence_before();
       mbar_arrive(bar_accfree);
     };
-    // Sum over the eight sources of four consecutive columns of one of this CTA's tokens.
+    // Sum over the sources of four consecutive columns of one of this CTA's tokens (fixed order).
     auto rb_sum4 = [&](int N, int tl, int col) -> float4 {
       float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-      for (int src = 0; src < kFfCluster; ++src) {
-        const float4 v = *reinterpret_cast<const float4*>(rb_p + (src * 8 + tl) * N + col);
+      for (int src = 0; src < CS; ++src) {
+        const float4 v = *reinterpret_cast<const float4*>(rb_p + (src * TPO + tl) * N + col);
         s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
       }
       return s;
     };
-    // LayerNorm of the K slice [kd0, kd0 + ks_d) of rows x[0:M) into the operand tiles (each row stored at r and r + 64).
-    // Waits for `word` >= target first.  y: where to also store the normalised slice (or null).
+    // LayerNorm of this CTA's K-slice columns of rows x[0:M) into the operand tiles (each row stored at r and
+    // r + 64).  Waits for `word` >= target first.  y: where to also store the normalised slice (or null).
     auto build_ln = [&](const float* x, const float2* stats, const float* g, const float* bta, int word, uint32_t target, bf16* y) {
-      float4 gg[2], bb[2];
+      float4 gg[KCMAX], bb[KCMAX];
 #pragma unroll
-      for (int kc = 0; kc < 2; ++kc)
+      for (int kc = 0; kc < KCMAX; ++kc)
         if (kc < nkc) {
-          gg[kc] = __ldg(reinterpret_cast<const float4*>(g + kd0 + 64 * kc + 4 * (lane & 15)));
-          bb[kc] = __ldg(reinterpret_cast<const float4*>(bta + kd0 + 64 * kc + 4 * (lane & 15)));
+          gg[kc] = __ldg(reinterpret_cast<const float4*>(g + 64 * (kc0 + kc) + 4 * (lane & 15)));
+          bb[kc] = __ldg(reinterpret_cast<const float4*>(bta + 64 * (kc0 + kc) + 4 * (lane & 15)));
         }
       wait_counter(word, target);
-      float4 xv[16];
+      float4 xv[KCMAX * 8];
 #pragma unroll
-      for (int kc = 0; kc < 2; ++kc)
+      for (int kc = 0; kc < KCMAX; ++kc)
 #pragma unroll
         for (int it = 0; it < 8; ++it) {
           const int row = ww * 16 + it * 2 + (lane >> 4);
-          xv[kc * 8 + it] = (kc < nkc && row < M) ? __ldcg(reinterpret_cast<const float4*>(x + (long long)row * d + kd0 + 64 * kc + 4 * (lane & 15)))
+          xv[kc * 8 + it] = (kc < nkc && row < M) ? __ldcg(reinterpret_cast<const float4*>(x + (long long)row * d + 64 * (kc0 + kc) + 4 * (lane & 15)))
                                                    : make_float4(0.f, 0.f, 0.f, 0.f);
         }
       // row statistics from the groups of 64 features: two threads per row, NC / 2 groups each
@@ -597,7 +625,7 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
       if (part == 0) s_rowstat[srow] = make_float2(mean, rsqrtf(m2 / (float)d + a.eps));
       ff_workers_sync();
 #pragma unroll
-      for (int kc = 0; kc < 2; ++kc)
+      for (int kc = 0; kc < KCMAX; ++kc)
         if (kc < nkc) {
 #pragma unroll
           for (int it = 0; it < 8; ++it) {
@@ -614,89 +642,103 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
             asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(ad), "r"(lo), "r"(hi) : "memory");
             asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(ad + 8192u), "r"(lo), "r"(hi) : "memory");
             if (y != nullptr && row < M)
-              *reinterpret_cast<uint2*>(y + (long long)row * d + kd0 + 64 * kc + 4 * (lane & 15)) = make_uint2(lo, hi);
+              *reinterpret_cast<uint2*>(y + (long long)row * d + 64 * (kc0 + kc) + 4 * (lane & 15)) = make_uint2(lo, hi);
           }
         }
       fence_proxy_async_smem();
       mbar_arrive(bar_xa);
     };
-    // Residual epilogue of a product whose cluster owns features [64c, 64c+64): thread = (token wtid/16, four
-    // features); xres (this thread's four values of the residual stream, which it also wrote last time) +=
-    // sum + bias; leaves the (mean, sum of squared deviations) of the 64 features.
-    float4 xres = make_float4(0.f, 0.f, 0.f, 0.f);
-    auto residual_epilogue = [&](const float* bias, float* xout, float2* stats_out) {
-      const int tl = wtid >> 4, f4 = (wtid & 15) * 4, m = 8 * (int)rank + tl, col = 64 * c + f4;
-      const float4 bv = __ldg(reinterpret_cast<const float4*>(bias + col));
-      rb_wait();
-      const float4 s = rb_sum4(64, tl, f4);
-      const float4 v = make_float4(xres.x + (s.x + bv.x), xres.y + (s.y + bv.y), xres.z + (s.z + bv.z), xres.w + (s.w + bv.w));
-      xres = v;
-      if (m < M) *reinterpret_cast<float4*>(xout + (long long)m * d + col) = v;
+    // Mean and sum of squared deviations of 64 features held four per thread by 16 consecutive lanes.
+    auto group_stats = [&](const float4& v, float& mu, float& q) {
       float sm = (v.x + v.y) + (v.z + v.w);
 #pragma unroll
       for (int o = 8; o > 0; o >>= 1) sm += __shfl_xor_sync(0xffffffffu, sm, o);
-      const float mu = sm * (1.0f / 64.0f);
+      mu = sm * (1.0f / 64.0f);
       const float d0 = v.x - mu, d1 = v.y - mu, d2 = v.z - mu, d3 = v.w - mu;
-      float q = (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
+      q = (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
 #pragma unroll
       for (int o = 8; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
-      if ((wtid & 15) == 0 && m < M) stats_out[(long long)m * NC + c] = make_float2(mu, q);
+    };
+    // Residual epilogue of a product whose cluster owns features [64c, 64c+64): item = (token, four features);
+    // xres (the item's four values of the residual stream, which this thread also wrote last time) += sum + bias;
+    // leaves the (mean, sum of squared deviations) of the 64 features.
+    float4 xres[Cfg::kRounds];
+#pragma unroll
+    for (int rd = 0; rd < Cfg::kRounds; ++rd) xres[rd] = make_float4(0.f, 0.f, 0.f, 0.f);
+    auto residual_epilogue = [&](const float* bias, float* xout, float2* stats_out) {
+      const int f4 = (wtid & 15) * 4, col = 64 * c + f4;
+      const float4 bv = __ldg(reinterpret_cast<const float4*>(bias + col));
+      rb_wait();
+#pragma unroll
+      for (int rd = 0; rd < Cfg::kRounds; ++rd) {
+        const int tl = (wtid >> 4) + 8 * rd, m = tok0 + tl;
+        const bool mine = tl < ntok;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (mine) {
+          const float4 s = rb_sum4(64, tl, f4);
+          v = make_float4(xres[rd].x + (s.x + bv.x), xres[rd].y + (s.y + bv.y), xres[rd].z + (s.z + bv.z), xres[rd].w + (s.w + bv.w));
+          xres[rd] = v;
+          if (m < M) *reinterpret_cast<float4*>(xout + (long long)m * d + col) = v;
+        }
+        float mu, q;
+        group_stats(v, mu, q);
+        if (mine && (wtid & 15) == 0 && m < M) stats_out[(long long)m * NC + c] = make_float2(mu, q);
+      }
     };
 
     grid_dep_wait();
     plan();
     // ---------------------------------------------------------------- embedding (tree build + embed)
     {
-      const int tl = wtid >> 4, f4 = (wtid & 15) * 4, m = 8 * (int)rank + tl, col = 64 * c + f4;
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (m < M) {
-        const int depth = a.tree.depth[m];
-        int tok;
-        if (a.override_tokens) tok = a.override_tokens[m];
-        else if (m == 0) tok = a.root[0];
-        else tok = a.topk[(depth - 1) * a.draft_topk + a.tree.rank[m]];
-        const bool live = m < nv;
-        if (!live) tok = 0;
-        int pos = ctx + depth;
-        if (pos >= a.max_pos) { if (live && (wtid & 15) == 0) atomicOr(err, kErrCapacity); pos = a.max_pos - 1; }
-        const bf16* e;
-        if (tok >= 0 && tok < a.vocab) e = a.emb_audio + (long long)tok * d;
-        else if (tok >= a.vocab && tok < a.vocab + a.n_phonemes) e = a.emb_phon + (long long)(tok - a.vocab) * d;
-        else { if (live && (wtid & 15) == 0) atomicOr(err, kErrCapacity); e = a.emb_audio; }
-        const bf16* p = a.pos + (long long)pos * d;
-        const uint2 ev = *reinterpret_cast<const uint2*>(e + col), pv = *reinterpret_cast<const uint2*>(p + col);
-        const __nv_bfloat162 e0 = *reinterpret_cast<const __nv_bfloat162*>(&ev.x), e1 = *reinterpret_cast<const __nv_bfloat162*>(&ev.y);
-        const __nv_bfloat162 q0 = *reinterpret_cast<const __nv_bfloat162*>(&pv.x), q1 = *reinterpret_cast<const __nv_bfloat162*>(&pv.y);
-        v.x = __low2float(e0) + __low2float(q0); v.y = __high2float(e0) + __high2float(q0);
-        v.z = __low2float(e1) + __low2float(q1); v.w = __high2float(e1) + __high2float(q1);
-        *reinterpret_cast<float4*>(a.xa + (long long)m * d + col) = v;
-        xres = v;
-        if ((wtid & 15) == 0) {
-          long long row = -1;
-          if (live) {
-            const int slot = ctx + m;
-            const long long blk = kv_block_of(a.block_table, a.geom, 0, slot, err);
-            if (blk >= 0) row = a.geom.elem(blk, 0, 0, slot % kKvBlock);
+      const int f4 = (wtid & 15) * 4, col = 64 * c + f4;
+#pragma unroll
+      for (int rd = 0; rd < Cfg::kRounds; ++rd) {
+        const int tl = (wtid >> 4) + 8 * rd, m = tok0 + tl;
+        const bool mine = tl < ntok;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (mine && m < M) {
+          const int depth = a.tree.depth[m];
+          int tok;
+          if (a.override_tokens) tok = a.override_tokens[m];
+          else if (m == 0) tok = a.root[0];
+          else tok = a.topk[(depth - 1) * a.draft_topk + a.tree.rank[m]];
+          const bool live = m < nv;
+          if (!live) tok = 0;
+          int pos = ctx + depth;
+          if (pos >= a.max_pos) { if (live && (wtid & 15) == 0) atomicOr(err, kErrCapacity); pos = a.max_pos - 1; }
+          const bf16* e;
+          if (tok >= 0 && tok < a.vocab) e = a.emb_audio + (long long)tok * d;
+          else if (tok >= a.vocab && tok < a.vocab + a.n_phonemes) e = a.emb_phon + (long long)(tok - a.vocab) * d;
+          else { if (live && (wtid & 15) == 0) atomicOr(err, kErrCapacity); e = a.emb_audio; }
+          const bf16* p = a.pos + (long long)pos * d;
+          const uint2 ev = *reinterpret_cast<const uint2*>(e + col), pv = *reinterpret_cast<const uint2*>(p + col);
+          const __nv_bfloat162 e0 = *reinterpret_cast<const __nv_bfloat162*>(&ev.x), e1 = *reinterpret_cast<const __nv_bfloat162*>(&ev.y);
+          const __nv_bfloat162 q0 = *reinterpret_cast<const __nv_bfloat162*>(&pv.x), q1 = *reinterpret_cast<const __nv_bfloat162*>(&pv.y);
+          v.x = __low2float(e0) + __low2float(q0); v.y = __high2float(e0) + __high2float(q0);
+          v.z = __low2float(e1) + __low2float(q1); v.w = __high2float(e1) + __high2float(q1);
+          *reinterpret_cast<float4*>(a.xa + (long long)m * d + col) = v;
+          xres[rd] = v;
+          if ((wtid & 15) == 0) {
+            long long row = -1;
+            if (live) {
+              const int slot = ctx + m;
+              const long long blk = kv_block_of(a.block_table, a.geom, 0, slot, err);
+              if (blk >= 0) row = a.geom.elem(blk, 0, 0, slot % kKvBlock);
+            }
+            s_kvrow[tl] = row;
+            if (c == 0) { a.tokens[m] = tok; a.kv_row[m] = row; }
           }
-          s_kvrow[tl] = row;
-          if (c == 0) { a.tokens[m] = tok; a.kv_row[m] = row; }
+        } else if (mine && (wtid & 15) == 0) {
+          s_kvrow[tl] = -1;
         }
-      } else if ((wtid & 15) == 0) {
-        s_kvrow[tl] = -1;
+        float mu, q;
+        group_stats(v, mu, q);
+        if (mine && (wtid & 15) == 0 && m < M) a.stats_a[(long long)m * NC + c] = make_float2(mu, q);
       }
-      float sm = (v.x + v.y) + (v.z + v.w);
-#pragma unroll
-      for (int o = 8; o > 0; o >>= 1) sm += __shfl_xor_sync(0xffffffffu, sm, o);
-      const float mu = sm * (1.0f / 64.0f);
-      const float d0 = v.x - mu, d1 = v.y - mu, d2 = v.z - mu, d3 = v.w - mu;
-      float q = (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
-#pragma unroll
-      for (int o = 8; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
-      if ((wtid & 15) == 0 && m < M) a.stats_a[(long long)m * NC + c] = make_float2(mu, q);
       publish(kFfSyncXa);
     }
 
-    const int ntile = np_mine + ((rank == kFfTreeRank && nv > 0) ? 1 : 0);
+    const int ntile = np_mine + ((rank == CS - 1 && nv > 0) ? 1 : 0);
     unsigned long long anc_lo = 0ull;
     if (tok_t < nv && tok_t < M) { unsigned long long hi_unused; a.tree.anc_of(0, tok_t, anc_lo, hi_unused); }
 
@@ -710,8 +752,8 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
       {
         const float* bq = lvec(a.bqkv);
         rb_wait();
-        for (int it = wtid; it < 192; it += kFfWorkers) {
-          const int tl = it / 24, u = it % 24, m = 8 * (int)rank + tl;
+        for (int it = wtid; it < ntok * 24; it += kFfWorkers) {
+          const int tl = it / 24, u = it % 24, m = tok0 + tl;
           const int part = u >> 3, j0 = (u & 7) * 8;
           const float4 s0 = rb_sum4(192, tl, 8 * u), s1 = rb_sum4(192, tl, 8 * u + 4);
           const float* bp = bq + part * d + c * 64 + j0;
@@ -722,13 +764,13 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
             const uint32_t off = (uint32_t)m * 128u + ((uint32_t)((u & 7) ^ (m & 7)) << 4);
             if (part == 0) {
 #pragma unroll
-              for (uint32_t p = 0; p < (uint32_t)kFfCluster; ++p) {
+              for (uint32_t p = 0; p < (uint32_t)CS; ++p) {
                 const uint32_t q_rem = ff_mapa(xa + off, p);
                 ff_st_cluster_u4(q_rem, val);
                 ff_st_cluster_u4(q_rem + 8192u, val);
               }
             } else {
-              ff_st_cluster_u4(ff_mapa(xa + (part == 1 ? 16384u : 24576u) + off, (uint32_t)kFfTreeRank), val);
+              ff_st_cluster_u4(ff_mapa(xa + (part == 1 ? 16384u : 24576u) + off, (uint32_t)(CS - 1)), val);
               const long long row = s_kvrow[tl];
               if (row >= 0) *reinterpret_cast<uint4*>(pool_l + row + (part - 1) * kv_stride + (long long)c * tile_elems + j0) = val;
             }
@@ -739,7 +781,7 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
         ff_fence_cluster();
         __syncwarp();
         if (lane == 0)
-          for (uint32_t p = 0; p < (uint32_t)kFfCluster; ++p) ff_arrive_remote(ff_mapa(bar_qkv, p));
+          for (uint32_t p = 0; p < (uint32_t)CS; ++p) ff_arrive_remote(ff_mapa(bar_qkv, p));
         rb_done();
       }
       // ---------------------------------------------------------------- attention: this CTA's pages
@@ -763,8 +805,8 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
               const int valid = ctx - (p0 + t) * kKvBlock;
               if (valid < kKvBlock) {
                 if (wtid < kKvBlock && wtid >= valid) {
-                  const int seq = l * (nkc + 1 + np_mine + 1 + nrb * nkc + 1 + nk2) + nkc + 1 + t;
-                  uint4* vr = reinterpret_cast<uint4*>(ring_p + (seq % kFfSlots) * kFfSlotBytes + kFfTileBytes + wtid * 128);
+                  const int seq = l * ipl + offKV + t;
+                  uint4* vr = reinterpret_cast<uint4*>(ring_p + (seq % R) * kFfSlotBytes + kFfTileBytes + wtid * 128);
 #pragma unroll
                   for (int q8 = 0; q8 < 8; ++q8) vr[q8] = make_uint4(0, 0, 0, 0);
                 }
@@ -848,44 +890,50 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
         }
         rb_begin();
         {
-          const uint32_t dst = rb_owner + (uint32_t)((((int)rank * 2 + half_t) * 8 + tl_t) * 68) * 4u;
+          const uint32_t dst = rb_owner + (uint32_t)(((rank * 2 + half_t) * TPO + tl_t) * 68) * 4u;
 #pragma unroll
           for (int i = 0; i < 16; ++i) ff_st_cluster_f4(dst + 16u * i, oacc[4 * i], oacc[4 * i + 1], oacc[4 * i + 2], oacc[4 * i + 3]);
           ff_st_cluster_f4(dst + 256u, l_run, m_run, 0.f, 0.f);
         }
         rb_sent();
         tc_fence_before();
-        // owner: merge the 16 partials of each of its tokens
+        // owner: merge the 2 CS partials of each of its tokens
         rb_wait();
         {
-          const int tl = wtid >> 4, f4 = (wtid & 15) * 4, m = 8 * (int)rank + tl;
-          float mm[16], ll[16];
-          float mxx = -INFINITY;
+          const int f4 = (wtid & 15) * 4;
 #pragma unroll
-          for (int p = 0; p < 16; ++p) {
-            const float4 lm = *reinterpret_cast<const float4*>(rb_p + (p * 8 + tl) * 68 + 64);
-            ll[p] = lm.x; mm[p] = lm.y;
-            mxx = fmaxf(mxx, lm.y);
-          }
-          float Ls = 0.f;
-          float4 o4 = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int rd = 0; rd < Cfg::kRounds; ++rd) {
+            const int tl = (wtid >> 4) + 8 * rd, m = tok0 + tl;
+            if (tl < ntok) {
+              float mm[2 * CS], ll[2 * CS];
+              float mxx = -INFINITY;
 #pragma unroll
-          for (int p = 0; p < 16; ++p) {
-            const float w = (mm[p] == -INFINITY) ? 0.f : exp2f(mm[p] - mxx);
-            const float4 ov = *reinterpret_cast<const float4*>(rb_p + (p * 8 + tl) * 68 + f4);
-            Ls = fmaf(ll[p], w, Ls);
-            o4.x = fmaf(ov.x, w, o4.x); o4.y = fmaf(ov.y, w, o4.y); o4.z = fmaf(ov.z, w, o4.z); o4.w = fmaf(ov.w, w, o4.w);
-          }
-          if (m < M) {
-            const float inv = (m < nv && Ls > 0.f) ? 1.f / Ls : 0.f;
-            uint2 v;
-            v.x = pack_bf16(o4.x * inv, o4.y * inv);
-            v.y = pack_bf16(o4.z * inv, o4.w * inv);
-            *reinterpret_cast<uint2*>(a.o + (long long)m * d + c * 64 + f4) = v;
-            if (a.attn_tap) *reinterpret_cast<uint2*>(a.attn_tap + ((long long)l * M + m) * d + c * 64 + f4) = v;
+              for (int p = 0; p < 2 * CS; ++p) {
+                const float4 lm = *reinterpret_cast<const float4*>(rb_p + (p * TPO + tl) * 68 + 64);
+                ll[p] = lm.x; mm[p] = lm.y;
+                mxx = fmaxf(mxx, lm.y);
+              }
+              float Ls = 0.f;
+              float4 o4 = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+              for (int p = 0; p < 2 * CS; ++p) {
+                const float w = (mm[p] == -INFINITY) ? 0.f : exp2f(mm[p] - mxx);
+                const float4 ov = *reinterpret_cast<const float4*>(rb_p + (p * TPO + tl) * 68 + f4);
+                Ls = fmaf(ll[p], w, Ls);
+                o4.x = fmaf(ov.x, w, o4.x); o4.y = fmaf(ov.y, w, o4.y); o4.z = fmaf(ov.z, w, o4.z); o4.w = fmaf(ov.w, w, o4.w);
+              }
+              if (m < M) {
+                const float inv = (m < nv && Ls > 0.f) ? 1.f / Ls : 0.f;
+                uint2 v;
+                v.x = pack_bf16(o4.x * inv, o4.y * inv);
+                v.y = pack_bf16(o4.z * inv, o4.w * inv);
+                *reinterpret_cast<uint2*>(a.o + (long long)m * d + c * 64 + f4) = v;
+                if (a.attn_tap) *reinterpret_cast<uint2*>(a.attn_tap + ((long long)l * M + m) * d + c * 64 + f4) = v;
+              }
+            }
           }
         }
-        publish(kFfSyncO + (c * 64) / ks_d);
+        publish(kFfSyncO + c);
         rb_done();
       }
       // ---------------------------------------------------------------- output projection, rows [64c, 64c+64)
@@ -900,8 +948,8 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
         const float* b1 = lvec(a.b1);
         const int units = n1 / 8;                            // 16-byte units per token
         rb_wait();
-        for (int it = wtid; it < 8 * units; it += kFfWorkers) {
-          const int tl = it / units, u = it % units, m = 8 * (int)rank + tl;
+        for (int it = wtid; it < ntok * units; it += kFfWorkers) {
+          const int tl = it / units, u = it % units, m = tok0 + tl;
           const float4 s0 = rb_sum4(n1, tl, 8 * u), s1 = rb_sum4(n1, tl, 8 * u + 4);
           const float* bp = b1 + c * n1 + 8 * u;
           const float4 b0v = __ldg(reinterpret_cast<const float4*>(bp)), b1v = __ldg(reinterpret_cast<const float4*>(bp + 4));
@@ -909,7 +957,7 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
                                fmaxf(s1.x + b1v.x, 0.f), fmaxf(s1.y + b1v.y, 0.f), fmaxf(s1.z + b1v.z, 0.f), fmaxf(s1.w + b1v.w, 0.f)};
           if (m < M) *reinterpret_cast<uint4*>(a.mid + (long long)m * F + c * n1 + 8 * u) = ff_pack8(v8);
         }
-        publish(kFfSyncMid + (c * n1) / ks_f);
+        publish(kFfSyncMid + c);
         rb_done();
       }
       // ---------------------------------------------------------------- second feed-forward matrix, rows [64c, 64c+64)
@@ -928,8 +976,8 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
         }
         send_partial(128, true);
         rb_wait();
-        for (int it = wtid; it < 8 * 32; it += kFfWorkers) {
-          const int tl = it >> 5, f4 = (it & 31) * 4, m = 8 * (int)rank + tl;
+        for (int it = wtid; it < ntok * 32; it += kFfWorkers) {
+          const int tl = it >> 5, f4 = (it & 31) * 4, m = tok0 + tl;
           const float4 s = rb_sum4(128, tl, f4);
           if (m < M) *reinterpret_cast<float4*>(a.logits + (long long)m * a.vpad + 128 * t + f4) = s;
         }

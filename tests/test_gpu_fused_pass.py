@@ -26,7 +26,7 @@ def _sampling(wl, seed=7):
             P.Sampling.make(tau=wl.tau, temperature=wl.temperature, seed=seed))
 
 
-def _start(wl, n_iters, seed=11, prefill_rows=16):
+def _start(wl, n_iters, seed=11, prefill_rows=16, cluster=1):
     import paper_2410_21951_b200 as P
     w = W.make_weights(wl.shape, wl.seed())
     model = O.Model.from_shape(wl.shape, w)
@@ -37,6 +37,7 @@ def _start(wl, n_iters, seed=11, prefill_rows=16):
     table, total = W.shuffled_block_table(need, 64, seed, spare_pages=3)
     g = P.Vadusa(wl.shape, w, max_batch=1, max_tree_nodes=wl.tree_nodes, max_blocks_per_seq=table.shape[1],
                  kv_num_blocks=total, prefill_rows=prefill_rows)
+    g.set_fused_pass(cluster)
     g.set_tree(tpl.parent, tpl.rank)
     g.begin(table)
     g.prefill(toks[None, :].copy(), [len(toks)])
@@ -45,19 +46,21 @@ def _start(wl, n_iters, seed=11, prefill_rows=16):
     return w, model, tpl, g, table, st, (ph, pr)
 
 
-@pytest.mark.parametrize("heads,nodes,rows", [(8, 16, 16), (8, 48, 0), (16, 64, 0)])
-def test_fused_pass_lockstep_against_the_oracle(heads, nodes, rows):
+@pytest.mark.parametrize("heads,nodes,rows,cluster", [(8, 16, 16, 8), (8, 48, 0, 6), (16, 64, 0, 1), (16, 37, 16, 6)])
+def test_fused_pass_lockstep_against_the_oracle(heads, nodes, rows, cluster):
     """Lockstep iterations (logits, attention outputs per layer, draft, acceptance, committed K/V rows).  With
-    prefill_rows = 0 the prefix chunks also go through the persistent kernel, one chunk per pass."""
+    prefill_rows = 0 the prefix chunks also go through the persistent kernel, one chunk per pass.  Clusters of
+    8 CTAs (K slices of equal width, 8 tokens per owner) and of 6 (uneven K slices and token shares)."""
     caps = (6, 3, 2) if nodes < 64 else (10, 5, 3)
     wl = _wide_toy(nodes, heads=heads, d_ffn=256 * heads, tree_caps=caps, index=31 + heads)
-    w, model, tpl, g, table, st, _ = _start(wl, 6, prefill_rows=rows)
+    w, model, tpl, g, table, st, _ = _start(wl, 6, prefill_rows=rows, cluster=cluster)
     so, sg = _sampling(wl)
     launches0 = g.kernel_launches()
     rep = lockstep(g, table, model, {0: st}, tpl, so, sg, 5, "bf16", oracle_mode="memo", check_attn=True)
     assert rep.iterations == 5 and rep.attn_checked == 5
     assert rep.root_checked + rep.draft_sets_checked > 0 and rep.accept_checked + rep.accept_undecidable == 5
     # one launch for the pass: draft (3) + tree tokens (1) + pass (1) + accept, commit (2) per iteration
+    assert g.fused_pass_clusters() >= heads, "this device cannot hold one cluster per head"
     assert g.kernel_launches() - launches0 <= 5 * 8
     K, V = read_kv(g, table, 0, st.S)
     assert np.abs(K - st.kv.K[:, :st.S]).max() <= TOL["bf16"]
@@ -90,8 +93,8 @@ def test_fused_pass_planted_path_moves_rows_and_matches_stepwise_path():
     g.check()
 
 
-@pytest.mark.parametrize("ctx_len", [37, 1990, 2500])
-def test_fused_pass_long_context_with_injected_kv(ctx_len):
+@pytest.mark.parametrize("ctx_len,cluster", [(37, 8), (1990, 8), (2500, 8), (2500, 6)])
+def test_fused_pass_long_context_with_injected_kv(ctx_len, cluster):
     """Seeded random K/V rows as context (no prefill on either side): 1 page, 32 pages (four per CTA: two
     groups) and 40 pages with a ragged last page (five per CTA); logits and attention outputs of every
     node against the oracle's tree-masked pass."""
@@ -103,6 +106,7 @@ def test_fused_pass_long_context_with_injected_kv(ctx_len):
     N = wl.tree_nodes
     tpl = W.static_template(N, wl.tree_caps)
     g, table = make_gpu(wl.shape, w, 1, N, [ctx_len + N + 8], wl.seed(1))
+    g.set_fused_pass(cluster)
     g.begin(table, ctx_len=[ctx_len])
     g.set_tree(tpl.parent, tpl.rank)
     rng = np.random.default_rng(wl.seed(2) + ctx_len)
@@ -126,4 +130,5 @@ def test_fused_pass_long_context_with_injected_kv(ctx_len):
     e_a = max(np.abs(at[l] - out.attn[l]).max() for l in range(model.L))
     print(f"context {ctx_len}: max |logit err| {e_l:.2e}, max |attn err| {e_a:.2e}")
     assert e_l <= TOL["bf16"] and e_a <= TOL["bf16"]
+    assert g.fused_pass_clusters() >= 8
     g.check()
