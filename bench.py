@@ -33,7 +33,7 @@ TREE_NODES = 0          # 0: the workload's own tree; --tree-nodes 96 / 128: the
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the 49 projection launches of one C2 step, from the
-# ncu capture summarised in profiles/gemm_tc_kernel_c2.md; valid for the kernel sources with this hash only.
+# ncu capture of those launches (batch 1, 64 nodes); valid for the kernel sources with this hash only.
 _NCU_TRAFFIC = {"src_sha256_16": "718c66f6ec1bad54", "bytes_per_step": 327.97e6, "launches": 49}
 
 
@@ -49,7 +49,7 @@ def _gemm_traffic():
 
 
 # DRAM bytes of one tree_attention_tc_kernel launch relative to its algorithmic K/V bytes, from the ncu capture at
-# 24 sequences summarised in profiles/tree_attention_tc_kernel_c5_batch24.md (163.17 MB read + 3.83 MB written for
+# 24 sequences (163.17 MB read + 3.83 MB written for
 # 163.1 MB of K/V); every (head, sequence) CTA reads its own pages once, so the traffic of a launch grows in
 # proportion to its sequences' bytes.  Valid for the kernel sources with this hash only.
 _NCU_ATTN = {"src_sha256_16": "a1b015d014f84a83", "dram_over_algorithmic": 167.0 / 163.1}
@@ -377,7 +377,7 @@ def run_ours(args):
 
 
 def run_c5(args):
-    """Verify-step microbenchmark at BASELINE config 5: batch 64, ragged KV lengths 256-3000, a random
+    """Verify-step microbenchmark of configuration 5: batch 64, ragged KV lengths 256-3000, a random
     64-node topology per sequence, random bf16 K/V and tokens.  One step = draft heads + verify pass +
     accept/commit.  Reports per-kernel roofline fractions (attention: HBM; projections: bf16 tensor)."""
     import torch
@@ -467,7 +467,7 @@ def run_c5(args):
 
 
 def run_batch(args):
-    """BASELINE configs 3 (batch 16, vocab 2049, 42-node tree, tau 5, T 0.8, 500 tokens) and 4 (batch 32,
+    """Configurations 3 (batch 16, vocab 2049, 42-node tree, tau 5, T 0.8, 500 tokens) and 4 (batch 32,
     contexts 1000-4000 in a paged cache, 64-node tree, tau in {1,3,5}, 256 iterations): prefill through the
     library, then timed draft+verify+accept/commit steps.  One JSON line per tolerance value."""
     import torch

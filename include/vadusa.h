@@ -150,7 +150,10 @@ int32_t vadusa_weight_count(const vadusa_config *cfg);
 vadusa_status vadusa_weight_info(const vadusa_config *cfg, int32_t index, vadusa_tensor_info *h_out);
 
 /* ---- life cycle ------------------------------------------------------------------ */
-/* Validates the configuration, records the pointers, clears the state area of the
+/* Binds a context to one model: the decoder-only speech-token model of Sec. III-A.1 (12 layers, 16 heads,
+ * d 1024, feed-forward 4096 in the paper; any shape the configuration checks allow) and its draft heads
+ * (Sec. II-A: one residual Linear+SiLU block and one vocabulary matrix per head).
+ * Validates the configuration, records the pointers, clears the state area of the
  * workspace.  Synchronises the stream once.  Makes cfg->device the calling thread's current
  * CUDA device; every later call on the context must be made with that device current.  A
  * context is not thread-safe: one thread at a time. */
@@ -168,7 +171,8 @@ const char *vadusa_last_error(const vadusa_ctx *ctx);   /* NUL-terminated, owned
 vadusa_status vadusa_set_tree(vadusa_ctx *ctx, int32_t n_nodes, const int32_t *h_parent,
                               const int32_t *h_rank, int32_t per_sequence);
 
-/* Starts a batch.  block_table: device int32 [batch][max_blocks_per_seq], the KV
+/* Starts a batch of independent utterances (Sec. II-A treats one; nothing is exchanged between sequences,
+ * each has its own context, tree scores and acceptance).  block_table: device int32 [batch][max_blocks_per_seq], the KV
  * blocks of every sequence in logical order; it must cover every position the
  * sequence can reach plus max_tree_nodes (tree nodes are scored in place behind the
  * context).  h_ctx_len: host int32 [batch], tokens already present in the cache
@@ -228,7 +232,10 @@ vadusa_status vadusa_accept_and_commit(vadusa_ctx *ctx, const vadusa_sampling *s
                                        int32_t *path_nodes, int32_t *path_tokens, int64_t *kv_slots,
                                        uint64_t *edge_bits, int32_t *next_root);
 
-/* Runs draft -> verify -> accept+commit until every sequence has max_new_tokens tokens
+/* The decoding loop of Sec. II-A (Fig. 1b-c): draft heads propose, the base model scores the candidate tree in
+ * one pass, Algorithm 1 keeps the longest accepted path, and the base head's distribution at the last accepted
+ * token starts the next iteration.
+ * Runs draft -> verify -> accept+commit until every sequence has max_new_tokens tokens
  * (or max_iters iterations, if > 0).  out_tokens: int32 [batch][max_new_tokens]
  * (a sequence's surplus tokens of its last iteration are dropped); out_len: int32
  * [batch].  Synchronises; returns device-side errors.  h_stats may be NULL. */
@@ -245,18 +252,22 @@ vadusa_status vadusa_generate_host(vadusa_ctx *ctx, const vadusa_sampling *sampl
                                    int32_t *h_out_tokens, int32_t *h_out_len, vadusa_stats *h_stats);
 
 /* ---- state ---------------------------------------------------------------------- */
-vadusa_status vadusa_get_lengths(vadusa_ctx *ctx, int32_t *h_ctx_len);  /* synchronises */
+/* Tokens in each sequence's cache: prefix plus what the iterations so far have committed (Sec. II-A: an
+ * iteration commits between 1 and n_draft_heads + 1 tokens, so the length is the only way to know how far a
+ * sequence has come).  h_ctx_len: host int32 [batch].  Synchronises; returns device-side errors. */
+vadusa_status vadusa_get_lengths(vadusa_ctx *ctx, int32_t *h_ctx_len);
 vadusa_status vadusa_check(vadusa_ctx *ctx);                            /* synchronises; device error word */
 int64_t vadusa_kernel_launches(const vadusa_ctx *ctx);                  /* total kernels enqueued so far */
 
 /* A verify pass over ONE sequence of at most 64 tree nodes (the batch-1 step of Sec. II-A: one tree per
- * iteration) runs, for bf16 models with head_dim 64 and 8 or 16 heads, as a single persistent kernel that
- * keeps the whole grid resident and hands activations from step to step through shared memory of thread-block
- * clusters and counters in L2, instead of one kernel per projection.  It computes the same quantities with
- * the same rounding points.  Its clusters (one per head) have 8 CTAs where the device can hold all of them at
- * once, else 6.  enable = 0 selects the kernel-per-step path for such passes too (used to compare the two);
- * 1 (the default) lets the library choose; 6 or 8 ask for that cluster size where it fits.  Host-side switch:
- * takes effect with the next call. */
+ * iteration) can run, for bf16 models with head_dim 64 and 8 or 16 heads, as a single persistent kernel that
+ * keeps the whole grid resident (one thread-block cluster per head), lets weights and context K/V run ahead
+ * of the dependency chain through a TMA ring, and hands activations from step to step through the clusters'
+ * shared memory and counters in L2 instead of one kernel per projection.  It computes the same quantities with
+ * the same rounding points.  Its clusters have 8 CTAs where the device can hold one per head at once, else 6.
+ * enable = 0 (the default): kernel-per-step path, which is the faster one on the devices measured so far;
+ * 1: the persistent kernel with the cluster size the library chooses; 6 or 8: that cluster size where it fits.
+ * Host-side switch: takes effect with the next call. */
 vadusa_status vadusa_set_fused_pass(vadusa_ctx *ctx, int32_t enable);
 /* How many of that kernel's clusters (one per head, of the chosen size) the device can hold at once, as found
  * when the first such pass was enqueued (-1 before).  The persistent kernel is used only if this is >= n_heads. */
@@ -318,8 +329,10 @@ vadusa_status vadusa_profile_end(vadusa_ctx *ctx, vadusa_kernel_time *h_out, int
  * GPU that loads the library holds until the process exits.  It is meant for code that may
  * not call cudaMalloc: a plug-in inside another framework's memory plan, a real-time audio
  * loop that must not touch the allocator once it runs, a process whose device memory was
- * handed out completely before this library was loaded.  The call makes no allocation of
- * any kind, on the host or on the device.
+ * handed out completely before this library was loaded.  The call itself allocates nothing,
+ * on the host or on the device; but the FIRST call on a device makes the CUDA runtime load this
+ * part of the library and reserve the 2 MiB array there, which fails (VADUSA_ECUDA) if the
+ * device has no memory left: make one call at start-up, before memory is handed out.
  *   draft_w [heads][d_model][d_model], draft_u [heads][ceil(vocab/128)*128][d_model] in the
  *   model dtype (0 fp32, 1 bf16; the layout of the weight blob), draft_b fp32 [heads][d_model],
  *   hstar [batch][d_model] in the model dtype, topk_out int32 [batch][heads][topk]; all device
@@ -331,7 +344,9 @@ vadusa_status vadusa_profile_end(vadusa_ctx *ctx, vadusa_kernel_time *h_out, int
  *   make that first call outside any stream capture.
  * All calls on one GPU share the array and it keeps what the last call left there; every
  *   call overwrites what it reads, so nothing needs clearing, but two calls that overlap on
- *   the GPU (different streams, no ordering between them) race on it. */
+ *   the GPU (different streams, no ordering between them) race on it.
+ * On the host the call and vadusa_static_last_error() share unsynchronised state (the per-device
+ *   address table and the message buffer): call them from one thread at a time. */
 vadusa_status vadusa_draft_topk_static(const void *draft_w, const float *draft_b, const void *draft_u,
                                        const void *hstar, int32_t dtype, int32_t batch, int32_t d_model,
                                        int32_t vocab, int32_t n_draft_heads, int32_t topk, int32_t eos_masked,

@@ -15,19 +15,15 @@ import numpy as np
 
 
 def verify_branch(cands: Sequence[int], sets: Sequence[Sequence[int]]) -> int:
-    """Algorithm 1, after the sample sets v_0..v_k have been drawn.
+    """Tolerance check of one branch (Algorithm 1, Sec. II-C), after the draw sets have been made.
 
-    cands = (c_0, ..., c_k); c_0 is always kept; c_{i+1} is kept while it lies in
-    v_i; the first miss ends the branch.  Returns k* (index of the last kept
-    candidate), so k*+1 tokens are accepted."""
-    k = len(cands) - 1
-    k_star = k
-    for i in range(k):
-        if cands[i + 1] in sets[i]:
-            continue
-        k_star = i
-        break
-    return k_star
+    cands = (c_0, ..., c_k) are the branch's tokens from the root down; sets[i] holds
+    the tau tokens the base head drew at c_i.  The root is the base head's own token and
+    is always kept; the accepted part of the branch ends just before the first child
+    that is missing from its parent's draws.  Returns the index of the last accepted
+    candidate (so that many + 1 tokens are accepted)."""
+    misses = [i for i in range(len(cands) - 1) if cands[i + 1] not in sets[i]]
+    return misses[0] if misses else len(cands) - 1
 
 
 def select_best(branches: Sequence[Tuple[Tuple[int, ...], int]]) -> int:

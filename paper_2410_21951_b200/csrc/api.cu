@@ -47,7 +47,7 @@ struct vadusa_ctx {
   int tree_per_seq = 0;
   int max_rank_used = 0;
   int tree_max_depth = 0;
-  int fused_enabled = 1;      // single-sequence passes may run as one persistent kernel
+  int fused_enabled = 0;      // single-sequence passes run as one persistent kernel (0: no, 1: yes, 6 / 8: with that cluster size)
   int fused_clusters = -1;    // clusters of that kernel that can be resident at once on this device (-1: not asked yet)
   int fused_cs = -1;          // CTAs per cluster chosen for it (8 or 6; 0: the device cannot hold one cluster per head)
   int fused_n8 = 0, fused_n6 = 0;
@@ -834,9 +834,9 @@ vadusa_status set_kernel_attributes(vadusa_ctx* ctx) {
   CU(cudaFuncSetAttribute(tree_attention_simt_kernel<bf16, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(64)));
   CU(cudaFuncSetAttribute(tree_attention_simt_kernel<bf16, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(32)));
   CU(cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmemBytes));
-  // the accept kernel keeps one row of keys and one of probabilities in shared memory
-  if (2 * vpad(&ctx->cfg) * (int)sizeof(float) > 48 * 1024)
-    CU(cudaFuncSetAttribute(accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * vpad(&ctx->cfg) * (int)sizeof(float)));
+  // the accept kernel keeps one row of keys and one of probabilities in shared memory.  The limit is an attribute of
+  // the function on this device, shared by every context: always the library's largest vocabulary
+  CU(cudaFuncSetAttribute(accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 24576 * (int)sizeof(float)));
   // ask for the largest shared-memory carve-out so that several CTAs fit on an SM
   CU(cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
   return VADUSA_OK;

@@ -45,12 +45,13 @@ constexpr unsigned long long kFfWaitNs = 400ull * 1000 * 1000;
 template <int CS> struct FfCfg {
   static constexpr int kTpo = (64 + CS - 1) / CS;                       // tokens per owner, at most
   static constexpr int kMaxKc = (16 + CS - 1) / CS;                     // chunks of a CTA's K slice of d_model, at most
-  static constexpr int kSlots = CS >= 8 ? 8 : 6;                        // ring slots
+  static constexpr int kSlots = CS >= 8 ? 7 : 6;                        // ring slots
   static constexpr uint32_t kRingBytes = kSlots * kFfSlotBytes;
   // LayerNorm operand: one 128-row tile (16 KB) per chunk; also the Q tile + the tree's K and V tiles (32 KB)
   static constexpr uint32_t kXaBytes = kMaxKc * 16384u < 32768u ? 32768u : kMaxKc * 16384u;
-  static constexpr uint32_t kRbBytes = CS * kTpo * 256 * 4;             // receive buffer of the cluster reductions
-  static constexpr int kSmemBytes = (int)(kRingBytes + kXaBytes + kRbBytes + kFfMiscBytes + 1024 /*alignment*/);
+  static constexpr uint32_t kRbBytes = 64 * (256 + 4) * 4;              // this CTA's K-slice partial [64 tokens][N + 4], read by the owners
+  static constexpr uint32_t kQoBytes = ((kTpo * 192 * 2 + 1023) / 1024) * 1024;   // q/k/v rows of the owned tokens, read by the peers
+  static constexpr int kSmemBytes = (int)(kRingBytes + kXaBytes + kRbBytes + kQoBytes + kFfMiscBytes + 1024 /*alignment*/);
   static constexpr int kRounds = (kTpo * 16 + kFfWorkers - 1) / kFfWorkers;   // passes of 128 threads over (token, 4 features)
 };
 
@@ -127,6 +128,22 @@ __device__ __forceinline__ void ff_st_cluster_f4(uint32_t addr, float a, float b
 __device__ __forceinline__ void ff_st_cluster_u4(uint32_t addr, uint4 v) {
   asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
+__device__ __forceinline__ float4 ff_ld_cluster_f4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint4 ff_ld_cluster_u4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared::cluster.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void ff_st_shared_f4(uint32_t addr, float a, float b, float c, float d) {
+  asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+__device__ __forceinline__ void ff_st_shared_u4(uint32_t addr, uint4 v) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
 __device__ __forceinline__ void ff_arrive_remote(uint32_t remote_bar) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
 }
@@ -186,17 +203,16 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
     const __grid_constant__ CUtensorMap tmKV,    // [L][blocks * 2 * H * 64][64]  box 64 x 64
     const FusedArgs a) {
   using Cfg = FfCfg<CS>;
-  constexpr int R = Cfg::kSlots, TPO = Cfg::kTpo, KCMAX = Cfg::kMaxKc;
+  constexpr int R = Cfg::kSlots, KCMAX = Cfg::kMaxKc;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_p = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t ring = base, xa = base + Cfg::kRingBytes, rb = xa + Cfg::kXaBytes, bars = rb + Cfg::kRbBytes;
+  const uint32_t ring = base, xa = base + Cfg::kRingBytes, rb = xa + Cfg::kXaBytes, qo = rb + Cfg::kRbBytes, bars = qo + Cfg::kQoBytes;
   uint8_t* ring_p = base_p;
-  float* rb_p = reinterpret_cast<float*>(base_p + Cfg::kRingBytes + Cfg::kXaBytes);
-  uint8_t* misc_p = base_p + Cfg::kRingBytes + Cfg::kXaBytes + Cfg::kRbBytes;
+  uint8_t* misc_p = base_p + Cfg::kRingBytes + Cfg::kXaBytes + Cfg::kRbBytes + Cfg::kQoBytes;
   const uint32_t full0 = bars, empty0 = bars + 64, bar_xa = bars + 128, bar_acc = bars + 136, bar_accfree = bars + 144,
                  bar_s = bars + 152, bar_p = bars + 160, bar_o = bars + 168, bar_qkv = bars + 176,
-                 bar_rbfull = bars + 184, bar_rbfree = bars + 192, holder = bars + 200;
+                 bar_rbfull = bars + 184, bar_rbfree = bars + 192, holder = bars + 200, bar_q = bars + 208;
   volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(misc_p + 200);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc_p + 204);
   float2* s_rowstat = reinterpret_cast<float2*>(misc_p + 256);         // [64] (mean, rstd)
@@ -221,7 +237,7 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
     for (int s = 0; s < R; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
     mbar_init(bar_xa, kFfWorkers); mbar_init(bar_acc, 1); mbar_init(bar_accfree, kFfWorkers);
     mbar_init(bar_s, 1); mbar_init(bar_p, kFfWorkers); mbar_init(bar_o, 1);
-    mbar_init(bar_qkv, 4 * CS); mbar_init(bar_rbfull, 4 * CS); mbar_init(bar_rbfree, CS);
+    mbar_init(bar_qkv, 4 * CS); mbar_init(bar_rbfull, 4 * CS); mbar_init(bar_rbfree, CS); mbar_init(bar_q, kFfWorkers);
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmQkv); tma_prefetch_desc(&tmWo); tma_prefetch_desc(&tmW1); tma_prefetch_desc(&tmW2);
@@ -417,9 +433,7 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
         if (!ok) break;
         umma_commit(bar_acc);
         // ---- attention of head c over this CTA's pages (and the tree's own keys in the last CTA)
-        ok = ok && ff_wait([&] { return ff_try_wait_cluster(bar_qkv, n_qkv & 1); }, err, abort_flag);
-        ++n_qkv;
-        ff_fence_proxy_all();
+        wait_local(bar_q, n_qkv);               // the workers have gathered the Q tile (and the tree's K, V tiles)
         tc_fence_after();
         for (int t0 = 0; t0 < ntile && ok; t0 += kFfGroup) {
           const int npg = min(kFfGroup, ntile - t0);
@@ -512,15 +526,10 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
     const int wtid = tid - 64, ww = warp - 2, wq = warp & 3;
     const int lane_t = 32 * wq + lane;                       // this thread's TMEM lane
     const int tok_t = lane_t & 63, half_t = lane_t >> 6;     // token of the lane, which copy of it
-    const int owner_t = ff_owner(tok_t, 64, CS);             // the CTA that sums this token's partial rows
-    int own_first_t, own_cnt_t;
-    ff_split(64, CS, owner_t, own_first_t, own_cnt_t);
-    const int tl_t = tok_t - own_first_t;
     int tok0, ntok;                                          // the tokens this CTA owns
     ff_split(64, CS, rank, tok0, ntok);
     const uint32_t trow = tmem + ((uint32_t)(32 * wq) << 16);
-    const uint32_t rb_owner = ff_mapa(rb, (uint32_t)owner_t);
-    uint32_t n_acc = 0, n_rb = 0, n_s = 0, n_o = 0;
+    uint32_t n_acc = 0, n_rb = 0, n_s = 0, n_o = 0, n_qkv = 0;
     const long long kv_stride = (long long)a.geom.n_heads * kKvBlock * a.geom.head_dim;   // K row -> V row of a head
     const int tile_elems = kKvBlock * a.geom.head_dim;
 
@@ -532,11 +541,11 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
       if (wtid == 0) ff_wait([&] { return ff_ld_acquire(a.sync + word) >= target; }, err, abort_flag);
       ff_workers_sync();
     };
-    auto publish = [&](int word) {                           // every worker has stored its part
-      ff_fence_proxy_global();
-      __threadfence();
+    // every worker has stored its part; tma: the data is read by TMA loads (async proxy) of other CTAs
+    auto publish = [&](int word, bool tma) {
+      if (tma) ff_fence_proxy_global();
       ff_workers_sync();
-      if (wtid == 0) ff_red_release(a.sync + word, 1u);
+      if (wtid == 0) { __threadfence(); ff_red_release(a.sync + word, 1u); }
     };
     // the receive buffers of the cluster are free again (every peer has read what the last round left)
     auto rb_begin = [&]() {
@@ -557,33 +566,35 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
         for (uint32_t p = 0; p < (uint32_t)CS; ++p) ff_arrive_remote(ff_mapa(bar_rbfree, p));
       ++n_rb;
     };
-    // K-slice partial D[token][0:N) of this CTA -> the owners of the tokens (receive buffer: [source][token][N]).
-    // dup: tokens are stored twice in the operand, the second copy's lanes send the upper half of the columns;
-    // else lanes 0..63 send everything.
+    // K-slice partial D[token][0:N) of this CTA -> its own shared memory as [token][N + 4] fp32 (rows padded by 16
+    // bytes: the lanes of a warp, one token each, then fall into different banks); the owners of the tokens read it
+    // from there.  dup: tokens are stored twice in the operand, the second copy's lanes take the upper half of the
+    // columns; else lanes 0..63 store everything.
     auto send_partial = [&](int N, bool dup) {
       wait_bar(bar_acc, n_acc);
       tc_fence_after();
       rb_begin();
       const int ncol = dup ? N / 2 : (half_t == 0 ? N : 0), col0 = dup ? half_t * (N / 2) : 0;
-      const uint32_t dst = rb_owner + (uint32_t)((rank * TPO + tl_t) * N + col0) * 4u;
+      const uint32_t dst = rb + (uint32_t)(tok_t * (N + 4) + col0) * 4u;
       for (int c0 = 0; c0 < ncol; c0 += 32) {                // (ncol is the same in all lanes of a warp)
         float v[32];
         tmem_ld32(trow + kFfColAcc + col0 + c0, v);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) ff_st_cluster_f4(dst + (uint32_t)(c0 + 4 * i) * 4u, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+        for (int i = 0; i < 8; ++i) ff_st_shared_f4(dst + (uint32_t)(c0 + 4 * i) * 4u, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
       }
       rb_sent();
       tc_fence_before();
       mbar_arrive(bar_accfree);
     };
-    // Sum over the sources of four consecutive columns of one of this CTA's tokens (fixed order).
+    // Sum over the CTAs of the cluster (fixed order) of four consecutive columns of one of this CTA's tokens.
     auto rb_sum4 = [&](int N, int tl, int col) -> float4 {
+      const uint32_t off = rb + (uint32_t)((tok0 + tl) * (N + 4) + col) * 4u;
+      float4 v[CS];
+#pragma unroll
+      for (int src = 0; src < CS; ++src) v[src] = ff_ld_cluster_f4(ff_mapa(off, (uint32_t)src));
       float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-      for (int src = 0; src < CS; ++src) {
-        const float4 v = *reinterpret_cast<const float4*>(rb_p + (src * TPO + tl) * N + col);
-        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
-      }
+      for (int src = 0; src < CS; ++src) { s.x += v[src].x; s.y += v[src].y; s.z += v[src].z; s.w += v[src].w; }
       return s;
     };
     // LayerNorm of this CTA's K-slice columns of rows x[0:M) into the operand tiles (each row stored at r and
@@ -735,7 +746,7 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
         group_stats(v, mu, q);
         if (mine && (wtid & 15) == 0 && m < M) a.stats_a[(long long)m * NC + c] = make_float2(mu, q);
       }
-      publish(kFfSyncXa);
+      publish(kFfSyncXa, false);
     }
 
     const int ntile = np_mine + ((rank == CS - 1 && nv > 0) ? 1 : 0);
@@ -760,29 +771,40 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
           const float4 b0v = __ldg(reinterpret_cast<const float4*>(bp)), b1v = __ldg(reinterpret_cast<const float4*>(bp + 4));
           const float v8[8] = {s0.x + b0v.x, s0.y + b0v.y, s0.z + b0v.z, s0.w + b0v.w, s1.x + b1v.x, s1.y + b1v.y, s1.z + b1v.z, s1.w + b1v.w};
           const uint4 val = ff_pack8(v8);
-          if (m < M) {
-            const uint32_t off = (uint32_t)m * 128u + ((uint32_t)((u & 7) ^ (m & 7)) << 4);
-            if (part == 0) {
-#pragma unroll
-              for (uint32_t p = 0; p < (uint32_t)CS; ++p) {
-                const uint32_t q_rem = ff_mapa(xa + off, p);
-                ff_st_cluster_u4(q_rem, val);
-                ff_st_cluster_u4(q_rem + 8192u, val);
-              }
-            } else {
-              ff_st_cluster_u4(ff_mapa(xa + (part == 1 ? 16384u : 24576u) + off, (uint32_t)(CS - 1)), val);
-              const long long row = s_kvrow[tl];
-              if (row >= 0) *reinterpret_cast<uint4*>(pool_l + row + (part - 1) * kv_stride + (long long)c * tile_elems + j0) = val;
-            }
+          // the row goes to this CTA's own shared memory ([token][q | k | v], 384 bytes), where the peers fetch it;
+          // k and v also go to the cache slot of the node
+          ff_st_shared_u4(qo + (uint32_t)(tl * 384 + u * 16), val);
+          if (m < M && part != 0) {
+            const long long row = s_kvrow[tl];
+            if (row >= 0) *reinterpret_cast<uint4*>(pool_l + row + (part - 1) * kv_stride + (long long)c * tile_elems + j0) = val;
           }
         }
-        // the tiles are read by the tensor cores of the peers
-        asm volatile("fence.proxy.async.shared::cluster;" ::: "memory");
         ff_fence_cluster();
         __syncwarp();
         if (lane == 0)
           for (uint32_t p = 0; p < (uint32_t)CS; ++p) ff_arrive_remote(ff_mapa(bar_qkv, p));
         rb_done();
+        // every owner has staged its rows: fetch the q rows of all tokens into the Q tile (each at r and r + 64) and,
+        // in the CTA that scores the tree's own keys, the k and v rows into their tiles
+        ff_wait([&] { return ff_try_wait_cluster(bar_qkv, n_qkv & 1); }, err, abort_flag);
+        ++n_qkv;
+        {
+          const int nparts = rank == CS - 1 ? 3 : 1;
+          for (int it = wtid; it < nparts * 512; it += kFfWorkers) {
+            const int part = it >> 9, m = (it >> 3) & 63, u = it & 7;
+            if (m < M) {
+              const int ow = ff_owner(m, 64, CS);
+              int of, oc;
+              ff_split(64, CS, ow, of, oc);
+              const uint4 val = ff_ld_cluster_u4(ff_mapa(qo + (uint32_t)((m - of) * 384 + part * 128 + u * 16), (uint32_t)ow));
+              const uint32_t off = (uint32_t)m * 128u + ((uint32_t)(u ^ (m & 7)) << 4);
+              if (part == 0) { ff_st_shared_u4(xa + off, val); ff_st_shared_u4(xa + 8192u + off, val); }
+              else ff_st_shared_u4(xa + (part == 1 ? 16384u : 24576u) + off, val);
+            }
+          }
+          fence_proxy_async_smem();
+          mbar_arrive(bar_q);
+        }
       }
       // ---------------------------------------------------------------- attention: this CTA's pages
       {
@@ -890,10 +912,10 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
         }
         rb_begin();
         {
-          const uint32_t dst = rb_owner + (uint32_t)(((rank * 2 + half_t) * TPO + tl_t) * 68) * 4u;
+          const uint32_t dst = rb + (uint32_t)(lane_t * 68) * 4u;      // [lane = copy * 64 + token][64 features, l, m, pad]
 #pragma unroll
-          for (int i = 0; i < 16; ++i) ff_st_cluster_f4(dst + 16u * i, oacc[4 * i], oacc[4 * i + 1], oacc[4 * i + 2], oacc[4 * i + 3]);
-          ff_st_cluster_f4(dst + 256u, l_run, m_run, 0.f, 0.f);
+          for (int i = 0; i < 16; ++i) ff_st_shared_f4(dst + 16u * i, oacc[4 * i], oacc[4 * i + 1], oacc[4 * i + 2], oacc[4 * i + 3]);
+          ff_st_shared_f4(dst + 256u, l_run, m_run, 0.f, 0.f);
         }
         rb_sent();
         tc_fence_before();
@@ -906,19 +928,23 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
             const int tl = (wtid >> 4) + 8 * rd, m = tok0 + tl;
             if (tl < ntok) {
               float mm[2 * CS], ll[2 * CS];
+              float4 ovv[2 * CS];
               float mxx = -INFINITY;
 #pragma unroll
-              for (int p = 0; p < 2 * CS; ++p) {
-                const float4 lm = *reinterpret_cast<const float4*>(rb_p + (p * TPO + tl) * 68 + 64);
+              for (int p = 0; p < 2 * CS; ++p) {            // partial p: CTA p / 2, copy p % 2 of the token
+                const uint32_t src = ff_mapa(rb + (uint32_t)(((p & 1) * 64 + m) * 68) * 4u, (uint32_t)(p >> 1));
+                const float4 lm = ff_ld_cluster_f4(src + 256u);
+                ovv[p] = ff_ld_cluster_f4(src + (uint32_t)f4 * 4u);
                 ll[p] = lm.x; mm[p] = lm.y;
-                mxx = fmaxf(mxx, lm.y);
               }
+#pragma unroll
+              for (int p = 0; p < 2 * CS; ++p) mxx = fmaxf(mxx, mm[p]);
               float Ls = 0.f;
               float4 o4 = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
               for (int p = 0; p < 2 * CS; ++p) {
                 const float w = (mm[p] == -INFINITY) ? 0.f : exp2f(mm[p] - mxx);
-                const float4 ov = *reinterpret_cast<const float4*>(rb_p + (p * TPO + tl) * 68 + f4);
+                const float4 ov = ovv[p];
                 Ls = fmaf(ll[p], w, Ls);
                 o4.x = fmaf(ov.x, w, o4.x); o4.y = fmaf(ov.y, w, o4.y); o4.z = fmaf(ov.z, w, o4.z); o4.w = fmaf(ov.w, w, o4.w);
               }
@@ -933,13 +959,13 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
             }
           }
         }
-        publish(kFfSyncO + c);
+        publish(kFfSyncO + c, true);
         rb_done();
       }
       // ---------------------------------------------------------------- output projection, rows [64c, 64c+64)
       send_partial(64, false);
       residual_epilogue(lvec(a.bo), a.xb, a.stats_b);
-      publish(kFfSyncXb);
+      publish(kFfSyncXb, false);
       rb_done();
       // ---------------------------------------------------------------- first feed-forward matrix, rows [c n1, (c+1) n1)
       build_ln(a.xb, a.stats_b, lvec(a.ln2_g), lvec(a.ln2_b), kFfSyncXb, (uint32_t)(G * (l + 1)), nullptr);
@@ -957,13 +983,13 @@ __global__ void __launch_bounds__(kFfThreads, 1) fused_forward_kernel(
                                fmaxf(s1.x + b1v.x, 0.f), fmaxf(s1.y + b1v.y, 0.f), fmaxf(s1.z + b1v.z, 0.f), fmaxf(s1.w + b1v.w, 0.f)};
           if (m < M) *reinterpret_cast<uint4*>(a.mid + (long long)m * F + c * n1 + 8 * u) = ff_pack8(v8);
         }
-        publish(kFfSyncMid + c);
+        publish(kFfSyncMid + c, true);
         rb_done();
       }
       // ---------------------------------------------------------------- second feed-forward matrix, rows [64c, 64c+64)
       send_partial(64, false);
       residual_epilogue(lvec(a.b2), a.xa, a.stats_a);
-      publish(kFfSyncXa);
+      publish(kFfSyncXa, false);
       rb_done();
     }
     // ---------------------------------------------------------------- final LayerNorm + vocabulary head

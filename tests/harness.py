@@ -72,6 +72,17 @@ def read_kv(g, table, b: int, S: int):
     return np.concatenate(Ks, axis=1).astype(np.float64), np.concatenate(Vs, axis=1).astype(np.float64)
 
 
+def read_kv_rows(g, table, b: int, positions):
+    """Rows [L, len(positions), H, dh] (float64) of sequence b at the given logical positions."""
+    view = g.kv_view()
+    Ks, Vs = [], []
+    for pos in positions:
+        blk, off = int(table[b, pos // 64]), pos % 64
+        Ks.append(view[:, blk, 0, :, off].float().cpu().numpy())
+        Vs.append(view[:, blk, 1, :, off].float().cpu().numpy())
+    return np.stack(Ks, axis=1).astype(np.float64), np.stack(Vs, axis=1).astype(np.float64)
+
+
 @dataclass
 class LockstepReport:
     iterations: int = 0
@@ -84,6 +95,7 @@ class LockstepReport:
     max_logit_err: float = 0.0
     max_attn_err: float = 0.0
     attn_checked: int = 0
+    decisions: int = 0               # iterations x followed sequences
     accept_lens: List[int] = field(default_factory=list)
     # acceptance tests by (draft head, rank) on the compared iterations: applied / passed
     tested: np.ndarray = field(default_factory=lambda: np.zeros((15, 16), dtype=np.int64))
@@ -202,6 +214,7 @@ def lockstep(g, table, model, states: Dict[int, "O.State"], template, sp_oracle,
     lens = g.lengths()
     for b, st in states.items():
         assert lens[b] == st.S
+    rep.decisions = rep.iterations * len(states)
     print(f"lockstep[{dtype}]: {rep.iterations} iterations, {len(states)} sequences; roots checked {rep.root_checked}, "
           f"draft heads fully checked {rep.draft_heads_checked}/{rep.draft_heads_total} (top-r sets {rep.draft_sets_checked}), "
           f"accept decisions checked {rep.accept_checked} (undecidable {rep.accept_undecidable}); "
@@ -209,6 +222,19 @@ def lockstep(g, table, model, states: Dict[int, "O.State"], template, sp_oracle,
           f"{(format(rep.max_attn_err, '.2e') + ' over ' + str(rep.attn_checked) + ' passes') if rep.attn_checked else 'not checked'}; "
           f"mean accepted {np.mean(rep.accept_lens):.2f}")
     return rep
+
+
+def assert_floors(rep: LockstepReport, root: float, accept: float, draft_sets_per_decision: float):
+    """A lockstep run counts for parity only as far as its decisions were decidable under the margin: at
+    least the given fractions of the root samples and acceptance decisions, and that many top-r candidate
+    sets per (iteration, sequence), must have been compared bit for bit."""
+    n = max(rep.decisions, 1)
+    msg = (f"decidable: roots {rep.root_checked}/{n}, accept decisions {rep.accept_checked}/{n}, "
+           f"draft top-r sets {rep.draft_sets_checked} ({rep.draft_sets_checked / n:.1f} per decision)")
+    print(msg)
+    assert rep.root_checked >= root * n, msg
+    assert rep.accept_checked >= accept * n, msg
+    assert rep.draft_sets_checked >= draft_sets_per_decision * n, msg
 
 
 def _clone_state(model, st):

@@ -7,7 +7,8 @@ import pytest
 
 import oracle as O
 import workloads as W
-from harness import (MARGIN, MARGINS, TOL, expected_slots, inject_kv, lockstep, make_gpu, read_kv, tokens_with_phonemes)
+from harness import (MARGIN, MARGINS, TOL, assert_floors, expected_slots, inject_kv, lockstep, make_gpu, read_kv,
+                     read_kv_rows, tokens_with_phonemes)
 
 pytestmark = pytest.mark.gpu
 
@@ -343,8 +344,8 @@ def test_six_draft_heads_accept_up_to_seven_tokens():
 
 
 def test_c1_generate_matches_oracle_and_plain_ar():
-    """BASELINE config 1 end to end: free-running vadusa_generate (greedy, tolerance 1, 100
-    tokens) equals the oracle's speculative decoding and plain AR decoding token for token
+    """Configuration 1 (2 layers, d 256, fp32, 16-node tree) end to end: free-running vadusa_generate (greedy,
+    tolerance 1, 100 tokens) equals the oracle's speculative decoding and plain AR decoding token for token
     up to the first position where the oracle's top-2 margin is below 1e-3."""
     torch = _torch()
     wl = W.workload("C1")
@@ -383,31 +384,63 @@ def test_c1_lockstep_full():
     states, _ = _prefill_both(wl, g, table, model, [0])
     so, sg = _sampling(wl)
     rep = lockstep(g, table, model, states, tpl, so, sg, 40, "fp32", oracle_mode="memo", check_attn=True)
-    assert rep.max_logit_err <= 1e-4 and rep.accept_checked >= 35
+    assert rep.max_logit_err <= 1e-4 and rep.accept_checked >= 35 and rep.attn_checked == 40
+    assert_floors(rep, root=0.8, accept=0.85, draft_sets_per_decision=3)
     g.check()
 
 
-def test_c2_lockstep_sampled_iterations():
-    """BASELINE config 2 (12 layers, d 1024, 64-node tree, tau 3, T 1.0): prefill of the
-    325-token prefix and the first iterations in lockstep."""
+def test_c2_lockstep_64_iterations():
+    """Configuration 2 (12 layers, d 1024, 16 heads, bf16, 64-node tree, tolerance 3, temperature 1.0): prefill
+    of the 325-token prefix, then 64 iterations in lockstep with the oracle's tree-masked pass, attention
+    outputs of every layer included.  Most decisions must be decidable under the bf16 margin."""
     wl = W.workload("C2")
-    w, model, tpl, g, table = _setup(wl, 4, [0])
+    w, model, tpl, g, table = _setup(wl, 64, [0])
     states, _ = _prefill_both(wl, g, table, model, [0])
     so, sg = _sampling(wl)
-    rep = lockstep(g, table, model, states, tpl, so, sg, 4, "bf16", oracle_mode="tree", check_attn=True)
-    assert rep.iterations == 4
+    rep = lockstep(g, table, model, states, tpl, so, sg, 64, "bf16", oracle_mode="tree", check_attn=True)
+    assert rep.iterations == 64 and rep.attn_checked == 64
+    assert_floors(rep, root=0.7, accept=0.5, draft_sets_per_decision=2)
     g.check()
 
 
-def test_c3_batch16_vocab2049_sampled_sequences():
-    """BASELINE config 3 (batch 16, vocab 2049, 42-node tree, tau 5, T 0.8): all sequences
-    run on the GPU, the oracle follows two of them."""
-    wl = W.workload("C3")
-    w, model, tpl, g, table = _setup(wl, 3, [0, 9])
-    states, _ = _prefill_both(wl, g, table, model, [0, 9])
+def test_c2_free_running_generate_matches_oracle_until_first_undecidable_iteration():
+    """Configuration 2, vadusa_generate running on its own (no override, no forced choice): its tokens equal
+    the oracle's speculative decoding up to the first iteration in which one of the oracle's decisions (root,
+    a used draft rank, an acceptance test) falls under the bf16 margin."""
+    torch = _torch()
+    wl = W.workload("C2")
+    n_tok = 28
+    w, model, tpl, g, table = _setup(wl, n_tok, [0])
+    states, _ = _prefill_both(wl, g, table, model, [0])
     so, sg = _sampling(wl)
-    rep = lockstep(g, table, model, states, tpl, so, sg, 3, "bf16", oracle_mode="tree")
-    assert rep.iterations == 3
+    traces = O.vadusa_generate(model, states[0], tpl, so, n_tok, mode="tree")
+    good = 0                                   # tokens committed before the first undecidable iteration
+    for t in traces:
+        if min(t.margin_root, t.margin_accept, float(t.margin_draft.min())) <= MARGINS["bf16"]:
+            break
+        good += t.accept_len
+    out = torch.full((1, n_tok), -1, dtype=torch.int32, device=g.dev)
+    out_len = torch.zeros(1, dtype=torch.int32, device=g.dev)
+    g.generate(sg, n_tok, out, out_len)
+    got = list(out.cpu().numpy()[0])
+    n = min(good, n_tok)
+    print(f"C2 free-running: {len(traces)} oracle iterations, {good} tokens before the first undecidable iteration")
+    assert got[:n] == states[0].tokens[:n]
+    assert n >= 3
+    g.check()
+
+
+def test_c3_batch16_vocab2049_all_sequences():
+    """Configuration 3 (batch 16, vocabulary 2049, 42-node tree, tolerance 5, temperature 0.8): the oracle
+    follows all 16 sequences for 8 iterations."""
+    wl = W.workload("C3")
+    seqs = list(range(wl.batch))
+    w, model, tpl, g, table = _setup(wl, 8, seqs)
+    states, _ = _prefill_both(wl, g, table, model, seqs)
+    so, sg = _sampling(wl)
+    rep = lockstep(g, table, model, states, tpl, so, sg, 8, "bf16", oracle_mode="tree", check_attn=True)
+    assert rep.iterations == 8 and rep.decisions == 128
+    assert_floors(rep, root=0.7, accept=0.5, draft_sets_per_decision=2)
     g.check()
 
 
@@ -419,16 +452,25 @@ def _random_context(model, S, rng, scale=1.0):
 
 @pytest.mark.parametrize("name", ["C4", "C5"])
 def test_long_ragged_contexts_with_injected_kv(name):
-    """BASELINE configs 4 and 5 at full batch and context lengths: the KV cache holds
-    seeded random bf16 rows (so no prefill is needed on either side), tree tokens and the
-    carried state are random; the oracle scores four sampled sequences (shortest, longest,
-    two others).  C5 uses a random topology per sequence."""
+    """Configurations 4 (batch 32, contexts 1000-4000, shared 64-node tree) and 5 (batch 64, contexts 256-3000, a
+    random topology per sequence) at full batch and context lengths: the KV cache holds seeded random bf16 rows
+    (so no prefill is needed on either side), tree tokens and the carried state are random; the oracle scores
+    four sampled sequences (shortest, longest, two others).  Configuration 4 goes on with the tolerance sweep
+    {1, 3, 5} from the same state (draws of the oracle planted below the root, so that the accepted sets differ
+    and grow with the tolerance, Sec. III-B) and with a forced five-token path whose committed K/V rows are read
+    back, one of them across a page boundary behind a context of almost 4000 tokens."""
     torch = _torch()
     wl = W.workload(name)
     w = W.make_weights(wl.shape, wl.seed())
     model = O.Model.from_shape(wl.shape, w)
     B, N = wl.batch, wl.tree_nodes
     lens = W.ragged_lengths(B, wl.context_len[0], wl.context_len[1], wl.seed(900))
+    if name == "C4":
+        # the longest context ends three rows before a page boundary: a five-token commit crosses it
+        lens = lens.copy()
+        b_edge = int(np.argmax(lens))
+        lens[b_edge] = (int(lens[b_edge]) // 64) * 64 - 3
+        assert lens[b_edge] > 3700
     g, table = make_gpu(wl.shape, w, B, N, [int(s) + N + 8 for s in lens], wl.seed(1))
     g.begin(table, ctx_len=lens)
     if wl.random_topology:
@@ -445,6 +487,8 @@ def test_long_ragged_contexts_with_injected_kv(name):
     def both_halves(ps):
         return {b % 4 < 2 for b in ps} == {True, False} and {b % 2 for b in ps} == {0, 1}
     picks.append(next(b for b in range(B) if b not in picks and both_halves(picks + [b])))
+    if name == "C4" and b_edge not in picks:
+        picks.append(b_edge)
     rng = np.random.default_rng(wl.seed(2))
     # every sequence gets random K/V on the GPU; the sampled ones also in the oracle
     view = g.kv_view()
@@ -490,6 +534,79 @@ def test_long_ragged_contexts_with_injected_kv(name):
             assert int(acc[b]) == len(path) and list(pn[b, :len(path)].cpu().numpy()) == path
             assert list(sl[b, :len(path)].cpu().numpy()) == expected_slots(table, b, S, len(path))
     assert np.array_equal(g.lengths(), lens + acc.cpu().numpy())
+    g.check()
+    if name != "C4":
+        return
+    # ---- tolerance sweep from the same state: the 1st, 3rd and 5th draw of the oracle at the root planted as
+    # the first three candidates below it
+    tpl = tpls[0]
+    d1 = [n for n in range(N) if tpl.depth[n] == 1]
+    toks2 = toks.copy()
+    outs = {}
+    for b in picks:
+        S = int(lens[b])
+        mask = np.zeros((N, N), dtype=bool)
+        for n in range(N):
+            mask[n, tpl.node_path(n)] = True
+        root_logits = O.forward_tree(model, states[b], [0] * N, toks[b], S + tpl.depth, mask).logits[0]
+        d5 = O.draws_at(model, root_logits, O.Sampling(tau=5, temperature=so.temperature, seed=so.seed), b, S + 1)
+        assert len(d5) == 5
+        toks2[b, d1[0]], toks2[b, d1[1]], toks2[b, d1[2]] = d5[0], d5[2], d5[4]
+        outs[b] = O.forward_tree(model, states[b], [0] * N, toks2[b], S + tpl.depth, mask)
+    dev_toks2 = torch.from_numpy(toks2).to(g.dev)
+    got = {}
+    checked = 0
+    for tau in (1, 3, 5):
+        so_t, sg_t = _sampling(wl, seed=5, tau=tau)
+        g.begin(table, ctx_len=lens)
+        g.verify_step(override=dev_toks2)
+        g.accept_and_commit(sg_t, accept_len=acc, path_nodes=pn, edge_bits=eb)
+        got[tau] = (acc.cpu().numpy().copy(), eb.cpu().numpy().astype(np.uint64).copy())
+        for b in picks:
+            S, out = int(lens[b]), outs[b]
+            draws = {n: O.draws_at(model, out.logits[n], so_t, b, S + int(tpl.depth[n]) + 1) for n in range(N)}
+            ok = O.tree_edge_accepts(tpl.parent, toks2[b], draws)
+            best, path = O.accept_from_edges(tpl.parent, tpl.depth, ok)
+            accd = {0}
+            want_bits = 1
+            margin = float("inf")
+            for n in range(1, N):
+                p = int(tpl.parent[n])
+                if p in accd:
+                    margin = min(margin, O.decode._edge_margin(model, out.logits[p], so_t, b, S + int(tpl.depth[p]) + 1, int(toks2[b, n])))
+                    if ok[n]:
+                        accd.add(n); want_bits |= 1 << n
+            if margin > MARGINS["bf16"]:
+                assert int(got[tau][0][b]) == len(path) and list(pn[b, :len(path)].cpu().numpy()) == path
+                assert int(got[tau][1][b]) == want_bits, f"tau {tau} seq {b}: {int(got[tau][1][b]):x} != {want_bits:x}"
+                assert len(path) >= 2 and (want_bits >> d1[0]) & 1            # the first draw is accepted at any tolerance
+                checked += 1
+    print(f"C4 tolerance sweep: {checked} of {3 * len(picks)} decisions decidable")
+    assert checked >= 6
+    # a larger tolerance accepts a superset of edges below the same accepted nodes and never a shorter path
+    for lo, hi in ((1, 3), (3, 5)):
+        assert np.all(got[lo][0] <= got[hi][0])
+        assert np.all((got[lo][1] & ~got[hi][1]) == 0)
+    for b in picks:
+        assert bin(int(got[5][1][b])).count("1") > bin(int(got[1][1][b])).count("1")
+    # ---- a forced five-token path: the committed rows, read back behind up to 3965 context tokens
+    leaf = int(np.nonzero(tpl.depth == tpl.max_depth)[0][0])
+    path = tpl.node_path(leaf)
+    g.begin(table, ctx_len=lens)
+    g.verify_step(override=dev_toks2)
+    forced = torch.full((B,), leaf, dtype=torch.int32, device=g.dev)
+    g.accept_and_commit(sg, forced_best=forced, accept_len=acc, path_nodes=pn, kv_slots=sl)
+    assert np.all(acc.cpu().numpy() == len(path))
+    crossed = 0
+    for b in picks:
+        S = int(lens[b])
+        assert list(pn[b, :len(path)].cpu().numpy()) == path
+        assert list(sl[b, :len(path)].cpu().numpy()) == expected_slots(table, b, S, len(path))
+        K, V = read_kv_rows(g, table, b, range(S, S + len(path)))
+        assert np.abs(K - outs[b].K[:, path]).max() <= TOL["bf16"] and np.abs(V - outs[b].V[:, path]).max() <= TOL["bf16"]
+        crossed += int(S // 64 != (S + len(path) - 1) // 64)
+    assert crossed >= 1
+    assert np.array_equal(g.lengths(), lens + len(path))
     g.check()
 
 

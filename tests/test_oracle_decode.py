@@ -232,7 +232,7 @@ def test_accept_rule_plain_topk_ignores_noise_for_membership():
 
 
 def test_full_config_c1_speculative_equals_ar():
-    """BASELINE config 1 (2 layers, d 256, 16-node tree, greedy, tolerance 1, 100 tokens)."""
+    """Configuration 1 (2 layers, d 256, 16-node tree, greedy, tolerance 1, 100 tokens)."""
     wl = W.workload("C1")
     m = O.Model.from_shape(wl.shape, W.make_weights(wl.shape, wl.seed()))
     ph, pr = W.prefix_for(wl, 0)

@@ -6,7 +6,8 @@ once it runs, a process whose device memory was given away before the library wa
 For them the draft heads' top-k exists in a form whose scratch is a fixed array inside the
 library.  This test feeds both forms the same weights and the same hidden state and expects
 the same candidate ids, twice in a row (the second call finds the first call's leftovers in
-the shared array), and checks that oversize requests are refused with a clear message.
+the shared array); the ids are also held against the CPU oracle's draft heads wherever the
+oracle's logit gaps decide them; oversize requests must be refused with a clear message.
 It runs last so that a failure here cannot hide a failure elsewhere.
 """
 import ctypes as C
@@ -14,6 +15,7 @@ import ctypes as C
 import numpy as np
 import pytest
 
+import oracle as O
 import workloads as W
 
 pytestmark = pytest.mark.gpu
@@ -44,6 +46,10 @@ def test_static_scratch_draft_matches_regular_draft_twice(dtype):
     du = blob[info["draft0.u"].offset:]
     K = g.cfg.draft_topk
     sp = P.Sampling.make(tau=1, temperature=0.0)
+    model = O.Model.from_shape(sh, w)
+    so = O.Sampling(tau=1, temperature=0.0)
+    from harness import MARGINS
+    checked = 0
     rng = np.random.default_rng(5)
     for call in range(2):
         h = torch.from_numpy(rng.standard_normal((wl.batch, sh.d_model)).astype(np.float32)).to(g.dev).to(g.tdtype)
@@ -56,6 +62,21 @@ def test_static_scratch_draft_matches_regular_draft_twice(dtype):
         P.draft_topk_static(dw, db, du, h, g.cfg.dtype, wl.batch, sh.d_model, sh.vocab, sh.n_draft_heads, K, True, got)
         torch.cuda.synchronize()
         want, got = want.cpu().numpy(), got.cpu().numpy()
+        # against the oracle's draft heads: the r + 1 best candidates are decided when the logit gap behind
+        # them exceeds the margin of the dtype, a single rank when the gaps on both sides do
+        hs = h.float().cpu().numpy().astype(np.float64)
+        for b in range(wl.batch):
+            ref = O.draft_topk(model, hs[b], K, so)
+            dl = O.draft_logits(model, hs[b])
+            for hd in range(sh.n_draft_heads):
+                srt = np.sort(O.sampling.masked_logits32(dl[hd], model.eos_id, True).astype(np.float64))[::-1]
+                gaps = srt[:K] - srt[1:K + 1]
+                for r in range(K):
+                    if gaps[r] > MARGINS[dtype]:
+                        assert set(got[b, hd, :r + 1]) == set(ref[hd, :r + 1]), f"call {call} seq {b} head {hd} top-{r + 1}"
+                        checked += 1
+                        if r == 0 or gaps[r - 1] > MARGINS[dtype]:
+                            assert got[b, hd, r] == ref[hd, r], f"call {call} seq {b} head {hd} rank {r}"
         if dtype == "fp32":
             assert np.array_equal(got, want), f"call {call}"
         else:
@@ -66,6 +87,7 @@ def test_static_scratch_draft_matches_regular_draft_twice(dtype):
                 for hd in range(sh.n_draft_heads):
                     assert len(set(got[b, hd]) & set(want[b, hd])) >= K - 1, f"call {call} seq {b} head {hd}"
                     assert got[b, hd, 0] in want[b, hd, :2]
+    assert checked > (40 if dtype == "fp32" else 4), checked
     g.close()
 
 
