@@ -273,6 +273,22 @@ def run_ours(args):
     tokens = int(g.lengths()[0]) - len0
     g.check()
 
+    # ---- per-step latency and accepted length (separate pass: one event per step, lengths read back after each)
+    n_lat = min(K, 200)
+    ev_a = [torch.cuda.Event(enable_timing=True) for _ in range(n_lat)]
+    ev_b = [torch.cuda.Event(enable_timing=True) for _ in range(n_lat)]
+    step_lens = []
+    prev_len = int(g.lengths()[0])
+    for i in range(n_lat):
+        ev_a[i].record()
+        steps(1)
+        ev_b[i].record()
+        cur = int(g.lengths()[0])                   # synchronises (outside the two events)
+        step_lens.append(cur - prev_len)
+        prev_len = cur
+    lat_us = sorted(ev_a[i].elapsed_time(ev_b[i]) * 1e3 for i in range(n_lat))
+    hist = {str(k): int(v) for k, v in zip(*np.unique(step_lens, return_counts=True))}
+
     # ---- per-kernel times of the same steps (events around every launch; separate pass)
     n_prof = min(K, 50)
     g.profile_begin()
@@ -305,6 +321,28 @@ def run_ours(args):
     pl_ms = p0.elapsed_time(p1)
     pl_tokens = int(g.lengths()[0]) - pl0
     g.check()
+
+    # ---- the same step with the verify pass as one persistent kernel (an alternative path of the library)
+    persistent = None
+    try:
+        g.set_fused_pass(1)
+        fresh()
+        steps(Wm)
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_f = min(K, 100)
+        barrier()
+        f0.record()
+        steps(n_f)
+        f1.record()
+        barrier()
+        g.check()
+        if g.fused_pass_clusters() >= wl.shape.n_heads:
+            persistent = {"what": "verify pass as one persistent kernel (vadusa_set_fused_pass(1)); this rank only",
+                          "ms_per_step": f0.elapsed_time(f1) / n_f, "steps": n_f,
+                          "clusters_resident": g.fused_pass_clusters()}
+    finally:
+        g.set_fused_pass(0)
+    fresh()
 
     # ---- end to end through the host-buffer entry: prefix from host memory, tokens back to host
     h_out = np.zeros((1, gen_cap), dtype=np.int32)
@@ -344,6 +382,20 @@ def run_ours(args):
         achieved = gemm_alg_per_step / (ms / K * 1e-3 * gemm_share) / 1e9 if gemm_ms > 0 else 0.0
         cores = os.cpu_count() or 1
         cpu_val, _, cpu_sample, _ = _oracle_run(wl, weights, tpl, ph, pr, steps=2, warmup=0, budget_s=30.0)
+        c5 = None
+        if world == 1 and not args.no_c5:
+            # the batch-64 microbenchmark (configuration 5), measured after the headline region: tree attention
+            # against the HBM roofline, the many-token products against the tensor roofline
+            g.close()
+            import copy
+            a5 = copy.copy(args)
+            a5.steps, a5.warmup, a5.batch = 20, 3, 0
+            l5 = measure_c5(a5)
+            c5 = {"workload": l5["config"]["workload"], "ms_per_step": l5["ms_per_step"],
+                  "attention": {k: l5["roofline"][k] for k in ("bound", "achieved", "peak", "unit", "frac", "traffic",
+                                                              "avg_launch_us", "algorithmic_bytes_per_launch")},
+                  "products": l5["tensor_roofline"], "kernel_time_shares": l5["roofline"]["kernel_time_shares"],
+                  "clocks": l5["clocks"]}
         line = {
             "metric": "generated speech tokens/s", "value": tokens / (ms * 1e-3), "unit": "tokens/s",
             "n_gpus": world, "steps": K, "warmup": Wm, "ms_per_step": ms / K, "higher_is_better": True,
@@ -369,6 +421,12 @@ def run_ours(args):
                     "h2d_bytes_per_step": len(prefix) * 4 / e2e_iters, "d2h_bytes_per_step": (gen_cap + 1) * 4 / e2e_iters,
                     "what": f"vadusa_generate_host: prefix from pinned host memory, prefill, {gen_cap} tokens, tokens back to host"},
             "gpu_launches": launches, "clocks": clocks,
+            "step_latency_us": {"p50": lat_us[len(lat_us) // 2], "p99": lat_us[min(len(lat_us) - 1, int(0.99 * len(lat_us)))],
+                                "max": lat_us[-1], "steps": n_lat,
+                                "what": "CUDA events around single steps (separate pass; a host read-back between steps)"},
+            "accepted_length_histogram": hist,
+            "persistent_pass": persistent,
+            "c5": c5,
         }
         print(json.dumps(line))
     g.close()
@@ -376,7 +434,7 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def run_c5(args):
+def measure_c5(args):
     """Verify-step microbenchmark of configuration 5: batch 64, ragged KV lengths 256-3000, a random
     64-node topology per sequence, random bf16 K/V and tokens.  One step = draft heads + verify pass +
     accept/commit.  Reports per-kernel roofline fractions (attention: HBM; projections: bf16 tensor)."""
@@ -462,8 +520,12 @@ def run_c5(args):
                          "kernel_time_shares": {k: round(v[1] / tot_ms, 4) for k, v in sorted(prof.items(), key=lambda kv: -kv[1][1])}},
             "tensor_roofline": {"peak_tflops": tf_peak, "peak_source": "measured sustained bf16 matmul", "kernels": gemm},
             "cpu_baseline": None, "e2e": None, "gpu_launches": launches, "clocks": clocks}
-    print(json.dumps(line))
     g.close()
+    return line
+
+
+def run_c5(args):
+    print(json.dumps(measure_c5(args)))
 
 
 def run_batch(args):
@@ -544,6 +606,7 @@ def main():
                     help="C3, C4: prefix chunks of 64 tokens scored per prefill pass (0: one per sequence)")
     ap.add_argument("--tree-nodes", type=int, default=0, choices=[0, 64, 96, 128],
                     help="C2 only: candidate-tree size (default: the workload's 64 nodes)")
+    ap.add_argument("--no-c5", action="store_true", help="C2 only: skip the batch-64 microbenchmark that follows the headline region")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=5)

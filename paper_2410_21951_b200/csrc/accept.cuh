@@ -50,6 +50,7 @@ __global__ void __launch_bounds__(256) accept_kernel(
   __shared__ int s_first[kMaxPath + 2];    // nodes are ordered by depth: first node of every depth, then nv
   __shared__ Best bscratch[32];
   __shared__ float fscratch[32];
+  __shared__ int s_scan[256];
 
   const int b = blockIdx.x, N = tree.n_nodes, nv = st.nvalid[b];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -104,19 +105,45 @@ __global__ void __launch_bounds__(256) accept_kernel(
       const bool noise = sp.accept_rule == 0;
       for (int j = tid; j < vocab; j += blockDim.x) keys[j] = key_of(row[j], j, rs, sp, noise);
       if (nuc) {
-        // Tokens outside the top-p nucleus cannot be drawn: give them the key -inf.  A token is
-        // inside iff the probability mass ahead of it (larger logit, or equal and lower id) is
-        // below top_p; probs[] holds exp((l - max) / T).
+        // Tokens outside the top-p nucleus cannot be drawn: give them the key -inf.  In the order "larger logit,
+        // then lower id" the nucleus is the prefix of tokens whose mass ahead of them is below top_p.  The mass
+        // strictly above a logit value falls as the value grows, so the smallest value v* whose mass above is
+        // still below top_p is found by bisection on the ordered bit pattern of the value (32 block-wide sums
+        // instead of one pass per token); tokens above v* are inside, tokens below it outside, and the tokens
+        // AT v* (equal logits, equal probability p*) are inside while (mass above v*) + (ties with a lower
+        // id) * p* stays below top_p.  probs[] holds exp((l - max) / T).
         const RowStats rst = row_stats(row, vocab, sp, fscratch);
         for (int j = tid; j < vocab; j += blockDim.x)
           probs[j] = expf((masked_logit(row[j], j, sp) - rst.maxl) * sp.inv_temperature);
         __syncthreads();
-        for (int j = tid; j < vocab; j += blockDim.x) {
-          const float lj = masked_logit(row[j], j, sp);
+        const float limit = sp.top_p * rst.z;
+        auto mass_above = [&](uint32_t k) -> float {              // sum of p over tokens whose value orders above k
           float m = 0.f;
-          for (int i = 0; i < vocab; ++i)
-            if (precedes(masked_logit(row[i], i, sp), i, lj, j)) m += probs[i];
-          if (!(m / rst.z < sp.top_p)) keys[j] = -INFINITY;
+          for (int j = tid; j < vocab; j += blockDim.x)
+            if (ordered_bits(masked_logit(row[j], j, sp)) > k) m += probs[j];
+          return block_sum(m, fscratch);
+        };
+        uint32_t lo = 0u, hi = 0xffffffffu;                       // mass_above(hi) = 0 < limit: v* in (lo, hi]
+        if (mass_above(0u) < limit) hi = 0u;                      // (everything is inside)
+        while (hi - lo > 1u) {
+          const uint32_t mid = lo + ((hi - lo) >> 1);
+          if (mass_above(mid) < limit) hi = mid; else lo = mid;
+        }
+        const float above = mass_above(hi);
+        // ties at v*: exclusive count of earlier ids with the same value, by contiguous chunks of ids
+        const int chunk = (vocab + (int)blockDim.x - 1) / (int)blockDim.x, j0 = tid * chunk, j1 = min(vocab, j0 + chunk);
+        int mine = 0;
+        for (int j = j0; j < j1; ++j) mine += ordered_bits(masked_logit(row[j], j, sp)) == hi ? 1 : 0;
+        __syncthreads();
+        s_scan[tid] = mine;
+        __syncthreads();
+        int before = 0;
+        for (int t = 0; t < tid; ++t) before += s_scan[t];
+        for (int j = j0; j < j1; ++j) {
+          const uint32_t kj = ordered_bits(masked_logit(row[j], j, sp));
+          bool inside = kj > hi;
+          if (kj == hi) { inside = above + (float)before * probs[j] < limit; ++before; }
+          if (!inside) keys[j] = -INFINITY;
         }
       }
       __syncthreads();
