@@ -539,7 +539,7 @@ def run_batch(args):
     sh = wl.shape
     weights = W.make_weights(sh, wl.seed())
     tpl = W.static_template(wl.tree_nodes, wl.tree_caps)
-    B = wl.batch
+    B = min(args.batch, wl.batch) if args.batch else wl.batch      # (a smaller batch: the first sequences; profiler captures)
     prefixes = [W.prefix_for(wl, b) for b in range(B)]
     toks = [np.concatenate([ph.astype(np.int32) + sh.vocab, pr.astype(np.int32)]) for ph, pr in prefixes]
     iters = wl.iterations if wl.iterations else wl.gen_tokens
@@ -601,7 +601,7 @@ def main():
     ap.add_argument("--workload", default="C2", choices=["C2", "C3", "C4", "C5"],
                     help="C2: the headline step (default); C3, C4: the batched configurations; C5: verify-step "
                          "microbenchmark at batch 64")
-    ap.add_argument("--batch", type=int, default=0, help="C5 only: smaller batch (for profiler captures)")
+    ap.add_argument("--batch", type=int, default=0, help="C3, C4, C5: smaller batch (for profiler captures)")
     ap.add_argument("--prefill-rows", type=int, default=64,
                     help="C3, C4: prefix chunks of 64 tokens scored per prefill pass (0: one per sequence)")
     ap.add_argument("--tree-nodes", type=int, default=0, choices=[0, 64, 96, 128],

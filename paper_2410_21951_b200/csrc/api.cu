@@ -14,6 +14,7 @@
 #include "accept.cuh"
 #include "attention_simt.cuh"
 #include "attention_tc.cuh"
+#include "attention_prefill_tc.cuh"
 #include "elementwise.cuh"
 #include "fwd_fused.cuh"
 #include "gemm_simt.cuh"
@@ -47,6 +48,7 @@ struct vadusa_ctx {
   int tree_per_seq = 0;
   int max_rank_used = 0;
   int tree_max_depth = 0;
+  int pf_tiles = 0;           // > 0 while a prefill pass runs: attention CTAs of the pass (pairs of chunks), listed in ws.pf_pairs
   int fused_enabled = 0;      // single-sequence passes run as one persistent kernel (0: no, 1: yes, 6 / 8: with that cluster size)
   int fused_clusters = -1;    // clusters of that kernel that can be resident at once on this device (-1: not asked yet)
   int fused_cs = -1;          // CTAs per cluster chosen for it (8 or 6; 0: the device cannot hold one cluster per head)
@@ -446,6 +448,34 @@ vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeVi
   };
   if constexpr (std::is_same<T, bf16>::value) {
     if (dh == 64) {
+      if (ctx->pf_tiles > 0 && tv.n_nodes == 64) {
+        // prefill pass: two consecutive chunks of a sequence per CTA (128 query rows per K/V page fetched)
+        const CUtensorMap *mq, *mkv;
+        const int M = ctx->batch * tv.n_nodes;
+        if (vadusa_status s = tensor_map(ctx, q, M, c.d_model, 64, 1, 0, &mq)) return s;
+        const long long rows = (long long)c.kv_num_blocks * 2 * c.n_heads * kKvBlock;
+        if (rows > 0x7fffffffLL) return fail(ctx, VADUSA_EINVAL, "KV pool too large for one tensor map");
+        if (vadusa_status s = tensor_map(ctx, c.kv_pool, (int)rows, 64, 64, c.n_layers, g.layer_stride, &mkv)) return s;
+        const int layer = (int)((reinterpret_cast<const char*>(pool) - reinterpret_cast<const char*>(c.kv_pool)) /
+                                (g.layer_stride * (long long)sizeof(bf16)));
+        cudaLaunchConfig_t lc = {};
+        lc.gridDim = dim3(c.n_heads, ctx->pf_tiles, 1);
+        lc.blockDim = dim3(kPfThreads);
+        lc.dynamicSmemBytes = kAttSmemBytes;
+        lc.stream = ctx->stream;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = at; lc.numAttrs = 1;
+        PROF(ctx, K_ATTENTION);
+        CU(cudaLaunchKernelEx(&lc, prefill_attention_tc_kernel, *mq, *mkv, layer, ctx->block_table,
+                              (const int32_t*)wsptr<int32_t>(ctx, ctx->ws.ctx_len),
+                              (const int32_t*)wsptr<int32_t>(ctx, ctx->ws.nvalid),
+                              (const int2*)wsptr<int2>(ctx, ctx->ws.pf_pairs), g, c.d_model,
+                              scale * 1.4426950408889634f, reinterpret_cast<bf16*>(out), err_word(ctx)));
+        LAUNCH_CHECK();
+        return VADUSA_OK;
+      }
       // tensor-core kernel; KV splits so that about two CTAs per SM exist even at batch 1
       const int splits = attention_splits(ctx, tv.n_nodes);
       const CUtensorMap *mq, *mkv;
@@ -794,7 +824,7 @@ vadusa_status prefill(vadusa_ctx* ctx, const int32_t* h_tokens, const int32_t* h
   int32_t* d_table = wsptr<int32_t>(ctx, ctx->ws.pf_block_table);
   int32_t* real_ctx_len = wsptr<int32_t>(ctx, ctx->ws.ctx_len);
   const int32_t* real_table = ctx->block_table;
-  std::vector<int32_t> stage((size_t)R * N), v_ctx(R), v_nv(R), v_seq(R), v_last(R);
+  std::vector<int32_t> stage((size_t)R * N), v_ctx(R), v_nv(R), v_seq(R), v_last(R), v_pairs(2 * (size_t)R);
   const TreeView tv = tree_of(ctx, true);
   for (size_t c0 = 0; c0 < chunks.size(); c0 += R) {
     const int rows = (int)(chunks.size() - c0 < (size_t)R ? chunks.size() - c0 : R);
@@ -808,12 +838,25 @@ vadusa_status prefill(vadusa_ctx* ctx, const int32_t* h_tokens, const int32_t* h
     CU(cudaMemcpyAsync(d_seq, v_seq.data(), rows * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream));
     CU(cudaMemcpyAsync(d_last, v_last.data(), rows * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream));
     CU(cudaMemcpyAsync(d_stage, stage.data(), (size_t)rows * N * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream));
+    // attention tiles of the pass: a full chunk and the chunk behind it in the same sequence share a CTA
+    int tiles = 0;
+    for (int r = 0; r < rows;) {
+      const Chunk& ch = chunks[c0 + r];
+      const bool pair = r + 1 < rows && chunks[c0 + r + 1].b == ch.b && ch.n == N;
+      v_pairs[2 * tiles] = r; v_pairs[2 * tiles + 1] = pair ? r + 1 : -1;
+      ++tiles;
+      r += pair ? 2 : 1;
+    }
+    CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.pf_pairs, v_pairs.data(), (size_t)tiles * 8, cudaMemcpyHostToDevice, ctx->stream));
     CU(cudaStreamSynchronize(ctx->stream));   // the staging vectors are reused by the next pass
     prefill_gather_kernel<<<rows, 128, 0, ctx->stream>>>(real_table, d_seq, c.max_blocks_per_seq, d_table);
     LAUNCH_CHECK();
     {
       RowsView view(ctx, rows, d_table, ctx->ws.pf_ctx_len, ctx->ws.pf_nvalid);
-      if (vadusa_status s = forward<T>(ctx, tv, d_stage, nullptr)) return s;
+      ctx->pf_tiles = tiles;
+      const vadusa_status s = forward<T>(ctx, tv, d_stage, nullptr);
+      ctx->pf_tiles = 0;
+      if (s) return s;
     }
     prefill_finish_kernel<T><<<rows, 256, 0, ctx->stream>>>(d_ctx, d_nv, d_last, N, wsptr<T>(ctx, ctx->ws.hfinal), c.d_model,
                                                             wsptr<float>(ctx, ctx->ws.logits), vp,
@@ -834,6 +877,8 @@ vadusa_status set_kernel_attributes(vadusa_ctx* ctx) {
   CU(cudaFuncSetAttribute(tree_attention_simt_kernel<bf16, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(64)));
   CU(cudaFuncSetAttribute(tree_attention_simt_kernel<bf16, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(32)));
   CU(cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmemBytes));
+  CU(cudaFuncSetAttribute(prefill_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmemBytes));
+  CU(cudaFuncSetAttribute(prefill_attention_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
   // the accept kernel keeps one row of keys and one of probabilities in shared memory.  The limit is an attribute of
   // the function on this device, shared by every context: always the library's largest vocabulary
   CU(cudaFuncSetAttribute(accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 24576 * (int)sizeof(float)));

@@ -189,6 +189,9 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
   if (warp == 1 && lane == 0) {
     // ---- MMA issuer
     constexpr uint32_t idesc = umma_idesc_bf16(kGemmRowsW, TN < 16 ? 16 : TN);
+    // the token operand is requested only after the upstream grid has finished: wait for that first, so that the
+    // bounded waits below time this kernel's own pipeline and not the upstream kernel's run time
+    grid_dep_wait();
     for (int i = 0; i < nchunks; ++i) {
       const int s = i % S;
       if (!mbar_wait(full0 + 8 * s, (i / S) & 1, err)) break;

@@ -119,6 +119,7 @@ struct WorkspaceLayout {
   // prefill: one row per prefix chunk of a pass (R = pass_rows)
   int64_t pf_ctx_len, pf_nvalid, pf_seq, pf_last;   // int32 [R]: tokens before the chunk, its length, its sequence, sequence if last chunk else -1
   int64_t pf_block_table;                // int32 [R][max_blocks_per_seq]: the block-table row of the chunk's sequence
+  int64_t pf_pairs;                      // int2 [R]: rows that share an attention CTA during prefill (y < 0: a single chunk)
   // single-sequence pass in one persistent kernel: residual stream after the attention block, LayerNorm statistics
   // per (token, group of 64 features) of both residual buffers, counters of the exchanges between clusters
   int64_t f_xb, f_stats_a, f_stats_b, f_sync;    // fp32 [64][d], float2 [64][d/64] x 2, uint32 [64]
@@ -158,6 +159,7 @@ inline WorkspaceLayout workspace_layout(const vadusa_config* c) {
   w.gen_out = take(B * kGenHostCap * 4); w.gen_len = take(B * 4);
   w.pf_ctx_len = take(R * 4); w.pf_nvalid = take(R * 4); w.pf_seq = take(R * 4); w.pf_last = take(R * 4);
   w.pf_block_table = take(R * (int64_t)c->max_blocks_per_seq * 4);
+  w.pf_pairs = take(R * 8);
   w.f_xb = take(64 * d * 4);
   w.f_stats_a = take(64 * (d / 64 + 1) * 8); w.f_stats_b = take(64 * (d / 64 + 1) * 8);
   w.f_sync = take(256);

@@ -113,6 +113,49 @@ def test_prefill_in_passes_of_many_chunks_and_behind_existing_context(dtype, row
     g.check()
 
 
+def test_prefill_of_4000_tokens_bf16_pairs_of_chunks():
+    """The prefilling pass (Fig. 1a) over long prefixes with 64-token chunks, head_dim 64, bf16: attention runs on
+    pairs of consecutive chunks (128 query rows per K/V page).  Two sequences of 4000 and 1531 tokens, fed in two
+    calls (the first leaves 37 and 64 tokens, so the second call's chunks start at unaligned and at aligned
+    positions, and one sequence has an odd number of chunks): every K/V row and the carried state (through the
+    first iteration's logits and decisions) against the oracle."""
+    import paper_2410_21951_b200 as P
+    wl = W.toy_workload(dtype="bf16", d_model=128, n_heads=2, d_ffn=256, vocab=203, tree_nodes=64, tree_caps=(10, 5, 3),
+                        tau=3, temperature=1.0, batch=2, phoneme_len=(60, 100), prompt_len=1471, index=23, max_pos=4200)
+    w = W.make_weights(wl.shape, wl.seed())
+    model = O.Model.from_shape(wl.shape, w)
+    tpl = W.static_template(wl.tree_nodes, wl.tree_caps)
+    prefixes = [W.prefix_for(wl, b) for b in range(wl.batch)]
+    # sequence 0: a longer prompt (4000 tokens in all)
+    ph0 = prefixes[0][0]
+    prefixes[0] = (ph0, W.markov_prompt(4000 - len(ph0), wl.shape.vocab - 1, wl.seed(50)))
+    toks = [tokens_with_phonemes(wl.shape, ph, pr) for ph, pr in prefixes]
+    assert len(toks[0]) == 4000
+    need = [len(t) + 2 * (tpl.max_depth + 1) + wl.tree_nodes for t in toks]
+    table, total = W.shuffled_block_table(need, 64, 29, spare_pages=2)
+    g = P.Vadusa(wl.shape, w, max_batch=wl.batch, max_tree_nodes=wl.tree_nodes, max_blocks_per_seq=table.shape[1],
+                 kv_num_blocks=total, prefill_rows=64)
+    g.set_tree(tpl.parent, tpl.rank)
+    g.begin(table)
+    cut = [37, 64]
+    for part in (0, 1):
+        seg = [t[:c] if part == 0 else t[c:] for t, c in zip(toks, cut)]
+        mat = np.zeros((wl.batch, max(len(x) for x in seg)), dtype=np.int32)
+        for b, x in enumerate(seg):
+            mat[b, :len(x)] = x
+        g.prefill(mat, [len(x) for x in seg])
+    assert list(g.lengths()) == [len(t) for t in toks]
+    states = {b: O.prefill_blocked(model, prefixes[b][0], prefixes[b][1], seq=b, chunk=128) for b in range(wl.batch)}
+    for b, st in states.items():
+        K, V = read_kv(g, table, b, st.S)
+        assert np.abs(K - st.kv.K[:, :st.S]).max() <= TOL["bf16"]
+        assert np.abs(V - st.kv.V[:, :st.S]).max() <= TOL["bf16"]
+    so, sg = _sampling(wl)
+    rep = lockstep(g, table, model, states, tpl, so, sg, 2, "bf16", oracle_mode="tree", check_attn=True)
+    assert rep.iterations == 2 and rep.root_checked >= 3
+    g.check()
+
+
 @pytest.mark.parametrize("nodes", [10, 24, 48])
 def test_bf16_small_token_counts_take_the_layernorm_fused_products(nodes):
     """d_model 256 (two groups of 128 features), one sequence: the token count selects the 16-, 32- and
