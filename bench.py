@@ -205,6 +205,88 @@ def aggregate(dist, device, ms, e2e_s, tokens, e2e_tokens, launches):
     return float(t[0]), float(t[1]), int(c[0]), int(c[1]), int(c[2])
 
 
+def fitted_heads_run(g, wl, tpl, bt, torch):
+    """Draft heads fitted with the base model frozen (the paper's "wot" setting: lambda 0.8, lr 0.002, 40 warm-up
+    steps), then the same step under greedy decoding with tolerance 1 (lossless), where what a head must predict
+    is a function of the context even for random-init base weights.  Training streams: the base model's own greedy
+    continuations of four other synthetic prefixes; evaluation on the headline prefix (held out), then once more
+    after the heads have also seen that continuation (memorised: the ceiling of this fitting on this model)."""
+    import workloads as W
+    import paper_2410_21951_b200 as P
+    sh = wl.shape
+    sp0 = P.Sampling.make(tau=1, temperature=0.0)
+    n_gen, T = 500, 512
+
+    def prefix_of(item):
+        ph = W.phonemes(wl.phoneme_len[0], sh.n_phonemes, wl.seed(item))
+        pr = W.markov_prompt(wl.prompt_len, sh.vocab - 1, wl.seed(item))
+        return np.concatenate([ph.astype(np.int32) + sh.vocab, pr.astype(np.int32)])
+
+    def stream_and_hidden(item):
+        prefix = prefix_of(item)
+        g.begin(bt)
+        g.prefill(prefix[None, :].copy(), [len(prefix)])
+        out = torch.full((1, n_gen), -1, dtype=torch.int32, device=g.dev)
+        out_len = torch.zeros(1, dtype=torch.int32, device=g.dev)
+        g.generate(sp0, n_gen, out, out_len)
+        full = np.concatenate([prefix, out.cpu().numpy()[0]]).astype(np.int32)
+        tap = torch.zeros(1, len(full), sh.d_model, dtype=g.tdtype, device=g.dev)
+        g.set_prefill_tap(tap)
+        g.begin(bt)
+        g.prefill(full[None, :].copy(), [len(full)])
+        g.set_prefill_tap(None)
+        t0 = len(prefix)
+        n = min(T, len(full) - t0)
+        tg = np.full((n, sh.n_draft_heads), -1, dtype=np.int32)
+        for i in range(sh.n_draft_heads):
+            m = max(0, min(n, len(full) - (t0 + 2 + i)))
+            tg[:m, i] = full[t0 + 2 + i:t0 + 2 + i + m]
+        return tap[0, t0:t0 + n].contiguous(), torch.from_numpy(tg).to(g.dev)
+
+    def evaluate(iters=200):
+        prefix = prefix_of(0)
+        g.begin(bt)
+        g.prefill(prefix[None, :].copy(), [len(prefix)])
+        for _ in range(5):
+            g.draft(sp0); g.verify_step(); g.accept_and_commit(sp0)
+        l0 = int(g.lengths()[0])
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(iters):
+            g.draft(sp0); g.verify_step(); g.accept_and_commit(sp0)
+        b.record()
+        torch.cuda.synchronize()
+        tokens = int(g.lengths()[0]) - l0
+        return {"mean_accepted_tokens": tokens / iters, "tokens_per_s": tokens / (a.elapsed_time(b) * 1e-3),
+                "ms_per_step": a.elapsed_time(b) / iters, "steps": iters}
+
+    before = evaluate()
+    train = [stream_and_hidden(item) for item in (1, 2, 3, 4)]
+    own = stream_and_hidden(0)
+    g.fit_begin(T, lam=0.8, lr=0.002, warmup=40)
+    loss = torch.zeros(1 + sh.n_draft_heads, dtype=torch.float32, device=g.dev)
+    first = None
+    for step in range(320):
+        h, tg = train[step % len(train)]
+        g.fit_step(h, tg, loss)
+        if step == 0:
+            first = float(loss[0])
+    held_out = evaluate()
+    held_out["loss_first_last"] = [first, float(loss[0])]
+    for step in range(160):
+        g.fit_step(own[0], own[1], loss)
+    memorised = evaluate()
+    memorised["loss_last"] = float(loss[0])
+    g.fit_end()
+    g.check()
+    return {"what": "greedy decoding, tolerance 1 (lossless), no forced choice; heads fitted by vadusa_fit_step with the base "
+                    "model frozen (lambda 0.8, lr 0.002, 40 warm-up steps, Adam); random-init base weights; this rank only",
+            "random_init_heads": before,
+            "fitted_on_four_other_prefixes_320_steps": held_out,
+            "then_160_steps_on_this_continuation": memorised}
+
+
 # ------------------------------------------------------------------------------ our arm
 def run_ours(args):
     import torch
@@ -358,6 +440,11 @@ def run_ours(args):
     e2e_tokens = int(h_len[0])
     e2e_iters = max(int(st.iterations), 1)
 
+    # ---- draft heads fitted on the base model's own continuations (changes the heads in the weight blob: last)
+    fitted = None
+    if world == 1 and not args.no_fit:
+        fitted = fitted_heads_run(g, wl, tpl, bt, torch)
+
     # ---- aggregate over ranks
     if world > 1:
         ms, e2e_s, tokens, e2e_tokens, launches = aggregate(dist, g.dev, ms, e2e_s, tokens, e2e_tokens, launches)
@@ -426,6 +513,7 @@ def run_ours(args):
                                 "what": "CUDA events around single steps (separate pass; a host read-back between steps)"},
             "accepted_length_histogram": hist,
             "persistent_pass": persistent,
+            "fitted_heads": fitted,
             "c5": c5,
         }
         print(json.dumps(line))
@@ -606,6 +694,7 @@ def main():
                     help="C3, C4: prefix chunks of 64 tokens scored per prefill pass (0: one per sequence)")
     ap.add_argument("--tree-nodes", type=int, default=0, choices=[0, 64, 96, 128],
                     help="C2 only: candidate-tree size (default: the workload's 64 nodes)")
+    ap.add_argument("--no-fit", action="store_true", help="C2 only: skip the draft-head fitting run that follows the headline region")
     ap.add_argument("--no-c5", action="store_true", help="C2 only: skip the batch-64 microbenchmark that follows the headline region")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)

@@ -307,6 +307,34 @@ vadusa_status vadusa_accept_stats(vadusa_ctx *ctx, int64_t *h_tested, int64_t *h
 vadusa_status vadusa_build_sparse_tree(const double *h_prob, int32_t depth, int32_t topk, int32_t n_nodes,
                                        int32_t *h_parent, int32_t *h_rank, double *h_expected_len);
 
+/* ---- fitting the draft heads (paper Sec. II-A, III-A.2) -----------------------------------
+ * "The i-th draft head is responsible for predicting the (i+1)-th next token by the supervision of a
+ * cross-entropy loss multiplied with lambda^i" (i >= 1), with the base model fixed (the paper's "wot" setting:
+ * lambda 0.8, learning rate 0.002, 40 warm-up steps).  The paper names no optimiser and no normalisation:
+ * here every head's cross-entropy is averaged over the positions that have a target, the optimiser is Adam
+ * (beta 0.9 / 0.999, eps 1e-8, no weight decay), and the learning rate rises linearly over the warm-up steps.
+ * Not part of the decoding path: plain fp32 arithmetic on fp32 master copies of the heads kept in `state`
+ * (device memory owned by the caller, >= vadusa_fit_state_bytes(cfg, max_tokens), 256-byte aligned).
+ * vadusa_fit_begin copies the heads from the weight blob; every vadusa_fit_step writes the updated heads
+ * back INTO THE CALLER'S WEIGHT BLOB (tensors "draft<i>.w/.b/.u", in the model dtype), so the next
+ * vadusa_draft uses them.
+ *   hidden  [n_tokens][d_model] in the model dtype: final-LayerNorm outputs of the frozen base model at
+ *           consecutive positions (vadusa_set_prefill_tap makes vadusa_prefill deliver them)
+ *   targets int32 [n_tokens][n_draft_heads]: targets[t][i] = the token at position t + 2 + i (the (i+2)-th
+ *           token after position t's own; head numbering from 0), or -1 where the stream has none
+ *   loss_out device fp32 [1 + n_draft_heads] or NULL: the weighted total, then each head's mean cross-entropy
+ * Work is enqueued on the context's stream; no call synchronises. */
+int64_t vadusa_fit_state_bytes(const vadusa_config *cfg, int32_t max_tokens);
+vadusa_status vadusa_fit_begin(vadusa_ctx *ctx, void *state, int64_t state_bytes, int32_t max_tokens, float lambda,
+                               float learning_rate, int32_t warmup_steps);
+vadusa_status vadusa_fit_step(vadusa_ctx *ctx, const void *hidden, const int32_t *targets, int32_t n_tokens,
+                              float *loss_out);
+vadusa_status vadusa_fit_end(vadusa_ctx *ctx);
+/* While set, vadusa_prefill also stores the final-LayerNorm output of every prefix token it scores:
+ * hidden_out [batch][stride][d_model] in the model dtype, row (b, s) for token s of the prefix passed in that
+ * call (stride >= the longest prefix).  NULL switches it off. */
+vadusa_status vadusa_set_prefill_tap(vadusa_ctx *ctx, void *hidden_out, int32_t stride);
+
 /* ---- measurement ------------------------------------------------------------------ */
 /* Between vadusa_profile_begin and vadusa_profile_end every kernel launch of the library
  * is bracketed by a pair of CUDA events on the context's stream.  vadusa_profile_end

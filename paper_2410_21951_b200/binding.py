@@ -70,6 +70,7 @@ EXPORTS = ["vadusa_workspace_bytes", "vadusa_weights_bytes", "vadusa_kv_pool_byt
            "vadusa_accept_and_commit", "vadusa_generate", "vadusa_generate_host", "vadusa_get_lengths",
            "vadusa_check", "vadusa_kernel_launches", "vadusa_profile_begin", "vadusa_profile_end",
            "vadusa_accept_stats", "vadusa_build_sparse_tree", "vadusa_set_logit_bias", "vadusa_set_fused_pass", "vadusa_fused_pass_clusters",
+           "vadusa_fit_state_bytes", "vadusa_fit_begin", "vadusa_fit_step", "vadusa_fit_end", "vadusa_set_prefill_tap",
            "vadusa_draft_topk_static", "vadusa_static_scratch_bytes", "vadusa_static_last_error"]
 
 _lib = None
@@ -103,6 +104,11 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "vadusa_kernel_launches": (I64, [P]),
         "vadusa_set_fused_pass": (I32, [P, I32]),
         "vadusa_fused_pass_clusters": (I32, [P]),
+        "vadusa_fit_state_bytes": (I64, [cfgp, I32]),
+        "vadusa_fit_begin": (I32, [P, P, I64, I32, C.c_float, C.c_float, I32]),
+        "vadusa_fit_step": (I32, [P, P, P, I32, P]),
+        "vadusa_fit_end": (I32, [P]),
+        "vadusa_set_prefill_tap": (I32, [P, P, I32]),
         "vadusa_draft_topk_static": (I32, [P, P, P, P, I32, I32, I32, I32, I32, I32, I32, P, P]),
         "vadusa_static_scratch_bytes": (I64, []),
         "vadusa_static_last_error": (C.c_char_p, []),
@@ -394,6 +400,28 @@ class Vadusa:
 
     def fused_pass_clusters(self) -> int:
         return int(self.L.vadusa_fused_pass_clusters(self.ctx))
+
+    # ---- draft-head fitting ----
+    def fit_begin(self, max_tokens: int, lam: float = 0.8, lr: float = 0.002, warmup: int = 40):
+        n = self.L.vadusa_fit_state_bytes(C.byref(self.cfg), max_tokens)
+        self._keep["fit_state"] = self.torch.zeros(n, dtype=self.torch.uint8, device=self.dev)
+        self._enter()
+        self._ck(self.L.vadusa_fit_begin(self.ctx, self._p(self._keep["fit_state"]), n, max_tokens, lam, lr, warmup))
+        self._leave()
+
+    def fit_step(self, hidden, targets, loss_out=None):
+        self._enter()
+        self._ck(self.L.vadusa_fit_step(self.ctx, self._p(hidden), self._p(targets), hidden.shape[0], self._p(loss_out)))
+        self._leave()
+
+    def fit_end(self):
+        self._ck(self.L.vadusa_fit_end(self.ctx))
+        self._keep.pop("fit_state", None)
+
+    def set_prefill_tap(self, hidden_out=None):
+        """hidden_out: device tensor [batch][stride][d_model] in the model dtype, or None."""
+        self._keep["prefill_tap"] = hidden_out
+        self._ck(self.L.vadusa_set_prefill_tap(self.ctx, self._p(hidden_out), 0 if hidden_out is None else hidden_out.shape[1]))
 
     def profile_begin(self):
         self._ck(self.L.vadusa_profile_begin(self.ctx))

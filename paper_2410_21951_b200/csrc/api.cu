@@ -16,6 +16,7 @@
 #include "attention_tc.cuh"
 #include "attention_prefill_tc.cuh"
 #include "elementwise.cuh"
+#include "fit.cuh"
 #include "fwd_fused.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
@@ -48,6 +49,12 @@ struct vadusa_ctx {
   int tree_per_seq = 0;
   int max_rank_used = 0;
   int tree_max_depth = 0;
+  // draft-head fitting (vadusa_fit_*): the caller's state buffer and the schedule
+  char* fit = nullptr;
+  int fit_tokens = 0, fit_step = 0, fit_warmup = 0;
+  float fit_lambda = 0.f, fit_lr = 0.f;
+  void* pf_tap = nullptr;     // where prefill also leaves the final hidden state of every prefix token ([batch][stride][d])
+  int pf_tap_stride = 0;
   int pf_tiles = 0;           // > 0 while a prefill pass runs: attention CTAs of the pass (pairs of chunks), listed in ws.pf_pairs
   int fused_enabled = 0;      // single-sequence passes run as one persistent kernel (0: no, 1: yes, 6 / 8: with that cluster size)
   int fused_clusters = -1;    // clusters of that kernel that can be resident at once on this device (-1: not asked yet)
@@ -863,9 +870,109 @@ vadusa_status prefill(vadusa_ctx* ctx, const int32_t* h_tokens, const int32_t* h
                                                             wsptr<T>(ctx, ctx->ws.hstar),
                                                             wsptr<float>(ctx, ctx->ws.logits_star), real_ctx_len);
     LAUNCH_CHECK();
+    if (ctx->pf_tap)
+      for (int r = 0; r < rows; ++r) {
+        const Chunk& ch = chunks[c0 + r];
+        if (ch.s0 + ch.n > ctx->pf_tap_stride) return fail(ctx, VADUSA_EINVAL, "prefill tap: row stride shorter than the prefix");
+        CU(cudaMemcpyAsync(reinterpret_cast<T*>(ctx->pf_tap) + ((long long)ch.b * ctx->pf_tap_stride + ch.s0) * c.d_model,
+                           wsptr<T>(ctx, ctx->ws.hfinal) + (long long)r * N * c.d_model, (size_t)ch.n * c.d_model * sizeof(T),
+                           cudaMemcpyDeviceToDevice, ctx->stream));
+      }
   }
   ctx->ctx_bound += longest;
   CU(cudaStreamSynchronize(ctx->stream));
+  return VADUSA_OK;
+}
+
+// ---- draft-head fitting -------------------------------------------------------------------
+struct FitLayout {
+  int64_t W, b, U, n_params;               // fp32 masters, contiguous: [heads][d][d], [heads][d], [heads][vpad][d]
+  int64_t m, v, g;                         // Adam moments and gradients, same shape as the masters
+  int64_t hf, pre, z, dz, logits, ce, count, total;
+};
+FitLayout fit_layout(const vadusa_config* c, int max_tokens) {
+  FitLayout f;
+  const int64_t hd = c->n_draft_heads, d = c->d_model, vp = vpad(c), T = max_tokens;
+  int64_t off = 0;
+  auto take = [&](int64_t bytes) { int64_t o = off; off = align_up(off + bytes, 256); return o; };
+  f.n_params = hd * (d * d + d + vp * d);
+  f.W = take(f.n_params * 4); f.b = f.W + hd * d * d * 4; f.U = f.b + hd * d * 4;
+  f.m = take(f.n_params * 4); f.v = take(f.n_params * 4); f.g = take(f.n_params * 4);
+  f.hf = take(T * d * 4); f.pre = take(hd * T * d * 4); f.z = take(hd * T * d * 4); f.dz = take(hd * T * d * 4);
+  f.logits = take(hd * T * vp * 4); f.ce = take(hd * T * 4); f.count = take(hd * 4);
+  f.total = off;
+  return f;
+}
+
+template <typename T>
+vadusa_status fit_begin(vadusa_ctx* ctx, const FitLayout& f) {
+  const vadusa_config& c = ctx->cfg;
+  const long long hd = c.n_draft_heads, d = c.d_model, vp = vpad(&c);
+  auto up = [&](const T* src, int64_t off, long long n) -> vadusa_status {
+    fit_to_f32_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, ctx->stream>>>(src, reinterpret_cast<float*>(ctx->fit + off), n);
+    LAUNCH_CHECK();
+    return VADUSA_OK;
+  };
+  if (vadusa_status s = up(as<T>(ctx->dw), f.W, hd * d * d)) return s;
+  if (vadusa_status s = up(as<T>(ctx->du), f.U, hd * vp * d)) return s;
+  CU(cudaMemcpyAsync(ctx->fit + f.b, ctx->db, (size_t)(hd * d * 4), cudaMemcpyDeviceToDevice, ctx->stream));
+  CU(cudaMemsetAsync(ctx->fit + f.m, 0, (size_t)(f.n_params * 4), ctx->stream));
+  CU(cudaMemsetAsync(ctx->fit + f.v, 0, (size_t)(f.n_params * 4), ctx->stream));
+  return VADUSA_OK;
+}
+
+template <typename T>
+vadusa_status fit_step(vadusa_ctx* ctx, const FitLayout& f, const T* hidden, const int32_t* targets, int Tn, float* loss_out) {
+  const vadusa_config& c = ctx->cfg;
+  const int hd = c.n_draft_heads, d = c.d_model, vp = vpad(&c), V = c.vocab;
+  auto P = [&](int64_t off) { return reinterpret_cast<float*>(ctx->fit + off); };
+  float *W = P(f.W), *b = P(f.b), *U = P(f.U), *gW = P(f.g), *gb = gW + (long long)hd * d * d, *gU = gb + (long long)hd * d;
+  float *hf = P(f.hf), *pre = P(f.pre), *z = P(f.z), *dz = P(f.dz), *lg = P(f.logits), *ce = P(f.ce);
+  int32_t* count = reinterpret_cast<int32_t*>(ctx->fit + f.count);
+  const long long hs = (long long)Tn * d, ls = (long long)Tn * vp;
+  cudaStream_t st = ctx->stream;
+  auto gemm = [&](const float* A, const float* B, float* C, int M, int N, int K, long long sam, long long sak, long long sbn,
+                  long long sbk, long long ldc, long long az, long long bz, long long cz) -> vadusa_status {
+    dim3 grid((N + 63) / 64, (M + 63) / 64, hd);
+    fit_gemm_kernel<<<grid, 256, 0, st>>>(A, B, C, M, N, K, sam, sak, sbn, sbk, ldc, az, bz, cz);
+    LAUNCH_CHECK();
+    return VADUSA_OK;
+  };
+  const unsigned eb = (unsigned)((hs + 255) / 256);
+  fit_to_f32_kernel<T><<<eb, 256, 0, st>>>(hidden, hf, hs);
+  LAUNCH_CHECK();
+  fit_count_kernel<<<1, 256, 0, st>>>(targets, Tn, hd, count);
+  LAUNCH_CHECK();
+  // forward: pre = h W^T (+ b), z = h + SiLU(pre), logits = z U^T
+  if (vadusa_status s = gemm(hf, W, pre, Tn, d, d, d, 1, d, 1, d, 0, (long long)d * d, hs)) return s;
+  fit_hidden_kernel<<<dim3(eb, hd), 256, 0, st>>>(pre, b, hf, z, Tn, d, hs);
+  LAUNCH_CHECK();
+  if (vadusa_status s = gemm(z, U, lg, Tn, vp, d, d, 1, d, 1, vp, hs, (long long)vp * d, ls)) return s;
+  // loss and d loss / d logits (over the logits)
+  fit_softmax_ce_kernel<<<dim3(Tn, hd), 256, 0, st>>>(lg, targets, count, Tn, hd, V, vp, ctx->fit_lambda, ce);
+  LAUNCH_CHECK();
+  fit_loss_kernel<<<1, 256, 0, st>>>(ce, count, Tn, hd, ctx->fit_lambda, loss_out);
+  LAUNCH_CHECK();
+  // backward: dU = dl^T z, dz = dl U, dpre = dz SiLU'(pre), dW = dpre^T h, db = column sums of dpre
+  if (vadusa_status s = gemm(lg, z, gU, vp, d, Tn, 1, vp, 1, d, d, ls, hs, (long long)vp * d)) return s;
+  if (vadusa_status s = gemm(lg, U, dz, Tn, d, vp, vp, 1, 1, d, d, ls, (long long)vp * d, hs)) return s;
+  fit_dpre_kernel<<<dim3(eb, hd), 256, 0, st>>>(dz, pre, hs, hs);
+  LAUNCH_CHECK();
+  if (vadusa_status s = gemm(dz, hf, gW, d, d, Tn, 1, d, 1, d, d, hs, 0, (long long)d * d)) return s;
+  fit_colsum_kernel<<<dim3((d + 255) / 256, hd), 256, 0, st>>>(dz, gb, Tn, d, hs);
+  LAUNCH_CHECK();
+  // update (Adam, linear warm-up), masters and the heads in the weight blob
+  ctx->fit_step++;
+  const float lr = ctx->fit_lr * fminf(1.0f, (float)ctx->fit_step / (float)(ctx->fit_warmup > 0 ? ctx->fit_warmup : 1));
+  const float c1 = (float)(1.0 - pow(0.9, (double)ctx->fit_step)), c2 = (float)(1.0 - pow(0.999, (double)ctx->fit_step));
+  float *mW = P(f.m), *vW = P(f.v);
+  const long long nW = (long long)hd * d * d, nb = (long long)hd * d, nU = (long long)hd * vp * d;
+  fit_adam_kernel<T><<<(unsigned)((nW + 255) / 256), 256, 0, st>>>(W, gW, mW, vW, const_cast<T*>(as<T>(ctx->dw)), nW, lr, c1, c2);
+  LAUNCH_CHECK();
+  fit_adam_kernel<float><<<(unsigned)((nb + 255) / 256), 256, 0, st>>>(b, gb, mW + nW, vW + nW, const_cast<float*>(ctx->db), nb, lr, c1, c2);
+  LAUNCH_CHECK();
+  fit_adam_kernel<T><<<(unsigned)((nU + 255) / 256), 256, 0, st>>>(U, gU, mW + nW + nb, vW + nW + nb, const_cast<T*>(as<T>(ctx->du)), nU, lr, c1, c2);
+  LAUNCH_CHECK();
   return VADUSA_OK;
 }
 
@@ -1302,6 +1409,13 @@ vadusa_status vadusa_generate(vadusa_ctx* ctx, const vadusa_sampling* sampling, 
       poll_pending = false;
       if (ctx->h_pinned[0] >= ctx->batch) break;
     }
+    // stay at most sixteen iterations ahead of the device: when the next poll is due and the last one has not come
+    // back, wait for it (iterations enqueued behind the end of the last sequence find nothing to do, but cost time)
+    if (poll_pending && (iters & 7) == 7) {
+      CU(cudaEventSynchronize(ctx->ev_poll));
+      poll_pending = false;
+      if (ctx->h_pinned[0] >= ctx->batch) break;
+    }
     const std::string iter_key = KeyBuilder("iteration").add(sp).add(out_tokens).add(max_new_tokens).add(ctx->batch)
                                      .add(ctx->n_nodes).add(ctx->block_table).add(attention_splits(ctx, ctx->n_nodes)).add(ctx->fused_enabled).k;
     vadusa_status s = run_graphed(ctx, iter_key, [&]() -> vadusa_status {
@@ -1443,6 +1557,51 @@ vadusa_status vadusa_build_sparse_tree(const double* h_prob, int32_t depth, int3
     h_rank[i] = tree[i].path.back();
   }
   if (h_expected_len) *h_expected_len = expected;
+  return VADUSA_OK;
+}
+
+int64_t vadusa_fit_state_bytes(const vadusa_config* cfg, int32_t max_tokens) {
+  if (check_config(cfg) || max_tokens < 1) return -1;
+  return fit_layout(cfg, max_tokens).total;
+}
+
+vadusa_status vadusa_fit_begin(vadusa_ctx* ctx, void* state, int64_t state_bytes, int32_t max_tokens, float lambda,
+                               float learning_rate, int32_t warmup_steps) {
+  if (!ctx) return VADUSA_EINVAL;
+  if (!ctx->wsp) return fail(ctx, VADUSA_ESTATE, "context is not initialised");
+  if (!state || max_tokens < 1 || ((uintptr_t)state & 255)) return fail(ctx, VADUSA_EINVAL, "fit state is NULL, unaligned or sized for no token");
+  if (!(lambda > 0.f && lambda <= 1.f) || !(learning_rate > 0.f) || warmup_steps < 0) return fail(ctx, VADUSA_EINVAL, "lambda must be in (0, 1], the learning rate positive");
+  const FitLayout f = fit_layout(&ctx->cfg, max_tokens);
+  if (state_bytes < f.total) return fail(ctx, VADUSA_ENOMEM, "fit state has %lld bytes, %lld needed", (long long)state_bytes, (long long)f.total);
+  if (ctx->cfg.n_draft_heads > 1 && ctx->dw_stride != (long long)ctx->cfg.d_model * ctx->cfg.d_model * esize(&ctx->cfg))
+    return fail(ctx, VADUSA_EINVAL, "draft matrices are not contiguous");
+  ctx->fit = reinterpret_cast<char*>(state);
+  ctx->fit_tokens = max_tokens; ctx->fit_step = 0; ctx->fit_warmup = warmup_steps;
+  ctx->fit_lambda = lambda; ctx->fit_lr = learning_rate;
+  return DISPATCH(fit_begin<float>(ctx, f), fit_begin<bf16>(ctx, f));
+}
+
+vadusa_status vadusa_fit_step(vadusa_ctx* ctx, const void* hidden, const int32_t* targets, int32_t n_tokens, float* loss_out) {
+  if (!ctx) return VADUSA_EINVAL;
+  if (!ctx->fit) return fail(ctx, VADUSA_ESTATE, "vadusa_fit_begin has not been called");
+  if (!hidden || !targets || n_tokens < 1 || n_tokens > ctx->fit_tokens) return fail(ctx, VADUSA_EINVAL, "fit step: NULL input or token count out of range");
+  const FitLayout f = fit_layout(&ctx->cfg, ctx->fit_tokens);
+  ctx->have_draft = false;
+  return DISPATCH(fit_step<float>(ctx, f, reinterpret_cast<const float*>(hidden), targets, n_tokens, loss_out),
+                  fit_step<bf16>(ctx, f, reinterpret_cast<const bf16*>(hidden), targets, n_tokens, loss_out));
+}
+
+vadusa_status vadusa_fit_end(vadusa_ctx* ctx) {
+  if (!ctx) return VADUSA_EINVAL;
+  ctx->fit = nullptr;
+  return VADUSA_OK;
+}
+
+vadusa_status vadusa_set_prefill_tap(vadusa_ctx* ctx, void* hidden_out, int32_t stride) {
+  if (!ctx) return VADUSA_EINVAL;
+  if (hidden_out && stride < 1) return fail(ctx, VADUSA_EINVAL, "prefill tap: stride must be positive");
+  ctx->pf_tap = hidden_out;
+  ctx->pf_tap_stride = hidden_out ? stride : 0;
   return VADUSA_OK;
 }
 
