@@ -22,6 +22,34 @@ namespace vadusa {
 
 constexpr int kPfThreads = 352;
 
+// Two 32-column loads (32 lanes x 32 fp32 each) issued back to back, one wait for both.
+__device__ __forceinline__ void tmem_ld32x2(uint32_t ta, float* a, uint32_t tb, float* b) {
+  uint32_t r[32], q[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(ta)
+      : "memory");
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(q[0]), "=r"(q[1]), "=r"(q[2]), "=r"(q[3]), "=r"(q[4]), "=r"(q[5]), "=r"(q[6]), "=r"(q[7]),
+        "=r"(q[8]), "=r"(q[9]), "=r"(q[10]), "=r"(q[11]), "=r"(q[12]), "=r"(q[13]), "=r"(q[14]), "=r"(q[15]),
+        "=r"(q[16]), "=r"(q[17]), "=r"(q[18]), "=r"(q[19]), "=r"(q[20]), "=r"(q[21]), "=r"(q[22]), "=r"(q[23]),
+        "=r"(q[24]), "=r"(q[25]), "=r"(q[26]), "=r"(q[27]), "=r"(q[28]), "=r"(q[29]), "=r"(q[30]), "=r"(q[31])
+      : "r"(tb)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) { a[i] = __uint_as_float(r[i]); b[i] = __uint_as_float(q[i]); }
+}
+
 __global__ void __launch_bounds__(kPfThreads, 1) prefill_attention_tc_kernel(
     const __grid_constant__ CUtensorMap tmQ,    // q [1][rows * 64][d_model], box 64 x 64
     const __grid_constant__ CUtensorMap tmKV,   // pool [layers][blocks * 2 * heads * 64][64], box 64 x 64
@@ -132,7 +160,9 @@ __global__ void __launch_bounds__(kPfThreads, 1) prefill_attention_tc_kernel(
       constexpr uint32_t idesc_qk = umma_idesc_bf16(128, 64);
       bool ok = ntiles == 0 || mbar_wait(bar_q, 0, err);
       for (int i = 0; i < ntiles && ok; ++i) {
-        if (i >= 3 && !mbar_wait(bar_o0 + 8 * (i % 3), ((i - 3) / 3) & 1, err)) break;
+        // score buffer i % 3 held page i - 3: free once the softmax threads are done with it (the weights have a
+        // buffer of their own, so this does not wait for that page's P V)
+        if (i >= 3 && !mbar_wait(bar_p0 + 8 * (i % 3), ((i - 3) / 3) & 1, err)) break;
         const int s = i % SK;
         if (!mbar_wait(full_k0 + 8 * s, (i / SK) & 1, err)) break;
         tc_fence_after();
@@ -162,15 +192,18 @@ __global__ void __launch_bounds__(kPfThreads, 1) prefill_attention_tc_kernel(
       float sc[32], mx;
       {
         float so[32];                                             // the other thread's keys: for the maximum only
-        tmem_ld32(tsp + 32 * (1 - khalf), so);
-        tmem_ld32(tsp + 32 * khalf, sc);
-        const int no = nvis - 32 * (1 - khalf), nm = nvis - 32 * khalf;
+        tmem_ld32x2(tsp + 32 * khalf, sc, tsp + 32 * (1 - khalf), so);
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        if (nvis < kKvBlock) {                                    // (a page on or past the row's diagonal)
+          const int no = nvis - 32 * (1 - khalf), nm = nvis - 32 * khalf;
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          sc[j] = j < nm ? sc[j] : -INFINITY;
-          mx4[j & 3] = fmax3(mx4[j & 3], sc[j], j < no ? so[j] : -INFINITY);
+          for (int j = 0; j < 32; ++j) {
+            sc[j] = j < nm ? sc[j] : -INFINITY;
+            so[j] = j < no ? so[j] : -INFINITY;
+          }
         }
+#pragma unroll
+        for (int j = 0; j < 32; ++j) mx4[j & 3] = fmax3(mx4[j & 3], sc[j], so[j]);
         mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       }
       if ((i + 1) * kKvBlock > total && tid < 64) {      // rows of V past the last token may hold anything: zero them
@@ -214,6 +247,8 @@ __global__ void __launch_bounds__(kPfThreads, 1) prefill_attention_tc_kernel(
         lv[j] = pack_bf16(pa - ha, pb - hb);
       }
       l_run += (psum4[0] + psum4[1]) + (psum4[2] + psum4[3]);
+      // weight buffer i % 3 was read by the P V of page i - 3 (issued two pages ago; normally long complete)
+      if (i >= 3 && !mbar_wait(bar_o0 + 8 * (i % 3), ((i - 3) / 3) & 1, err)) break;
       tmem_st16(tpp + 16 * khalf, hv);                   // keys 32 khalf .. +31: hi in columns 16 khalf .., lo in 32 + 16 khalf ..
       tmem_st16(tpp + 32 + 16 * khalf, lv);
       tmem_st_wait();
