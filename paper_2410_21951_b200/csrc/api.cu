@@ -339,6 +339,39 @@ vadusa_status launch_gemm_tc2(vadusa_ctx* ctx, int cls, const void* X, const voi
   return VADUSA_OK;
 }
 
+// Persistent CTA pairs: tiles of 256 features x 256 tokens dealt round-robin to as many pairs as balance the rounds.
+template <typename Epi>
+vadusa_status launch_gemm_tc2p(vadusa_ctx* ctx, int cls, const void* X, const void* W, int w_rows, int M, int N, int K,
+                               const Epi& epi) {
+  static unsigned long long attr_done = 0ull;
+  const unsigned long long dev_bit = 1ull << (ctx->cfg.device & 63);
+  if (!(attr_done & dev_bit)) {
+    CU(cudaFuncSetAttribute(gemm_tc2p_kernel<Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmP2Smem));
+    CU(cudaFuncSetAttribute(gemm_tc2p_kernel<Epi>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+    attr_done |= dev_bit;
+  }
+  const CUtensorMap *mw, *mx;
+  if (vadusa_status s = tensor_map(ctx, W, w_rows, K, kGemmRowsW, 1, 0, &mw)) return s;
+  if (vadusa_status s = tensor_map(ctx, X, M, K, kGemmP2TN / 2, 1, 0, &mx)) return s;
+  const int tiles = (N / (2 * kGemmRowsW)) * ((M + kGemmP2TN - 1) / kGemmP2TN);
+  const int rounds = (tiles + 73) / 74, npairs = (tiles + rounds - 1) / rounds;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(2 * npairs, 1, 1);
+  lc.blockDim = dim3(kGemmP2Threads);
+  lc.dynamicSmemBytes = kGemmP2Smem;
+  lc.stream = ctx->stream;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at; lc.numAttrs = 2;
+  PROF(ctx, cls);
+  CU(cudaLaunchKernelEx(&lc, gemm_tc2p_kernel<Epi>, *mw, *mx, M, N, K / kGemmBK, tiles, epi, err_word(ctx)));
+  LAUNCH_CHECK();
+  return VADUSA_OK;
+}
+
 // K split of a product with `tiles` output tiles of tn tokens: about one CTA per SM streams weights.
 static int gemm_ksplit(int tiles, int chunks, int tn) {
   int ksplit = 1;
@@ -387,6 +420,8 @@ vadusa_status gemm_tc(vadusa_ctx* ctx, int cls, const void* X, const void* W, in
   // the 256-token tile (two CTAs per SM) and the 128-token tile (two per SM with four stages when all CTAs are
   // resident at once, else three per SM with three stages) the one whose last wave is fuller; ties to the wider.
   if (M > 512 && batches == 1 && N % (2 * kGemmRowsW) == 0) {
+    // at least two full rounds of 256 x 256 tiles per pair: resident pairs whose epilogue runs under the next tile
+    if ((N / (2 * kGemmRowsW)) * ((M + 255) / 256) >= 148) return launch_gemm_tc2p(ctx, cls, X, W, w_rows, M, N, K, epi);
     auto fill = [](int ctas, int slots) { return (double)ctas / (double)(((ctas + slots - 1) / slots) * slots); };
     const int c256 = ntiles_n * ((M + 255) / 256), c128 = ntiles_n * ((M + 127) / 128);
     const double f256 = c256 >= 128 ? fill(c256, 296) : 0.0;

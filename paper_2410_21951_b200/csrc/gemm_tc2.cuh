@@ -158,3 +158,136 @@ __global__ void __launch_bounds__(128) gemm_tc2_kernel(const __grid_constant__ C
 }
 
 }  // namespace vadusa
+
+namespace vadusa {
+
+// ---- persistent variant --------------------------------------------------------------------------
+// The same CTA-pair product, but a pair stays resident and walks a list of output tiles (256 features x 256
+// tokens each; tile t -> token tile t / (N / 256), feature pair t % (N / 256), so that the pairs running at the
+// same time share token rows in L2): two accumulators of 256 columns in TMEM, so the epilogue of tile k (four
+// warps of their own) runs under the main loop of tile k + 1, and the TMA ring (six stages of 32 KB) streams on
+// across tile boundaries.  For products with at least two rounds of tiles per pair; one CTA per SM.
+// Warps: 0 TMA producer (lane 0, both CTAs), 1 TMEM owner / MMA issuer (leader's lane 0), 2..9 epilogue (two warps
+// per quarter of the TMEM lanes, half of the tile's tokens each: the epilogue, not the main loop, bounds a tile).
+constexpr int kGemmP2Threads = 320;
+constexpr int kGemmP2Stages = 6;
+constexpr int kGemmP2TN = 256;
+constexpr int kGemmP2StageBytes = kGemmRowsW * kGemmBK * 2 + (kGemmP2TN / 2) * kGemmBK * 2;      // 32 KB
+constexpr int kGemmP2Smem = kGemmP2Stages * kGemmP2StageBytes + 1024 /*alignment*/ + 256 /*barriers*/;
+
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t remote_bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+}
+
+template <typename Epi>
+__global__ void __launch_bounds__(kGemmP2Threads, 1) gemm_tc2p_kernel(const __grid_constant__ CUtensorMap tmW,
+                                                                      const __grid_constant__ CUtensorMap tmX /*box: 128 rows*/,
+                                                                      int M, int N, int nchunks, int ntiles, Epi epi, uint32_t* err) {
+  constexpr int S = kGemmP2Stages, TN = kGemmP2TN;
+  constexpr uint32_t kWBytes = kGemmRowsW * kGemmBK * 2, kXBytes = (TN / 2) * kGemmBK * 2;
+  constexpr int kRing = S * kGemmP2StageBytes;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* ring_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bars = base + kRing;        // full[S], empty[S], acc_full[2], acc_empty[2], tmem holder
+  const uint32_t full0 = bars, empty0 = bars + 8 * S, accf0 = bars + 16 * S, acce0 = accf0 + 16, holder = acce0 + 16;
+  volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(ring_ptr + kRing + 16 * S + 32);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();                  // 0: leader
+  const int pair = (int)blockIdx.x >> 1, npairs = (int)gridDim.x >> 1;
+  const int nfp = N / (2 * kGemmRowsW);                  // feature pairs per token tile
+  const int my_tiles = pair < ntiles ? (ntiles - pair + npairs - 1) / npairs : 0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    mbar_init(accf0, 1); mbar_init(accf0 + 8, 1);
+    mbar_init(acce0, 2); mbar_init(acce0 + 8, 2);        // one arrival per CTA of the pair
+    mbar_fence_init();
+    tma_prefetch_desc(&tmW);
+    tma_prefetch_desc(&tmX);
+  }
+  if (warp == 1) { tmem_alloc_pair(holder, 2 * TN); tmem_relinquish_pair(); }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                                    // the peer's barriers exist before anything signals them
+  tc_fence_after();
+  const uint32_t tmem = *holder_ptr;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---- TMA producer (both CTAs): own 128 weight rows, own half of the token tile; one chunk counter over all tiles
+      bool waited = false, ok = true;
+      long long g = 0;
+      for (int k = 0; k < my_tiles && ok; ++k) {
+        const int t = pair + k * npairs;
+        const int n0 = (t % nfp) * 2 * kGemmRowsW + (int)rank * kGemmRowsW, m0 = (t / nfp) * TN + (int)rank * (TN / 2);
+        for (int i = 0; i < nchunks; ++i, ++g) {
+          const int s = (int)(g % S);
+          if (g >= S && !mbar_wait(empty0 + 8 * s, (uint32_t)((g / S) - 1) & 1, err)) { ok = false; break; }
+          if (rank == 0) mbar_expect_tx(full0 + 8 * s, 2 * (kWBytes + kXBytes));
+          const uint32_t fb = map_to_cta(full0 + 8 * s, 0);
+          tma_load_3d_pair(base + s * kGemmP2StageBytes, &tmW, fb, i * kGemmBK, n0, 0);
+          if (!waited) { grid_dep_wait(); waited = true; }        // the tokens come from the upstream kernel
+          tma_load_3d_pair(base + s * kGemmP2StageBytes + kWBytes, &tmX, fb, i * kGemmBK, m0, 0);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {
+      // ---- MMA issuer (leader only): 256 features x 256 tokens per instruction, accumulator k & 1
+      constexpr uint32_t idesc = umma_idesc_bf16(2 * kGemmRowsW, TN);
+      bool ok = true;
+      long long g = 0;
+      for (int k = 0; k < my_tiles && ok; ++k) {
+        const int b = k & 1;
+        // both CTAs' epilogue warps have read what tile k - 2 left in this accumulator
+        if (k >= 2 && !mbar_wait_cluster(acce0 + 8 * b, (uint32_t)((k >> 1) - 1) & 1, err)) break;
+        tc_fence_after();
+        for (int i = 0; i < nchunks; ++i, ++g) {
+          const int s = (int)(g % S);
+          if (!mbar_wait(full0 + 8 * s, (uint32_t)(g / S) & 1, err)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t wa = base + s * kGemmP2StageBytes, xa = wa + kWBytes;
+#pragma unroll
+          for (int kk = 0; kk < kGemmBK / 16; ++kk)
+            umma_bf16_pair(tmem + TN * b, umma_desc_k_sw128(wa + 32 * kk), umma_desc_k_sw128(xa + 32 * kk), idesc, (i | kk) != 0);
+          umma_commit_pair(empty0 + 8 * s);
+        }
+        if (ok) umma_commit_pair(accf0 + 8 * b);
+      }
+    }
+  } else {
+    // ---- epilogue warps: TMEM lanes 32 (warp % 4) .. +31 = features n0 + 32 (warp % 4) + lane of this CTA
+    const int wq = warp & 3, chalf = (warp - 2) >> 2;
+    grid_dep_wait();
+    for (int k = 0; k < my_tiles; ++k) {
+      const int t = pair + k * npairs, b = k & 1;
+      const int n = (t % nfp) * 2 * kGemmRowsW + (int)rank * kGemmRowsW + 32 * wq + lane, m0 = (t / nfp) * TN;
+      const bool done = mbar_wait(accf0 + 8 * b, (uint32_t)(k >> 1) & 1, err);
+      tc_fence_after();
+      if (k == my_tiles - 1) grid_dep_launch();
+      const uint32_t trow = tmem + ((uint32_t)(32 * wq) << 16) + TN * b;
+      if (done) {
+#pragma unroll 1
+        for (int c0 = chalf * (TN / 2); c0 < (chalf + 1) * (TN / 2); c0 += 32) {
+          float v[32];
+          tmem_ld32(trow + c0, v);
+          if (n < N && m0 + c0 < M) epi.template col<32>(0, m0 + c0, n, v, M - (m0 + c0));
+        }
+      }
+      // this CTA's eight epilogue warps are done with the accumulator: one arrival at the leader
+      tc_fence_before();
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (threadIdx.x == 64) mbar_arrive_cluster(map_to_cta(acce0 + 8 * b, 0));
+    }
+    if (my_tiles == 0) grid_dep_launch();
+  }
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                                    // neither CTA frees while the other still reads
+  if (warp == 1) tmem_dealloc_pair(tmem, 2 * TN);
+}
+
+}  // namespace vadusa
