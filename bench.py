@@ -487,7 +487,7 @@ def run_ours(args):
             batched = {}
             for name in ("C3", "C4"):
                 ab = copy.copy(args)
-                ab.workload, ab.steps, ab.batch, ab.prefill_rows = name, 64, 0, 64
+                ab.workload, ab.steps, ab.batch, ab.prefill_rows = name, 64, 0, 256
                 batched[name.lower()] = [{"workload": ln["config"]["workload"], "tokens_per_s": ln["value"],
                                           "ms_per_step": ln["ms_per_step"],
                                           "mean_accepted_tokens": ln["config"]["mean_accepted_tokens"],
@@ -708,7 +708,7 @@ def main():
                     help="C2: the headline step (default); C3, C4: the batched configurations; C5: verify-step "
                          "microbenchmark at batch 64")
     ap.add_argument("--batch", type=int, default=0, help="C3, C4, C5: smaller batch (for profiler captures)")
-    ap.add_argument("--prefill-rows", type=int, default=64,
+    ap.add_argument("--prefill-rows", type=int, default=256,
                     help="C3, C4: prefix chunks of 64 tokens scored per prefill pass (0: one per sequence)")
     ap.add_argument("--tree-nodes", type=int, default=0, choices=[0, 64, 96, 128],
                     help="C2 only: candidate-tree size (default: the workload's 64 nodes)")

@@ -10,9 +10,8 @@
 // Per 64-key page:  S = Q K^T (128 x 64) -> two threads per row (eight softmax warps): each reads all 64
 // scores of the row for the scaling maximum (so both use the same one without talking to each other; it moves
 // lazily, as in the tree kernel), masks by position, exponentiates its own 32 keys and writes the weights as two
-// bf16 halves (hi, lo) into a weight buffer of its own (not over the scores, which the row's other thread may
-// still be reading) -> O += P V.  TMEM: three score buffers (columns 0..191), O (192..255), three weight
-// buffers (256..447).  Rings, barriers and bounded waits are those of tree_attention_tc_kernel.
+// bf16 halves (hi, lo) over the scores once all softmax threads have read them (a named barrier per page)
+// -> O += P V.  TMEM: three score / weight buffers (columns 0..191), O (192..255): two CTAs per SM.  Rings, barriers and bounded waits are those of tree_attention_tc_kernel.
 // Warps: 0-7 softmax (warp w and w + 4 share TMEM lanes 32 (w % 4) ..), 8 TMA producer, 9 TMEM owner / P V issuer,
 // 10 Q K^T issuer.
 #pragma once
@@ -50,7 +49,7 @@ __device__ __forceinline__ void tmem_ld32x2(uint32_t ta, float* a, uint32_t tb, 
   for (int i = 0; i < 32; ++i) { a[i] = __uint_as_float(r[i]); b[i] = __uint_as_float(q[i]); }
 }
 
-__global__ void __launch_bounds__(kPfThreads, 1) prefill_attention_tc_kernel(
+__global__ void __launch_bounds__(kPfThreads, 2) prefill_attention_tc_kernel(
     const __grid_constant__ CUtensorMap tmQ,    // q [1][rows * 64][d_model], box 64 x 64
     const __grid_constant__ CUtensorMap tmKV,   // pool [layers][blocks * 2 * heads * 64][64], box 64 x 64
     int layer, const int32_t* __restrict__ block_table /*[rows][max_blocks]*/, const int32_t* __restrict__ ctx_len,
@@ -66,6 +65,7 @@ __global__ void __launch_bounds__(kPfThreads, 1) prefill_attention_tc_kernel(
   const uint32_t full_k0 = bars, empty_k0 = bars + 8 * SK, full_v0 = bars + 16 * SK, empty_v0 = full_v0 + 8 * SV,
                  bar_q = bars + 16 * (SK + SV), bar_s0 = bar_q + 8, bar_p0 = bar_q + 32, bar_o0 = bar_q + 56, holder = bar_q + 80;
   volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(ring_ptr + kAttRingBytes + 1024 + 16 * (SK + SV) + 80);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(ring_ptr + kAttRingBytes + 1024 + 16 * (SK + SV) + 84);   // a wait of the softmax threads ran out
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int h = blockIdx.x;
@@ -74,11 +74,12 @@ __global__ void __launch_bounds__(kPfThreads, 1) prefill_attention_tc_kernel(
     for (int s = 0; s < 2 * (SK + SV); ++s) mbar_init(bars + 8 * s, 1);
     mbar_init(bar_q, 1); mbar_init(bar_s0, 1); mbar_init(bar_s0 + 8, 1); mbar_init(bar_s0 + 16, 1);
     for (int j = 0; j < 3; ++j) { mbar_init(bar_p0 + 8 * j, 256); mbar_init(bar_o0 + 8 * j, 1); }
+    *s_abort = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmQ);
     tma_prefetch_desc(&tmKV);
   }
-  if (warp == 9) { tmem_alloc(holder, 512); tmem_relinquish(); }
+  if (warp == 9) { tmem_alloc(holder, 256); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -143,7 +144,7 @@ __global__ void __launch_bounds__(kPfThreads, 1) prefill_attention_tc_kernel(
         if (!mbar_wait(bar_p0 + 8 * (i % 3), (i / 3) & 1, err)) break;
         if (!mbar_wait(full_v0 + 8 * (i % SV), (i / SV) & 1, err)) break;
         tc_fence_after();
-        const uint32_t va = ring_v + (i % SV) * kAttTileBytes, pa = tmem + 256 + 64 * (i % 3);
+        const uint32_t va = ring_v + (i % SV) * kAttTileBytes, pa = tmem + 64 * (i % 3);
 #pragma unroll
         for (int k = 0; k < 4; ++k)
           umma_bf16_ts(tmem + 192, pa + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, (i | k) != 0);
@@ -160,9 +161,8 @@ __global__ void __launch_bounds__(kPfThreads, 1) prefill_attention_tc_kernel(
       constexpr uint32_t idesc_qk = umma_idesc_bf16(128, 64);
       bool ok = ntiles == 0 || mbar_wait(bar_q, 0, err);
       for (int i = 0; i < ntiles && ok; ++i) {
-        // score buffer i % 3 held page i - 3: free once the softmax threads are done with it (the weights have a
-        // buffer of their own, so this does not wait for that page's P V)
-        if (i >= 3 && !mbar_wait(bar_p0 + 8 * (i % 3), ((i - 3) / 3) & 1, err)) break;
+        // score buffer i % 3 held the weights of page i - 3: free once that page's P V has completed
+        if (i >= 3 && !mbar_wait(bar_o0 + 8 * (i % 3), ((i - 3) / 3) & 1, err)) break;
         const int s = i % SK;
         if (!mbar_wait(full_k0 + 8 * s, (i / SK) & 1, err)) break;
         tc_fence_after();
@@ -183,10 +183,18 @@ __global__ void __launch_bounds__(kPfThreads, 1) prefill_attention_tc_kernel(
     const int qpos = (second ? ctxB : ctxA) + r;                  // this row's own position: the last key it sees
     const bool live = r < nv_h;
     const uint32_t trow = tmem + ((uint32_t)(32 * (warp & 3)) << 16);
+    // The softmax threads meet at a named barrier on every page, so none of them may leave the loop early: after a
+    // wait has run out (recorded in the error word) the remaining waits return at once and the loop runs to its end.
+    auto wait_ok = [&](uint32_t bar, uint32_t parity) -> bool {
+      if (*s_abort) return false;
+      if (mbar_wait(bar, parity, err)) return true;
+      *s_abort = 1;
+      return false;
+    };
     for (int i = 0; i < ntiles; ++i) {
-      if (!mbar_wait(bar_s0 + 8 * (i % 3), (i / 3) & 1, err)) break;
+      wait_ok(bar_s0 + 8 * (i % 3), (i / 3) & 1);
       tc_fence_after();
-      const uint32_t tsp = trow + 64 * (i % 3), tpp = trow + 256 + 64 * (i % 3);
+      const uint32_t tsp = trow + 64 * (i % 3), tpp = tsp;       // the weights go over the scores
       // keys i*64 + j with j < nvis are visible
       const int nvis = live ? min(max(qpos - i * kKvBlock + 1, 0), kKvBlock) : 0;
       float sc[32], mx;
@@ -206,9 +214,11 @@ __global__ void __launch_bounds__(kPfThreads, 1) prefill_attention_tc_kernel(
         for (int j = 0; j < 32; ++j) mx4[j & 3] = fmax3(mx4[j & 3], sc[j], so[j]);
         mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       }
+      // every softmax thread has the scores in registers: the buffer may now take the weights
+      asm volatile("bar.sync 2, 256;" ::: "memory");
       if ((i + 1) * kKvBlock > total && tid < 64) {      // rows of V past the last token may hold anything: zero them
         const int valid = total - i * kKvBlock;
-        mbar_wait(full_v0 + 8 * (i % SV), (i / SV) & 1, err);
+        wait_ok(full_v0 + 8 * (i % SV), (i / SV) & 1);
         if (tid >= valid) {
           uint4* vr = reinterpret_cast<uint4*>(ring_ptr + (SK + i % SV) * kAttTileBytes + tid * 128);
 #pragma unroll
@@ -224,7 +234,7 @@ __global__ void __launch_bounds__(kPfThreads, 1) prefill_attention_tc_kernel(
       }
       if (i > 0 && __any_sync(0xffffffffu, factor != 1.f)) {
         // (both threads of a row see the same maxima, so they take this branch together: each rescales half of O)
-        if (!mbar_wait(bar_o0 + 8 * ((i - 1) % 3), ((i - 1) / 3) & 1, err)) break;
+        wait_ok(bar_o0 + 8 * ((i - 1) % 3), ((i - 1) / 3) & 1);
         tc_fence_after();
         float ot[32];
         tmem_ld32(trow + 192 + 32 * khalf, ot);
@@ -247,15 +257,13 @@ __global__ void __launch_bounds__(kPfThreads, 1) prefill_attention_tc_kernel(
         lv[j] = pack_bf16(pa - ha, pb - hb);
       }
       l_run += (psum4[0] + psum4[1]) + (psum4[2] + psum4[3]);
-      // weight buffer i % 3 was read by the P V of page i - 3 (issued two pages ago; normally long complete)
-      if (i >= 3 && !mbar_wait(bar_o0 + 8 * (i % 3), ((i - 3) / 3) & 1, err)) break;
       tmem_st16(tpp + 16 * khalf, hv);                   // keys 32 khalf .. +31: hi in columns 16 khalf .., lo in 32 + 16 khalf ..
       tmem_st16(tpp + 32 + 16 * khalf, lv);
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(bar_p0 + 8 * (i % 3));
     }
-    if (ntiles > 0) { mbar_wait(bar_o0 + 8 * ((ntiles - 1) % 3), ((ntiles - 1) / 3) & 1, err); tc_fence_after(); }
+    if (ntiles > 0) { wait_ok(bar_o0 + 8 * ((ntiles - 1) % 3), ((ntiles - 1) / 3) & 1); tc_fence_after(); }
   }
   __syncwarp();
   grid_dep_launch();
@@ -294,7 +302,7 @@ __global__ void __launch_bounds__(kPfThreads, 1) prefill_attention_tc_kernel(
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 9) tmem_dealloc(tmem, 512);
+  if (warp == 9) tmem_dealloc(tmem, 256);
 }
 
 }  // namespace vadusa
