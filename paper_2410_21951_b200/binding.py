@@ -69,7 +69,7 @@ EXPORTS = ["vadusa_workspace_bytes", "vadusa_weights_bytes", "vadusa_kv_pool_byt
            "vadusa_begin", "vadusa_prefill", "vadusa_load_state", "vadusa_draft", "vadusa_verify_step",
            "vadusa_accept_and_commit", "vadusa_generate", "vadusa_generate_host", "vadusa_get_lengths",
            "vadusa_check", "vadusa_kernel_launches", "vadusa_profile_begin", "vadusa_profile_end",
-           "vadusa_accept_stats", "vadusa_build_sparse_tree", "vadusa_set_logit_bias", "vadusa_set_fused_pass", "vadusa_fused_pass_clusters",
+           "vadusa_accept_stats", "vadusa_build_sparse_tree", "vadusa_set_logit_bias", "vadusa_set_fused_pass", "vadusa_fused_pass_clusters", "vadusa_set_attention_stream",
            "vadusa_fit_state_bytes", "vadusa_fit_begin", "vadusa_fit_step", "vadusa_fit_end", "vadusa_set_prefill_tap",
            "vadusa_draft_topk_static", "vadusa_static_scratch_bytes", "vadusa_static_last_error"]
 
@@ -103,6 +103,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "vadusa_get_lengths": (I32, [P, P]), "vadusa_check": (I32, [P]),
         "vadusa_kernel_launches": (I64, [P]),
         "vadusa_set_fused_pass": (I32, [P, I32]),
+        "vadusa_set_attention_stream": (I32, [P, I32]),
         "vadusa_fused_pass_clusters": (I32, [P]),
         "vadusa_fit_state_bytes": (I64, [cfgp, I32]),
         "vadusa_fit_begin": (I32, [P, P, I64, I32, C.c_float, C.c_float, I32]),
@@ -397,6 +398,10 @@ class Vadusa:
     def set_fused_pass(self, enable):
         """False / True, or 6 / 8 to ask for that cluster size."""
         self._ck(self.L.vadusa_set_fused_pass(self.ctx, int(enable)))
+
+    def set_attention_stream(self, enable):
+        """Batches: True (default) page-stream attention kernel, False one thread block per (head, sequence)."""
+        self._ck(self.L.vadusa_set_attention_stream(self.ctx, int(bool(enable))))
 
     def fused_pass_clusters(self) -> int:
         return int(self.L.vadusa_fused_pass_clusters(self.ctx))

@@ -15,6 +15,7 @@
 #include "attention_simt.cuh"
 #include "attention_tc.cuh"
 #include "attention_prefill_tc.cuh"
+#include "attention_stream_tc.cuh"
 #include "elementwise.cuh"
 #include "fit.cuh"
 #include "fwd_fused.cuh"
@@ -56,6 +57,7 @@ struct vadusa_ctx {
   void* pf_tap = nullptr;     // where prefill also leaves the final hidden state of every prefix token ([batch][stride][d])
   int pf_tap_stride = 0;
   int pf_tiles = 0;           // > 0 while a prefill pass runs: attention CTAs of the pass (pairs of chunks), listed in ws.pf_pairs
+  int att_stream = 1;         // batches: attention as one persistent kernel over the stream of K/V pages (0: one CTA per head and sequence)
   int fused_enabled = 0;      // single-sequence passes run as one persistent kernel (0: no, 1: yes, 6 / 8: with that cluster size)
   int fused_clusters = -1;    // clusters of that kernel that can be resident at once on this device (-1: not asked yet)
   int fused_cs = -1;          // CTAs per cluster chosen for it (8 or 6; 0: the device cannot hold one cluster per head)
@@ -471,6 +473,13 @@ int attention_splits(const vadusa_ctx* ctx, int n_nodes) {
   return splits;
 }
 
+// Batches whose (head, sequence) items alone fill the device go through the persistent page-stream kernel.
+bool attention_streams(const vadusa_ctx* ctx, int n_nodes) {
+  const vadusa_config& c = ctx->cfg;
+  return ctx->att_stream && c.dtype == 1 && c.d_model / c.n_heads == 64 && n_nodes <= 64 && ctx->batch <= kAsMaxBatch &&
+         attention_splits(ctx, n_nodes) == 1 && (long long)c.max_blocks_per_seq * kKvBlock < (1ll << 24);
+}
+
 template <typename T>
 vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeView& tv, T* out) {
   const vadusa_config& c = ctx->cfg;
@@ -528,6 +537,26 @@ vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeVi
       if (vadusa_status s = tensor_map(ctx, c.kv_pool, (int)rows, 64, 64, c.n_layers, g.layer_stride, &mkv)) return s;
       const int layer = (int)((reinterpret_cast<const char*>(pool) - reinterpret_cast<const char*>(c.kv_pool)) /
                               (g.layer_stride * (long long)sizeof(bf16)));
+      if (attention_streams(ctx, tv.n_nodes)) {
+        // batches: every CTA takes an equal share of the stream of K/V pages of all (sequence, head) items
+        cudaLaunchConfig_t lc = {};
+        lc.gridDim = dim3(kAsGrid);
+        lc.blockDim = dim3(kAsThreads);
+        lc.dynamicSmemBytes = kAsSmemBytes;
+        lc.stream = ctx->stream;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = at; lc.numAttrs = 1;
+        PROF(ctx, K_ATTENTION);
+        CU(cudaLaunchKernelEx(&lc, tree_attention_stream_kernel, *mq, *mkv, layer, ctx->block_table,
+                              (const int32_t*)wsptr<int32_t>(ctx, ctx->ws.ctx_len),
+                              (const int32_t*)wsptr<int32_t>(ctx, ctx->ws.nvalid), tv, g, ctx->batch, c.d_model,
+                              scale * 1.4426950408889634f, reinterpret_cast<bf16*>(out),
+                              wsptr<float>(ctx, ctx->ws.att_xch), wsptr<uint32_t>(ctx, ctx->ws.att_cnt), err_word(ctx)));
+        LAUNCH_CHECK();
+        return VADUSA_OK;
+      }
       cudaLaunchConfig_t lc = {};
       lc.gridDim = dim3(c.n_heads, ctx->batch * ntile, splits);
       lc.blockDim = dim3(kAttThreads);
@@ -540,7 +569,8 @@ vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeVi
       at[1].val.programmaticStreamSerializationAllowed = 1;
       lc.attrs = at; lc.numAttrs = 2;
       PROF(ctx, K_ATTENTION);
-      CU(cudaLaunchKernelEx(&lc, tree_attention_tc_kernel, *mq, *mkv, layer, ctx->block_table,
+      // several splits: few pages per CTA, the weights keep 16 significant bits; one split: a batch, bf16 weights
+      CU(cudaLaunchKernelEx(&lc, splits > 1 ? tree_attention_tc_kernel<true> : tree_attention_tc_kernel<false>, *mq, *mkv, layer, ctx->block_table,
                             (const int32_t*)wsptr<int32_t>(ctx, ctx->ws.ctx_len),
                             (const int32_t*)wsptr<int32_t>(ctx, ctx->ws.nvalid),
                             (const int32_t*)(ctx->batch > 1 ? wsptr<int32_t>(ctx, ctx->ws.seq_order) : nullptr), tv, g, c.d_model,
@@ -1018,14 +1048,18 @@ vadusa_status set_kernel_attributes(vadusa_ctx* ctx) {
   CU(cudaFuncSetAttribute(tree_attention_simt_kernel<float, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(32)));
   CU(cudaFuncSetAttribute(tree_attention_simt_kernel<bf16, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(64)));
   CU(cudaFuncSetAttribute(tree_attention_simt_kernel<bf16, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(32)));
-  CU(cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmemBytes));
+  CU(cudaFuncSetAttribute(tree_attention_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmemBytes));
+  CU(cudaFuncSetAttribute(tree_attention_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmemBytes));
   CU(cudaFuncSetAttribute(prefill_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmemBytes));
+  CU(cudaFuncSetAttribute(tree_attention_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAsSmemBytes));
   CU(cudaFuncSetAttribute(prefill_attention_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
   // the accept kernel keeps one row of keys and one of probabilities in shared memory.  The limit is an attribute of
   // the function on this device, shared by every context: always the library's largest vocabulary
   CU(cudaFuncSetAttribute(accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 24576 * (int)sizeof(float)));
   // ask for the largest shared-memory carve-out so that several CTAs fit on an SM
-  CU(cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+  CU(cudaFuncSetAttribute(tree_attention_tc_kernel<true>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+  CU(cudaFuncSetAttribute(tree_attention_tc_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+  CU(cudaFuncSetAttribute(tree_attention_stream_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
   return VADUSA_OK;
 }
 
@@ -1194,6 +1228,7 @@ vadusa_status vadusa_init(const vadusa_weights* weights, const vadusa_config* cf
   CU(cudaMemsetAsync(ctx->wsp, 0, ctx->ws.tokens, ctx->stream));     // scalars, per-sequence state, trees
   CU(cudaMemsetAsync(ctx->wsp + ctx->ws.acc_stats, 0, 2ull * kStatDepth * kStatTopk * 8, ctx->stream));
   CU(cudaMemsetAsync(ctx->wsp + ctx->ws.f_sync, 0, 256, ctx->stream));
+  CU(cudaMemsetAsync(ctx->wsp + ctx->ws.att_cnt, 0, 2 * kAsGrid * 4, ctx->stream));
   // chain-shaped tree used by prefill: node i is the child of node i-1
   constexpr int T = VADUSA_MAX_TREE_NODES;
   static_assert(T == kMaxNodes, "node limit of the kernels");
@@ -1292,6 +1327,7 @@ vadusa_status vadusa_begin(vadusa_ctx* ctx, int32_t batch, const int32_t* block_
   ctx->have_draft = ctx->have_verify = false;
   CU(cudaMemsetAsync(ctx->wsp + ctx->ws.scalars, 0, 256, ctx->stream));
   CU(cudaMemsetAsync(ctx->wsp + ctx->ws.f_sync, 0, 256, ctx->stream));
+  CU(cudaMemsetAsync(ctx->wsp + ctx->ws.att_cnt, 0, 2 * kAsGrid * 4, ctx->stream));
   CU(cudaMemsetAsync(ctx->wsp + ctx->ws.gen_count, 0, batch * 4, ctx->stream));
   ctx->ctx_bound = 0;
   if (h_ctx_len) {
@@ -1383,7 +1419,7 @@ vadusa_status vadusa_verify_step(vadusa_ctx* ctx, const int32_t* tree_tokens_ove
   const int M = ctx->batch * tv.n_nodes;
   const std::string key = KeyBuilder("verify").add(tree_tokens_override).add(logits_out).add(attn_tap).add(hidden_out)
                               .add(ctx->batch).add(ctx->n_nodes).add(ctx->tree_per_seq).add(ctx->block_table)
-                              .add(attention_splits(ctx, ctx->n_nodes)).add(ctx->fused_enabled).k;
+                              .add(attention_splits(ctx, ctx->n_nodes)).add(ctx->fused_enabled).add(ctx->att_stream).k;
   vadusa_status s = run_graphed(ctx, key, [&]() -> vadusa_status {
     vadusa_status s = DISPATCH(forward<float>(ctx, tv, tree_tokens_override, reinterpret_cast<float*>(attn_tap)),
                                forward<bf16>(ctx, tv, tree_tokens_override, reinterpret_cast<bf16*>(attn_tap)));
@@ -1452,7 +1488,7 @@ vadusa_status vadusa_generate(vadusa_ctx* ctx, const vadusa_sampling* sampling, 
       if (ctx->h_pinned[0] >= ctx->batch) break;
     }
     const std::string iter_key = KeyBuilder("iteration").add(sp).add(out_tokens).add(max_new_tokens).add(ctx->batch)
-                                     .add(ctx->n_nodes).add(ctx->block_table).add(attention_splits(ctx, ctx->n_nodes)).add(ctx->fused_enabled).k;
+                                     .add(ctx->n_nodes).add(ctx->block_table).add(attention_splits(ctx, ctx->n_nodes)).add(ctx->fused_enabled).add(ctx->att_stream).k;
     vadusa_status s = run_graphed(ctx, iter_key, [&]() -> vadusa_status {
       vadusa_status s = DISPATCH(draft<float>(ctx, sp), draft<bf16>(ctx, sp));
       if (s) return s;
@@ -1643,6 +1679,13 @@ vadusa_status vadusa_set_prefill_tap(vadusa_ctx* ctx, void* hidden_out, int32_t 
 int64_t vadusa_kernel_launches(const vadusa_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 int32_t vadusa_fused_pass_clusters(const vadusa_ctx* ctx) { return ctx ? ctx->fused_clusters : -1; }
+
+vadusa_status vadusa_set_attention_stream(vadusa_ctx* ctx, int32_t enable) {
+  if (!ctx) return VADUSA_EINVAL;
+  if (enable != 0 && enable != 1) return fail(ctx, VADUSA_EINVAL, "enable must be 0 or 1");
+  ctx->att_stream = enable;
+  return VADUSA_OK;
+}
 
 vadusa_status vadusa_set_fused_pass(vadusa_ctx* ctx, int32_t enable) {
   if (!ctx) return VADUSA_EINVAL;

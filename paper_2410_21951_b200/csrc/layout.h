@@ -111,7 +111,8 @@ struct WorkspaceLayout {
   int64_t logits;                        // fp32 [M][vpad]
   int64_t hstar, logits_star;            // T [B][d], fp32 [B][vpad]
   int64_t z, dlogits;                    // T [heads][B][d], fp32 [heads][B][vpad]
-  int64_t att_xch;                       // fp32 split-KV exchange of the attention kernel: 296 slots of 64*64+128 floats
+  int64_t att_xch;                       // fp32 split-KV exchange of the attention kernels: 592 slots of 64*64+128 floats
+  int64_t att_cnt;                       // uint32 [592]: parts of an item that have arrived (page-stream attention); zero between launches
   int64_t gemm_part;                     // fp32 split-K exchange of the tensor-core products (kGemmPartBytes)
   int64_t ln_stats;                      // per-group LayerNorm statistics for the fused products (kLnStatsBytes)
   int64_t acc_stats;                     // uint64 [2][VADUSA_MAX_DEPTH][VADUSA_MAX_DRAFT_TOPK]: edges tested, edges accepted
@@ -152,7 +153,8 @@ inline WorkspaceLayout workspace_layout(const vadusa_config* c) {
   w.logits = take(M * vp * 4);
   w.hstar = take(B * d * es); w.logits_star = take(B * vp * 4);
   w.z = take(hd * B * d * es); w.dlogits = take(hd * B * vp * 4);
-  w.att_xch = take(296ll * (64 * 64 + 128) * 4);
+  w.att_xch = take(592ll * (64 * 64 + 128) * 4);
+  w.att_cnt = take(592 * 4);
   w.gemm_part = take(kGemmPartBytes);
   w.ln_stats = take(kLnStatsBytes);
   w.acc_stats = take(2ll * VADUSA_MAX_DEPTH * VADUSA_MAX_DRAFT_TOPK * 8);
