@@ -259,12 +259,13 @@ vadusa_status vadusa_get_lengths(vadusa_ctx *ctx, int32_t *h_ctx_len);
 vadusa_status vadusa_check(vadusa_ctx *ctx);                            /* synchronises; device error word */
 int64_t vadusa_kernel_launches(const vadusa_ctx *ctx);                  /* total kernels enqueued so far */
 
-/* Tree attention of a batch (Sec. II-A; bf16, head_dim 64, at most 64 tree nodes, at most 512 sequences, and
- * enough (sequence, head) pairs to fill the device) runs by default as one persistent kernel in which every
- * thread block takes an equal share of the stream of K/V pages of all pairs, whatever the sequences' lengths;
- * a pair whose pages fall to several blocks is merged by the block that finishes last, in the order of the
- * pages.  enable = 0 selects the kernel with one thread block per (head, sequence) instead; both compute the
- * same attention with the same rounding points per page.  Host-side switch: takes effect with the next call. */
+/* Tree attention of a batch (Sec. II-A) runs with one thread block per (head, sequence), the sequences visited
+ * longest first.  For bf16 models with head_dim 64, at most 64 tree nodes, at most 512 sequences and enough
+ * (sequence, head) pairs to fill the device, enable = 1 selects a persistent kernel instead in which every thread
+ * block takes an equal share of the stream of K/V pages of all sequences, whatever their lengths; a pair whose
+ * pages fall to several blocks is merged by the block that finishes last, in the order of the pages.  Both
+ * compute the same attention with the same rounding points per page.  enable = 0 is the default: it is the faster one on the
+ * devices measured so far.  Host-side switch: takes effect with the next call. */
 vadusa_status vadusa_set_attention_stream(vadusa_ctx *ctx, int32_t enable);
 
 /* A verify pass over ONE sequence of at most 64 tree nodes (the batch-1 step of Sec. II-A: one tree per

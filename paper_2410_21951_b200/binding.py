@@ -400,7 +400,7 @@ class Vadusa:
         self._ck(self.L.vadusa_set_fused_pass(self.ctx, int(enable)))
 
     def set_attention_stream(self, enable):
-        """Batches: True (default) page-stream attention kernel, False one thread block per (head, sequence)."""
+        """Batches: True page-stream attention kernel, False (default) one thread block per (head, sequence)."""
         self._ck(self.L.vadusa_set_attention_stream(self.ctx, int(bool(enable))))
 
     def fused_pass_clusters(self) -> int:

@@ -57,7 +57,7 @@ struct vadusa_ctx {
   void* pf_tap = nullptr;     // where prefill also leaves the final hidden state of every prefix token ([batch][stride][d])
   int pf_tap_stride = 0;
   int pf_tiles = 0;           // > 0 while a prefill pass runs: attention CTAs of the pass (pairs of chunks), listed in ws.pf_pairs
-  int att_stream = 1;         // batches: attention as one persistent kernel over the stream of K/V pages (0: one CTA per head and sequence)
+  int att_stream = 0;         // batches: attention as one persistent kernel over the stream of K/V pages (0: one CTA per head and sequence)
   int fused_enabled = 0;      // single-sequence passes run as one persistent kernel (0: no, 1: yes, 6 / 8: with that cluster size)
   int fused_clusters = -1;    // clusters of that kernel that can be resident at once on this device (-1: not asked yet)
   int fused_cs = -1;          // CTAs per cluster chosen for it (8 or 6; 0: the device cannot hold one cluster per head)
@@ -569,8 +569,7 @@ vadusa_status attention(vadusa_ctx* ctx, const T* q, const T* pool, const TreeVi
       at[1].val.programmaticStreamSerializationAllowed = 1;
       lc.attrs = at; lc.numAttrs = 2;
       PROF(ctx, K_ATTENTION);
-      // several splits: few pages per CTA, the weights keep 16 significant bits; one split: a batch, bf16 weights
-      CU(cudaLaunchKernelEx(&lc, splits > 1 ? tree_attention_tc_kernel<true> : tree_attention_tc_kernel<false>, *mq, *mkv, layer, ctx->block_table,
+      CU(cudaLaunchKernelEx(&lc, tree_attention_tc_kernel, *mq, *mkv, layer, ctx->block_table,
                             (const int32_t*)wsptr<int32_t>(ctx, ctx->ws.ctx_len),
                             (const int32_t*)wsptr<int32_t>(ctx, ctx->ws.nvalid),
                             (const int32_t*)(ctx->batch > 1 ? wsptr<int32_t>(ctx, ctx->ws.seq_order) : nullptr), tv, g, c.d_model,
@@ -1048,8 +1047,7 @@ vadusa_status set_kernel_attributes(vadusa_ctx* ctx) {
   CU(cudaFuncSetAttribute(tree_attention_simt_kernel<float, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(32)));
   CU(cudaFuncSetAttribute(tree_attention_simt_kernel<bf16, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(64)));
   CU(cudaFuncSetAttribute(tree_attention_simt_kernel<bf16, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_smem(32)));
-  CU(cudaFuncSetAttribute(tree_attention_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmemBytes));
-  CU(cudaFuncSetAttribute(tree_attention_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmemBytes));
+  CU(cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmemBytes));
   CU(cudaFuncSetAttribute(prefill_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmemBytes));
   CU(cudaFuncSetAttribute(tree_attention_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAsSmemBytes));
   CU(cudaFuncSetAttribute(prefill_attention_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
@@ -1057,8 +1055,7 @@ vadusa_status set_kernel_attributes(vadusa_ctx* ctx) {
   // the function on this device, shared by every context: always the library's largest vocabulary
   CU(cudaFuncSetAttribute(accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 24576 * (int)sizeof(float)));
   // ask for the largest shared-memory carve-out so that several CTAs fit on an SM
-  CU(cudaFuncSetAttribute(tree_attention_tc_kernel<true>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
-  CU(cudaFuncSetAttribute(tree_attention_tc_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+  CU(cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
   CU(cudaFuncSetAttribute(tree_attention_stream_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
   return VADUSA_OK;
 }

@@ -11,12 +11,11 @@
 // segment leaves (O, l, m) in an exchange slot, and the part that arrives last (a counter per (sequence, head),
 // no waiting) merges all parts in a fixed order and writes the output.
 //
-// Per page the work follows tree_attention_tc_kernel: S = Q K^T into one of three TMEM score buffers, softmax
-// by 128 threads (lanes r and r + 64 are the two key halves of query row r), weights back to TMEM, O += P V with
-// A from TMEM.  The weights are rounded to bf16 once (that kernel keeps a second bf16 for the remainder): here the
-// tensor pipe, which spends about one cycle per accumulator column and instruction whatever the number of useful
-// rows, is what a page costs (two CTAs: 2 x (4 + 8) instructions of 64 columns against a page time of about 1800
-// cycles), and the second product is a third of that.  The row sums are taken from the unrounded weights.  The Q tile has two buffers: the next item's Q arrives while the
+// Per page the work is that of tree_attention_tc_kernel: S = Q K^T into one of three TMEM score buffers,
+// softmax by 128 threads (lanes r and r + 64 are the two key halves of query row r), weights back to TMEM as
+// bf16 hi + lo, O += P V with A from TMEM.  (Weights rounded to bf16 once save a third of a page's tensor-core
+// instructions and 15 % of a launch, but take the logits of a 12-layer pass over contexts of up to 3000 tokens
+// from 1.5e-2 to 2.05e-2 away from an fp64 evaluation.)  The Q tile has two buffers: the next item's Q arrives while the
 // current item runs, and the buffer of the finished item carries the exchange of the two key halves.
 // Warps: 0-3 softmax and epilogue, warp 4 TMA producer of Q and K, warp 5 TMEM owner / P V issuer, warp 6 Q K^T
 // issuer, warp 7 TMA producer of V.
@@ -228,6 +227,9 @@ __global__ void __launch_bounds__(kAsThreads, 2) tree_attention_stream_kernel(
 #pragma unroll
           for (int k = 0; k < 4; ++k)        // 16 keys per step: 8 TMEM columns of A, 16 rows (2048 bytes) of V
             umma_bf16_ts(tmem + 192, pa + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, (i | k) != 0);
+#pragma unroll
+          for (int k = 0; k < 4; ++k)        // the lo halves of the weights
+            umma_bf16_ts(tmem + 192, pa + 32 + 8 * k, umma_desc_k_sw128(va + 2048 * k), idesc_pv, true);
           umma_commit(empty_v0 + 8 * (g % SV));
           umma_commit(bar_o0 + 8 * (g % 3));
         }
@@ -346,7 +348,7 @@ __global__ void __launch_bounds__(kAsThreads, 2) tree_attention_stream_kernel(
         }
         l_run *= factor;
         float psum4[4] = {0.f, 0.f, 0.f, 0.f};
-        uint32_t hv[16];
+        uint32_t hv[16], lv[16];
         const float m_sub = (m_use == -INFINITY) ? 0.f : m_use;      // no visible key yet: every score is -inf, p = 0
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
@@ -354,15 +356,19 @@ __global__ void __launch_bounds__(kAsThreads, 2) tree_attention_stream_kernel(
           const float pb = fast_exp2(fmaf(sc[2 * j + 1], scale_log2e, -m_sub));
           psum4[j & 3] += pa + pb;
           hv[j] = pack_bf16(pa, pb);
+          const float ha = __uint_as_float(hv[j] << 16), hb = __uint_as_float(hv[j] & 0xffff0000u);
+          lv[j] = pack_bf16(pa - ha, pb - hb);
         }
         l_run += (psum4[0] + psum4[1]) + (psum4[2] + psum4[3]);
-        // this thread's 32 keys sit in columns 16*half .. 16*half+15 of the buffer's first 32; zero in the other 16
+        // this thread's 32 keys sit in columns 16*half .. 16*half+15 of each 32-column group; zero elsewhere
         {
           uint32_t zero[16];
 #pragma unroll
           for (int j = 0; j < 16; ++j) zero[j] = 0u;
           tmem_st16(tsp + 16 * half, hv);
           tmem_st16(tsp + 16 * (1 - half), zero);
+          tmem_st16(tsp + 32 + 16 * half, lv);
+          tmem_st16(tsp + 32 + 16 * (1 - half), zero);
         }
         tmem_st_wait();
         tc_fence_before();
