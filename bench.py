@@ -34,7 +34,7 @@ TREE_NODES = 0          # 0: the workload's own tree; --tree-nodes 96 / 128: the
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the 49 projection launches of one C2 step, from the
 # ncu capture of those launches (batch 1, 64 nodes); valid for the kernel sources with this hash only.
-_NCU_TRAFFIC = {"src_sha256_16": "c556915c27437597", "bytes_per_step": 327.98e6, "launches": 49}
+_NCU_TRAFFIC = {"src_sha256_16": "e4985711aa50c962", "bytes_per_step": 327.98e6, "launches": 49}
 
 
 def _gemm_traffic():
@@ -49,10 +49,10 @@ def _gemm_traffic():
 
 
 # DRAM bytes of one tree_attention_tc_kernel launch relative to its algorithmic K/V bytes, from the ncu capture at
-# 24 sequences (163.17 MB read + 3.83 MB written for
-# 163.1 MB of K/V); every (head, sequence) CTA reads its own pages once, so the traffic of a launch grows in
-# proportion to its sequences' bytes.  Valid for the kernel sources with this hash only.
-_NCU_ATTN = {"src_sha256_16": "a1b015d014f84a83", "dram_over_algorithmic": 167.0 / 163.1}
+# 24 sequences (two launches: 163.17 / 163.15 MB read, 3.15 / 0.13 MB written, for 163.1 MB of K/V); every
+# (head, sequence) CTA reads its own pages once, so the traffic of a launch grows in proportion to its sequences'
+# bytes.  Valid for the kernel sources with this hash only.
+_NCU_ATTN = {"src_sha256_16": "2acaf0fd3fd1cdbc", "dram_over_algorithmic": 164.8 / 163.1}
 
 
 def _attn_traffic(algorithmic_bytes):
