@@ -63,6 +63,7 @@ struct vadusa_ctx {
   int fused_cs = -1;          // CTAs per cluster chosen for it (8 or 6; 0: the device cannot hold one cluster per head)
   int fused_n8 = 0, fused_n6 = 0;
   long long ctx_bound = 0;    // host-side upper bound of the longest context (grows by the longest path per commit)
+  long long ctx_lo = 0;       // host-side lower estimate of it (one token per iteration); exact after begin, prefill, get_lengths
   const int32_t* block_table = nullptr;
   bool have_draft = false, have_verify = false;
   int64_t launches = 0;
@@ -464,12 +465,18 @@ bool ln_product(vadusa_ctx* ctx, int cls, const float* x, const float* g, const 
   return false;
 }
 
-// KV splits of the tensor-core attention: enough CTAs for about two per SM even at batch 1.
+// KV splits of the tensor-core attention: enough CTAs for about two per SM even at batch 1, but no more than four
+// per (head, sequence) while the contexts are short (a 16-head pass over 400-1100 tokens: 64 CTAs of two to five
+// pages leave SMs to the next kernel's early CTAs and their weight loads, 128 CTAs of one or two pages do not;
+// 0.538 -> 0.528 ms per step).  The estimate of the context is the host's lower one: never behind by more than
+// the tokens accepted beyond one per iteration since the last exact value.
 // (Ragged batches are balanced by visiting the sequences longest first, see seq_order_kernel.)
+constexpr long long kAttLongContext = 1536;
 int attention_splits(const vadusa_ctx* ctx, int n_nodes) {
   int splits = 1;
   const int ntile = (n_nodes + 63) / 64;                 // CTAs per (head, sequence): one per 64 nodes
-  while (splits < 8 && ctx->cfg.n_heads * ctx->batch * ntile * splits * 2 <= 296) splits *= 2;
+  const int cap = ctx->ctx_lo + n_nodes > kAttLongContext ? 8 : 4;
+  while (splits < cap && ctx->cfg.n_heads * ctx->batch * ntile * splits * 2 <= 296) splits *= 2;
   return splits;
 }
 
@@ -944,6 +951,7 @@ vadusa_status prefill(vadusa_ctx* ctx, const int32_t* h_tokens, const int32_t* h
       }
   }
   ctx->ctx_bound += longest;
+  ctx->ctx_lo += longest;
   CU(cudaStreamSynchronize(ctx->stream));
   return VADUSA_OK;
 }
@@ -1327,12 +1335,14 @@ vadusa_status vadusa_begin(vadusa_ctx* ctx, int32_t batch, const int32_t* block_
   CU(cudaMemsetAsync(ctx->wsp + ctx->ws.att_cnt, 0, 2 * kAsGrid * 4, ctx->stream));
   CU(cudaMemsetAsync(ctx->wsp + ctx->ws.gen_count, 0, batch * 4, ctx->stream));
   ctx->ctx_bound = 0;
+  ctx->ctx_lo = 0;
   if (h_ctx_len) {
     for (int b = 0; b < batch; ++b) {
       if (h_ctx_len[b] < 0 || h_ctx_len[b] > (int64_t)ctx->cfg.max_blocks_per_seq * 64)
         return fail(ctx, VADUSA_EINVAL, "context length of sequence %d out of range", b);
       if (h_ctx_len[b] > ctx->ctx_bound) ctx->ctx_bound = h_ctx_len[b];
     }
+    ctx->ctx_lo = ctx->ctx_bound;
     CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.ctx_len, h_ctx_len, batch * 4, cudaMemcpyHostToDevice, ctx->stream));
     CU(cudaStreamSynchronize(ctx->stream));
   } else {
@@ -1450,6 +1460,7 @@ vadusa_status vadusa_accept_and_commit(vadusa_ctx* ctx, const vadusa_sampling* s
   });
   if (s) return s;
   ctx->ctx_bound += ctx->tree_max_depth + 1;
+  ctx->ctx_lo += 1;
   ctx->have_verify = ctx->have_draft = false;
   return VADUSA_OK;
 }
@@ -1496,6 +1507,7 @@ vadusa_status vadusa_generate(vadusa_ctx* ctx, const vadusa_sampling* sampling, 
     });
     if (s) return s;
     ctx->ctx_bound += ctx->tree_max_depth + 1;
+    ctx->ctx_lo += 1;
     if (!poll_pending && (iters & 7) == 7) {
       CU(cudaMemcpyAsync(ctx->h_pinned, done_word(ctx), 4, cudaMemcpyDeviceToHost, ctx->stream));
       CU(cudaEventRecord(ctx->ev_poll, ctx->stream));
@@ -1550,7 +1562,11 @@ vadusa_status vadusa_get_lengths(vadusa_ctx* ctx, int32_t* h_ctx_len) {
   if (vadusa_status s = need_batch(ctx)) return s;
   if (!h_ctx_len) return fail(ctx, VADUSA_EINVAL, "h_ctx_len is NULL");
   CU(cudaMemcpyAsync(h_ctx_len, ctx->wsp + ctx->ws.ctx_len, ctx->batch * 4, cudaMemcpyDeviceToHost, ctx->stream));
-  return device_errors(ctx);
+  if (vadusa_status s = device_errors(ctx)) return s;       // (synchronises)
+  long long longest = 0;
+  for (int b = 0; b < ctx->batch; ++b) longest = h_ctx_len[b] > longest ? h_ctx_len[b] : longest;
+  ctx->ctx_lo = ctx->ctx_bound = longest;                   // both estimates are exact again
+  return VADUSA_OK;
 }
 
 vadusa_status vadusa_check(vadusa_ctx* ctx) {

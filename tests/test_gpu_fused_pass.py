@@ -93,11 +93,12 @@ def test_fused_pass_planted_path_moves_rows_and_matches_stepwise_path():
     g.check()
 
 
-@pytest.mark.parametrize("ctx_len,cluster", [(37, 8), (1990, 8), (2500, 8), (2500, 6)])
+@pytest.mark.parametrize("ctx_len,cluster", [(37, 8), (1990, 8), (2500, 8), (2500, 6), (700, 0), (1500, 0), (2500, 0)])
 def test_fused_pass_long_context_with_injected_kv(ctx_len, cluster):
     """Seeded random K/V rows as context (no prefill on either side): 1 page, 32 pages (four per CTA: two
     groups) and 40 pages with a ragged last page (five per CTA); logits and attention outputs of every
-    node against the oracle's tree-masked pass."""
+    node against the oracle's tree-masked pass.  cluster = 0: the kernel-per-step path on the same inputs (its
+    attention kernel cuts one sequence's pages into four parts up to 1536 tokens and into eight beyond)."""
     import torch
     import paper_2410_21951_b200 as P
     wl = _wide_toy(64, heads=8, tree_caps=(10, 5, 3), index=41)
@@ -130,5 +131,5 @@ def test_fused_pass_long_context_with_injected_kv(ctx_len, cluster):
     e_a = max(np.abs(at[l] - out.attn[l]).max() for l in range(model.L))
     print(f"context {ctx_len}: max |logit err| {e_l:.2e}, max |attn err| {e_a:.2e}")
     assert e_l <= TOL["bf16"] and e_a <= TOL["bf16"]
-    assert g.fused_pass_clusters() >= 8
+    assert cluster == 0 or g.fused_pass_clusters() >= 8
     g.check()
