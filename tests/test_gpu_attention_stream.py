@@ -81,6 +81,14 @@ def test_page_stream_attention_on_ragged_batches(nodes, per_seq, lens_kind):
         g.check()
         taps[stream] = attn.float().cpu().numpy().astype(np.float64)
         lgs[stream] = logits.cpu().numpy().astype(np.float64)
+        if stream:
+            # once more from the same state: the counters of the merged pairs are back at zero, and whichever
+            # part of a pair arrives last, the parts are summed in the same order: bit-identical outputs
+            attn2 = torch.zeros_like(attn)
+            begin()
+            g.verify_step(override=dev_toks, attn_tap=attn2)
+            g.check()
+            assert torch.equal(attn, attn2)
     worst_a = worst_l = 0.0
     for b in range(B):
         tpl = tpls[b]
