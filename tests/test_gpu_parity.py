@@ -570,6 +570,7 @@ def test_long_ragged_contexts_with_injected_kv(name):
     g.accept_and_commit(sg, accept_len=acc, path_nodes=pn, kv_slots=sl, edge_bits=eb)
     lg = logits.cpu().numpy().astype(np.float64)
     at = attn.float().cpu().numpy().astype(np.float64)
+    first_pass = {}
     for b in picks:
         tpl = tpls[b]
         mask = np.zeros((N, N), dtype=bool)
@@ -577,6 +578,7 @@ def test_long_ragged_contexts_with_injected_kv(name):
             mask[n, tpl.node_path(n)] = True
         S = int(lens[b])
         out = O.forward_tree(model, states[b], [0] * N, toks[b], S + tpl.depth, mask)
+        first_pass[b] = out
         e_l = np.abs(lg[b] - out.logits).max()
         e_a = max(np.abs(at[l, b] - out.attn[l]).max() for l in range(model.L))
         print(f"{name} seq {b} (context {int(lens[b])}): max |logit err| {e_l:.2e}, max |attn err| {e_a:.2e}")
@@ -593,6 +595,22 @@ def test_long_ragged_contexts_with_injected_kv(name):
             assert list(sl[b, :len(path)].cpu().numpy()) == expected_slots(table, b, S, len(path))
     assert np.array_equal(g.lengths(), lens + acc.cpu().numpy())
     g.check()
+    # the same pass through the page-stream attention kernel (opt-in) at the full batch and context lengths
+    g.set_attention_stream(True)
+    g.begin(table, ctx_len=lens)
+    if wl.random_topology:
+        g.set_tree(np.stack([t.parent for t in tpls]), np.stack([t.rank for t in tpls]), per_sequence=True)
+    g.verify_step(override=torch.from_numpy(toks).to(g.dev), logits_out=logits, attn_tap=attn)
+    g.check()
+    g.set_attention_stream(False)
+    lg2 = logits.cpu().numpy().astype(np.float64)
+    at2 = attn.float().cpu().numpy().astype(np.float64)
+    for b in picks:
+        out = first_pass[b]
+        e_l = np.abs(lg2[b] - out.logits).max()
+        e_a = max(np.abs(at2[l, b] - out.attn[l]).max() for l in range(model.L))
+        print(f"{name} seq {b}, page-stream attention: max |logit err| {e_l:.2e}, max |attn err| {e_a:.2e}")
+        assert e_l <= TOL["bf16"] and e_a <= TOL["bf16"]
     if name != "C4":
         return
     # ---- tolerance sweep from the same state: the 1st, 3rd and 5th draw of the oracle at the root planted as
