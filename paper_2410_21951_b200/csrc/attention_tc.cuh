@@ -78,6 +78,35 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+// Two independent fp32 operations in one instruction (each half rounds as the scalar form does).
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
+      "mov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+  return d;
+}
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "add.rn.f32x2 rd, ra, rb;\n\t"
+      "mov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return d;
+}
+__device__ __forceinline__ float2 fsub2(float2 a, float2 b) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "sub.rn.f32x2 rd, ra, rb;\n\t"
+      "mov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return d;
+}
+
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
   float r;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
@@ -286,19 +315,26 @@ __global__ void __launch_bounds__(kAttThreads) tree_attention_tc_kernel(
         }
       }
       l_run *= factor;
-      float psum4[4] = {0.f, 0.f, 0.f, 0.f};
+      float2 psum4[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};   // four chains of pairs
       uint32_t hv[16], lv[16];
       const float m_sub = (m_use == -INFINITY) ? 0.f : m_use;      // no visible key yet: every score is -inf, p = 0
+      const float2 sc2 = make_float2(scale_log2e, scale_log2e), nm2 = make_float2(-m_sub, -m_sub);
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
-        const float pa = fast_exp2(fmaf(sc[2 * j], scale_log2e, -m_sub));
-        const float pb = fast_exp2(fmaf(sc[2 * j + 1], scale_log2e, -m_sub));
-        psum4[j & 3] += pa + pb;
-        hv[j] = pack_bf16(pa, pb);
-        const float ha = __uint_as_float(hv[j] << 16), hb = __uint_as_float(hv[j] & 0xffff0000u);
-        lv[j] = pack_bf16(pa - ha, pb - hb);
+        // two keys per instruction where the pipe has a paired form (fma, add, sub)
+        const float2 x = ffma2(make_float2(sc[2 * j], sc[2 * j + 1]), sc2, nm2);
+        const float2 pp = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+        psum4[j & 3] = fadd2(psum4[j & 3], pp);
+        hv[j] = pack_bf16(pp.x, pp.y);
+        const float2 hh = make_float2(__uint_as_float(hv[j] << 16), __uint_as_float(hv[j] & 0xffff0000u));
+        const float2 ll = fsub2(pp, hh);
+        lv[j] = pack_bf16(ll.x, ll.y);
       }
-      l_run += (psum4[0] + psum4[1]) + (psum4[2] + psum4[3]);
+      {
+        const float2 s01 = fadd2(psum4[0], psum4[1]), s23 = fadd2(psum4[2], psum4[3]);
+        const float2 st = fadd2(s01, s23);
+        l_run += st.x + st.y;
+      }
       // this thread's 32 keys sit in columns 16*half .. 16*half+15 of each 32-column group; zero elsewhere
       {
         uint32_t zero[16];
