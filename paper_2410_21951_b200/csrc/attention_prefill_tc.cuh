@@ -245,18 +245,25 @@ __global__ void __launch_bounds__(kPfThreads, 2) prefill_attention_tc_kernel(
       }
       l_run *= factor;
       const float m_sub = (m_use == -INFINITY) ? 0.f : m_use;
-      float psum4[4] = {0.f, 0.f, 0.f, 0.f};
+      float2 psum4[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};   // four chains of pairs
       uint32_t hv[16], lv[16];
+      const float2 sc2 = make_float2(scale_log2e, scale_log2e), nm2 = make_float2(-m_sub, -m_sub);
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
-        const float pa = fast_exp2(fmaf(sc[2 * j], scale_log2e, -m_sub));
-        const float pb = fast_exp2(fmaf(sc[2 * j + 1], scale_log2e, -m_sub));
-        psum4[j & 3] += pa + pb;
-        hv[j] = pack_bf16(pa, pb);
-        const float ha = __uint_as_float(hv[j] << 16), hb = __uint_as_float(hv[j] & 0xffff0000u);
-        lv[j] = pack_bf16(pa - ha, pb - hb);
+        // two keys per instruction where the pipe has a paired form (fma, add, sub)
+        const float2 x = ffma2(make_float2(sc[2 * j], sc[2 * j + 1]), sc2, nm2);
+        const float2 pp = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+        psum4[j & 3] = fadd2(psum4[j & 3], pp);
+        hv[j] = pack_bf16(pp.x, pp.y);
+        const float2 hh = make_float2(__uint_as_float(hv[j] << 16), __uint_as_float(hv[j] & 0xffff0000u));
+        const float2 ll = fsub2(pp, hh);
+        lv[j] = pack_bf16(ll.x, ll.y);
       }
-      l_run += (psum4[0] + psum4[1]) + (psum4[2] + psum4[3]);
+      {
+        const float2 s01 = fadd2(psum4[0], psum4[1]), s23 = fadd2(psum4[2], psum4[3]);
+        const float2 st = fadd2(s01, s23);
+        l_run += st.x + st.y;
+      }
       tmem_st16(tpp + 16 * khalf, hv);                   // keys 32 khalf .. +31: hi in columns 16 khalf .., lo in 32 + 16 khalf ..
       tmem_st16(tpp + 32 + 16 * khalf, lv);
       tmem_st_wait();
